@@ -1,0 +1,177 @@
+/*
+ * l2a.h -- C ABI of the B200 (sm_100a) hot path of the L2A conditional attention layer.
+ *
+ * The layer (paper Section 3.1, Eq. 2-5): every token gets causal sliding-window ("Local")
+ * attention s_t; tokens whose routing decision d_t = 1 additionally get exact causal ("Global")
+ * attention a_t over the full prefix; the output is o_t = s_t + d_t * a_t.  The kernel-level
+ * method (Section 3.2, Algorithm 1): routed queries are compacted into a contiguous buffer with
+ * their original positions recorded (Q_idx), attention is tiled over the compact rows with the
+ * causal mask taken from the true positions, and the result is scattered back.
+ *
+ * Conventions shared by every call
+ *   - Every pointer is a DEVICE pointer unless its comment says "host".  The caller owns all
+ *     buffers, including the workspaces; the library allocates no device memory, keeps no state
+ *     between calls, and never synchronises the stream (only l2a_workspace_status does).
+ *   - Tensors are contiguous bf16:  Q, O, dO, dQ, S_save, A_c : [B, Lq, Hq, D]
+ *                                   K, V, dK, dV              : [B, Lk, Hkv, D]
+ *     D contiguous, base pointers 16-byte aligned.  D is 64 or 128.  Hq % Hkv == 0 (GQA: query
+ *     head h reads KV head h / (Hq/Hkv)).
+ *   - Positions are 0-based.  Query row t sits at position p = t + q_pos_offset; the local
+ *     neighbourhood is max(0, p - window) <= j <= p (self plus `window` predecessors, the mask
+ *     0 <= i - j <= w of Section 2), the global neighbourhood is 0 <= j <= p.
+ *   - Routing is per token and shared by all heads (the router projection has one output, Eq. 3).
+ *   - Each call validates its arguments on the host and returns L2A_ERR_* before launching
+ *     anything; work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default).
+ *   - Device-side waits are bounded; a wait that runs out is recorded in the workspace's status
+ *     word and the kernels finish without writing further results (see l2a_workspace_status).
+ */
+#ifndef L2A_H_
+#define L2A_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  L2A_OK = 0,
+  L2A_ERR_INVALID_ARG = -1,    /* NULL pointer, bad shape, misaligned base pointer          */
+  L2A_ERR_UNSUPPORTED = -2,    /* valid request this build does not implement               */
+  L2A_ERR_WORKSPACE = -3,      /* workspace pointer NULL / misaligned / too small           */
+  L2A_ERR_CUDA = -4,           /* a CUDA runtime or driver call failed (launch, encode)     */
+  L2A_ERR_DEVICE_TIMEOUT = -5  /* a bounded device-side wait ran out (l2a_workspace_status) */
+} l2a_status;
+
+/* l2a_params.flags */
+#define L2A_FLAG_SAVE_FOR_BWD 1u  /* forward also writes S_save and A_c (needed by l2a_backward)  */
+#define L2A_FLAG_SKIP_LOCAL 2u    /* forward: no local module; O = d * A (the "SWA-0" ablation)   */
+#define L2A_FLAG_SKIP_GLOBAL 4u   /* forward: local module only; O = S (first phase of the layer, */
+                                  /* before the router has seen S)                                */
+
+/* router_kind of l2a_route_compact */
+#define L2A_ROUTER_MASK_U8 0     /* router = uint8 [B, Lq], non-zero => routed                    */
+#define L2A_ROUTER_LOGITS_F32 1  /* router = fp32 logits [B, Lq]; d = (z >= logit_threshold)      */
+
+typedef struct l2a_params {
+  int32_t B, Lq, Lk, Hq, Hkv, D;
+  int32_t window;       /* W >= 0: keys j with 0 <= p - j <= W                                    */
+  int32_t q_pos_offset; /* p = t + q_pos_offset; pass Lk - Lq for bottom-right aligned causality  */
+  float softmax_scale;  /* scores are softmax_scale * q.k ; pass 0 for the default 1/sqrt(D)      */
+  uint32_t flags;       /* L2A_FLAG_*                                                             */
+} l2a_params;
+
+/* Version / capability string of the loaded library (host pointer, static storage). */
+const char* l2a_version(void);
+
+/* Human-readable name of a status code (host pointer, static storage). */
+const char* l2a_status_string(l2a_status s);
+
+/*
+ * Workspace sizes in bytes for the three calls, for the given shape (worst case over routing:
+ * they do not depend on how many tokens are routed).  Any of the three outputs may be NULL.
+ * Workspaces must be 256-byte aligned device memory.  Contents need not be preserved between
+ * calls, except that the backward reads nothing from the forward's workspace either: everything
+ * the backward needs is passed explicitly.
+ */
+l2a_status l2a_workspace_bytes(const l2a_params* p, size_t* route_ws_bytes, size_t* fwd_ws_bytes,
+                               size_t* bwd_ws_bytes);
+
+/*
+ * Reads the status word the kernels of earlier calls left in workspace `ws` (any of the three).
+ * Synchronises `stream`.  Returns L2A_OK, or L2A_ERR_DEVICE_TIMEOUT if a bounded device-side wait
+ * ran out in some kernel that used this workspace since it was last used by a successful call.
+ */
+l2a_status l2a_workspace_status(const void* ws, void* stream);
+
+/*
+ * Routing decision and query compaction (Eq. 3; Section 3.2 "consolidated into a compact,
+ * contiguous buffer ... original sequence positions recorded"; Algorithm 1, step 1).
+ *
+ *   router      in : [B, Lq] uint8 mask or fp32 logits, per router_kind.  For logits the decision
+ *                    is taken on the logit in fp32, d = (z >= logit_threshold); threshold 0 is
+ *                    sigmoid(z) >= 0.5, the tie z == threshold routes, NaN does not.
+ *   d_mask      out: [B, Lq] uint8, 0 or 1.
+ *   q_idx       out: [B, Lq] int32.  Row b holds the routed row indices t of batch entry b in
+ *                    ascending order in its first n_routed[b] entries; the rest is -1.
+ *   n_routed    out: [B] int32 (stays on the device; nothing here reads it on the host).
+ *   prefix      out: [B, Lq + 1] int32, prefix[b][t] = number of routed rows u < t
+ *                    (the compact index of row t if it is routed); prefix[b][Lq] = n_routed[b].
+ *   route_ws       : workspace of at least route_ws_bytes.
+ * Integer results are exact.  Returns L2A_ERR_INVALID_ARG for NULL/misaligned pointers or a bad
+ * router_kind; nothing is launched in that case.
+ */
+l2a_status l2a_route_compact(const l2a_params* p, const void* router, int router_kind, float logit_threshold,
+                             uint8_t* d_mask, int32_t* q_idx, int32_t* n_routed, int32_t* prefix,
+                             void* route_ws, size_t route_ws_bytes, void* stream);
+
+/*
+ * Forward of the layer (Eq. 2, 4, 5; Algorithm 1 for the global part).
+ *
+ *   Q, K, V     in : bf16, layouts above.
+ *   d_mask, q_idx, n_routed, prefix
+ *               in : exactly as written by l2a_route_compact for the same shape.
+ *   O           out: bf16 [B, Lq, Hq, D];  O_t = S_t + d_t * A_t, rounded to bf16 once more after
+ *                    the sum for routed rows; rows with d_t = 0 are bit-identical to a run with
+ *                    no routed rows at all.
+ *   S_save      out: bf16 [B, Lq, Hq, D], the local output s_t.  Required with
+ *                    L2A_FLAG_SAVE_FOR_BWD, otherwise may be NULL.
+ *   A_c         out: bf16 [B, Lq, Hq, D] worst case; compact row c of batch b (c < n_routed[b])
+ *                    holds a_t of row t = q_idx[b][c] (Algorithm 1's O_c).  Rows >= n_routed[b]
+ *                    are not written.  Required with L2A_FLAG_SAVE_FOR_BWD, otherwise may be NULL.
+ *   lse_loc     out: fp32 [B, Hq, Lq], natural-log log-sum-exp of the local scores of row t.
+ *   lse_glb     out: fp32 [B, Hq, Lq], first n_routed[b] entries of each (b, h) row: natural-log
+ *                    log-sum-exp of the global scores of compact row c (Algorithm 1's L_c).
+ *                    Both lse outputs may be NULL unless L2A_FLAG_SAVE_FOR_BWD is set.
+ *   fwd_ws         : workspace of at least fwd_ws_bytes (holds the compact query buffer Q_c).
+ * Scores and soft-max run in fp32, probabilities are rounded to bf16 for the second contraction,
+ * accumulation is fp32.  Returns L2A_ERR_UNSUPPORTED for D not in {64, 128}.
+ */
+l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const void* V,
+                       const uint8_t* d_mask, const int32_t* q_idx, const int32_t* n_routed,
+                       const int32_t* prefix, void* O, void* S_save, void* A_c, float* lse_loc,
+                       float* lse_glb, void* fwd_ws, size_t fwd_ws_bytes, void* stream);
+
+/*
+ * Backward of the layer: the vector-Jacobian product of l2a_forward with the routing mask held
+ * fixed (Section 3.2: gradients only for active queries in the global part, reusing L_c and Q_idx;
+ * the local part is a sliding-window attention backward).  With one Q/K/V set feeding both
+ * modules, dQ_t = dQ_loc,t + d_t * dQ_glb,t and dK, dV sum both modules' contributions and the
+ * query heads of each KV group.
+ *
+ *   Q, K, V, d_mask, q_idx, n_routed, prefix : as given to l2a_forward.
+ *   dO          in : bf16 [B, Lq, Hq, D], gradient of the loss w.r.t. O.
+ *   S_save, A_c, lse_loc, lse_glb
+ *               in : as written by l2a_forward with L2A_FLAG_SAVE_FOR_BWD.
+ *   dQ          out: bf16 [B, Lq, Hq, D].
+ *   dK, dV      out: bf16 [B, Lk, Hkv, D].
+ *   dgate       out: optional fp32 [B, Lq] (may be NULL): sum over heads of dO_t . a_t for routed
+ *                    rows, 0 elsewhere -- the loss-dependent term of the straight-through router
+ *                    gradient (Eq. 7) for the rows whose global output was computed.
+ *   bwd_ws         : workspace of at least bwd_ws_bytes.
+ */
+l2a_status l2a_backward(const l2a_params* p, const void* Q, const void* K, const void* V,
+                        const uint8_t* d_mask, const int32_t* q_idx, const int32_t* n_routed,
+                        const int32_t* prefix, const void* dO, const void* S_save, const void* A_c,
+                        const float* lse_loc, const float* lse_glb, void* dQ, void* dK, void* dV,
+                        float* dgate, void* bwd_ws, size_t bwd_ws_bytes, void* stream);
+
+/*
+ * Convenience for callers that hold HOST buffers: copies Q, K, V and the router input to the
+ * device buffers the caller supplies, runs l2a_route_compact + l2a_forward, copies O back, and
+ * synchronises the stream.  All `h_` pointers are host memory (pinned memory gives asynchronous
+ * copies), all `d_` pointers device memory of the sizes the corresponding arguments above need.
+ * Exists so that end-to-end time including the transfers can be measured through the C ABI.
+ */
+l2a_status l2a_forward_host(const l2a_params* p, const void* h_Q, const void* h_K, const void* h_V,
+                            const void* h_router, int router_kind, float logit_threshold, void* h_O,
+                            void* d_Q, void* d_K, void* d_V, void* d_router, uint8_t* d_mask,
+                            int32_t* d_q_idx, int32_t* d_n_routed, int32_t* d_prefix, void* d_O,
+                            void* route_ws, size_t route_ws_bytes, void* fwd_ws, size_t fwd_ws_bytes,
+                            void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* L2A_H_ */

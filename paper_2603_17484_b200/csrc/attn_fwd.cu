@@ -1,0 +1,415 @@
+// Forward attention kernel for sm_100a: one kernel, two modes.
+//
+//   local  mode (Eq. 2, sliding-window mask of Section 2): query rows are sequence rows; key blocks
+//          wholly outside the band [p - W, p] are never loaded.
+//   global mode (Eq. 4; Algorithm 1): query rows are the compacted routed rows (Q_c); the causal
+//          mask uses the true position Q_idx of each compact row; the key loop of a tile stops at
+//          the block holding its largest position; the epilogue scatters the result to O by
+//          position and combines it with the local output already there (Eq. 5), and also stores
+//          the compact output O_c and log-sum-exp L_c.
+//
+// Structure (per CTA: two 128-row query tiles of one head, sharing the K/V stream):
+//   warps 0-3 / 4-7 : soft-max + correction + epilogue of tile 0 / 1 (one thread per query row)
+//   warp 8          : TMA producer (Q once; K and V blocks through 2-stage rings)
+//   warp 9          : tcgen05 MMA issuer and TMEM owner
+//   TMEM (512 cols) : S0 | S1 | O0 | O1 (fp32); the bf16 probabilities P overwrite the first half
+//                     of their own S columns and are consumed from TMEM as the A operand of P*V.
+// While one tile's soft-max runs on the CUDA cores, the tensor core works on the other tile.
+// The online soft-max follows Algorithm 1 (running max m, running sum l, rescaled accumulator),
+// in the exp2 domain, with the rescale skipped while the maximum grows by less than 2^8.
+#include "l2a_common.cuh"
+#include "sm100_prims.cuh"
+
+namespace l2a {
+
+namespace {
+
+constexpr int kNumTiles = 2;
+constexpr int kStages = 2;
+constexpr int kFwdThreads = 320;
+constexpr float kRescaleThreshold = 8.0f;  // log2 units
+
+template <int D>
+struct FwdSmem {
+  static constexpr int kQTileBytes = kTileM * D * 2;
+  static constexpr int kKVTileBytes = kTileN * D * 2;
+  static constexpr int kBoxBytes = 128 * 128;  // one TMA box: 128 rows x 64 bf16 (128 B)
+  static constexpr int kQOff = 0;
+  static constexpr int kKOff = kQOff + kNumTiles * kQTileBytes;
+  static constexpr int kVOff = kKOff + kStages * kKVTileBytes;
+  static constexpr int kBarOff = kVOff + kStages * kKVTileBytes;
+  static constexpr int kTotal = kBarOff + 256 + 1024 /* alignment slack */;
+};
+
+struct Barriers {
+  uint64_t q_full[kNumTiles];
+  uint64_t k_full[kStages], k_empty[kStages];
+  uint64_t v_full[kStages], v_empty[kStages];
+  uint64_t s_full[kNumTiles];
+  uint64_t p_full[kNumTiles];
+  uint64_t o_final;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+struct TileRange {
+  int active;    // tile has at least one valid row
+  int min_pos, max_pos;
+  int lo, hi;    // first / last key block
+};
+
+template <int D>
+__global__ void __launch_bounds__(kFwdThreads, 1)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                const __grid_constant__ CUtensorMap mapV, const FwdArgs a) {
+  using SM = FwdSmem<D>;
+  constexpr int kDBoxes = D / 64;      // 64-element boxes per row
+  constexpr int kKSteps = D / 16;      // MMA k-steps of Q*K^T
+  constexpr int kOCol0 = 2 * kTileN;   // first TMEM column of the O accumulators
+
+  // ---- work item: heaviest first (largest row index first), heads fastest for K/V reuse in L2
+  const int n_pairs = (a.Lq + kRowsPerCta - 1) / kRowsPerCta;
+  const int h = blockIdx.x % a.Hq;
+  const int rest = blockIdx.x / a.Hq;
+  const int b = rest % a.B;
+  const int pi = n_pairs - 1 - rest / a.B;
+  const int g = h / (a.Hq / a.Hkv);
+  const int n_rows = a.global_mode ? a.n_routed[b] : a.Lq;  // valid (compact) rows of this batch entry
+  const int row0 = pi * kRowsPerCta;
+  if (row0 >= n_rows) return;
+
+  const int32_t* q_idx_b = a.q_idx + (int64_t)b * a.Lq;
+  const int w_eff = a.global_mode ? 0x3fffffff : a.window;
+
+  TileRange tr[kNumTiles];
+  int jlo = 0x7fffffff, jhi = -1;
+#pragma unroll
+  for (int t = 0; t < kNumTiles; ++t) {
+    const int first = row0 + t * kTileM;
+    int last = first + kTileM - 1;
+    if (last > n_rows - 1) last = n_rows - 1;
+    tr[t].active = first < n_rows;
+    if (tr[t].active) {
+      tr[t].min_pos = (a.global_mode ? q_idx_b[first] : first) + a.q_pos_offset;
+      tr[t].max_pos = (a.global_mode ? q_idx_b[last] : last) + a.q_pos_offset;
+      const int lo_pos = tr[t].min_pos - w_eff;
+      tr[t].lo = lo_pos > 0 ? lo_pos / kTileN : 0;
+      tr[t].hi = tr[t].max_pos / kTileN;
+      jlo = min(jlo, tr[t].lo);
+      jhi = max(jhi, tr[t].hi);
+    } else {
+      tr[t].min_pos = tr[t].max_pos = 0;
+      tr[t].lo = 1; tr[t].hi = 0;
+    }
+  }
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sQ = smem + SM::kQOff;
+  uint8_t* sK = smem + SM::kKOff;
+  uint8_t* sV = smem + SM::kVOff;
+  Barriers* bar = reinterpret_cast<Barriers*>(smem + SM::kBarOff);
+  volatile int* abort_flag = &bar->abort_flag;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  if (tid == 0) {
+    for (int t = 0; t < kNumTiles; ++t) {
+      mbar_init(&bar->q_full[t], 1);
+      mbar_init(&bar->s_full[t], 1);
+      mbar_init(&bar->p_full[t], kTileM);
+    }
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&bar->k_full[s], 1);
+      mbar_init(&bar->k_empty[s], 1);
+      mbar_init(&bar->v_full[s], 1);
+      mbar_init(&bar->v_empty[s], 1);
+    }
+    mbar_init(&bar->o_final, 1);
+    bar->abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 9) {
+    tmem_alloc(&bar->tmem_base, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bar->tmem_base;
+
+  if (warp == 8) {
+    // =========================================================================== TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&mapQ);
+      tma_prefetch_desc(&mapK);
+      tma_prefetch_desc(&mapV);
+      for (int t = 0; t < kNumTiles; ++t) {
+        if (!tr[t].active) continue;
+        mbar_expect_tx(&bar->q_full[t], SM::kQTileBytes);
+        for (int x = 0; x < kDBoxes; ++x)
+          tma_load_3d(sQ + t * SM::kQTileBytes + x * SM::kBoxBytes, &mapQ, &bar->q_full[t], h * D + x * 64,
+                      row0 + t * kTileM, b);
+      }
+      for (int j = jlo; j <= jhi; ++j) {
+        const int it = j - jlo, s = it % kStages;
+        const uint32_t ph = (it / kStages) & 1;
+        if (!mbar_wait(&bar->k_empty[s], ph ^ 1, abort_flag)) break;
+        mbar_expect_tx(&bar->k_full[s], SM::kKVTileBytes);
+        for (int x = 0; x < kDBoxes; ++x)
+          tma_load_3d(sK + s * SM::kKVTileBytes + x * SM::kBoxBytes, &mapK, &bar->k_full[s], g * D + x * 64,
+                      j * kTileN, b);
+        if (!mbar_wait(&bar->v_empty[s], ph ^ 1, abort_flag)) break;
+        mbar_expect_tx(&bar->v_full[s], SM::kKVTileBytes);
+        for (int x = 0; x < kDBoxes; ++x)
+          tma_load_3d(sV + s * SM::kKVTileBytes + x * SM::kBoxBytes, &mapV, &bar->v_full[s], g * D + x * 64,
+                      j * kTileN, b);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 9) {
+    // =========================================================================== MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = idesc_bf16_f32(kTileM, kTileN, 0, 0);
+      constexpr uint32_t idesc_pv = idesc_bf16_f32(kTileM, D, 0, 1);
+      uint32_t p_cnt[kNumTiles] = {0, 0};
+      bool ok = true;
+
+      auto issue_qk = [&](int t, int j) {
+        const int s = (j - jlo) % kStages;
+        const uint32_t qa = smem_u32(sQ + t * SM::kQTileBytes);
+        const uint32_t ka = smem_u32(sK + s * SM::kKVTileBytes);
+#pragma unroll
+        for (int kk = 0; kk < kKSteps; ++kk) {
+          const uint32_t off = (kk >> 2) * SM::kBoxBytes + (kk & 3) * 32;
+          mma_ss(tmem + t * kTileN, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(ka + off, 16, 1024),
+                 idesc_qk, kk > 0);
+        }
+        tc_commit(&bar->s_full[t]);
+      };
+      auto in_range = [&](int t, int j) { return tr[t].active && j >= tr[t].lo && j <= tr[t].hi; };
+
+      // first key block: Q*K^T for both tiles
+      if (!mbar_wait(&bar->k_full[0], 0, abort_flag)) ok = false;
+      for (int t = 0; ok && t < kNumTiles; ++t) {
+        if (!in_range(t, jlo)) continue;
+        if (!mbar_wait(&bar->q_full[t], 0, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        issue_qk(t, jlo);
+      }
+      if (ok) tc_commit(&bar->k_empty[0]);
+
+      for (int j = jlo; ok && j <= jhi; ++j) {
+        const int it = j - jlo, s = it % kStages;
+        const uint32_t ph = (it / kStages) & 1;
+        const int sn = (it + 1) % kStages;
+        const uint32_t phn = ((it + 1) / kStages) & 1;
+        bool v_ready = false, k_ready = false;
+        for (int t = 0; ok && t < kNumTiles; ++t) {
+          if (in_range(t, j)) {
+            if (!mbar_wait(&bar->p_full[t], p_cnt[t] & 1, abort_flag)) { ok = false; break; }
+            ++p_cnt[t];
+            if (!v_ready) {
+              if (!mbar_wait(&bar->v_full[s], ph, abort_flag)) { ok = false; break; }
+              v_ready = true;
+            }
+            tc_fence_after();
+            const uint32_t va = smem_u32(sV + s * SM::kKVTileBytes);
+#pragma unroll
+            for (int kk = 0; kk < kTileN / 16; ++kk)
+              mma_ts(tmem + kOCol0 + t * D, tmem + t * kTileN + kk * 8,
+                     smem_desc_sw128(va + kk * 2048, SM::kBoxBytes, 1024), idesc_pv, (j > tr[t].lo) || (kk > 0));
+          }
+          if (j + 1 <= jhi && in_range(t, j + 1)) {
+            if (!k_ready) {
+              if (!mbar_wait(&bar->k_full[sn], phn, abort_flag)) { ok = false; break; }
+              k_ready = true;
+            }
+            if (j + 1 == tr[t].lo && !mbar_wait(&bar->q_full[t], 0, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            issue_qk(t, j + 1);
+          }
+        }
+        if (!ok) break;
+        // V block j is released once both tiles' P*V have drained; K block j+1 once both Q*K^T have
+        if (!v_ready && !mbar_wait(&bar->v_full[s], ph, abort_flag)) break;
+        tc_commit(&bar->v_empty[s]);
+        if (j + 1 <= jhi) {
+          if (!k_ready && !mbar_wait(&bar->k_full[sn], phn, abort_flag)) break;
+          tc_commit(&bar->k_empty[sn]);
+        }
+      }
+      if (ok) tc_commit(&bar->o_final);
+    }
+    __syncwarp();
+  } else {
+    // =========================================================================== soft-max warpgroups
+    const int t = warp >> 2;                 // tile of this warpgroup
+    const int r = (warp & 3) * 32 + lane;    // row inside the tile == TMEM lane
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const uint32_t s_addr = tmem + lane_base + t * kTileN;
+    const uint32_t o_addr = tmem + lane_base + kOCol0 + t * D;
+    if (tr[t].active) {
+      const int row = row0 + t * kTileM + r;           // sequence row (local) or compact row (global)
+      const bool valid = row < n_rows;
+      const int seq_row = valid ? (a.global_mode ? q_idx_b[row] : row) : -1;
+      const int pos = valid ? seq_row + a.q_pos_offset : -1;
+      const int pos_lo = valid ? (pos - w_eff) : 0x7fffffff;   // smallest visible key position
+      float m_use = -INFINITY;   // reference maximum, exp2 domain
+      float l = 0.f;
+      bool ok = true;
+      const int n_my = tr[t].hi - tr[t].lo + 1;
+
+      for (int i = 0; i < n_my; ++i) {
+        const int j = tr[t].lo + i;
+        // warp-uniform outcome: the TMEM loads/stores below are warp-collective
+        if (!__all_sync(0xffffffffu, mbar_wait(&bar->s_full[t], i & 1, abort_flag))) { ok = false; break; }
+        tc_fence_after();
+        float s[kTileN];
+#pragma unroll
+        for (int c = 0; c < kTileN / 32; ++c) {
+          uint32_t v[32];
+          tmem_ld32(s_addr + c * 32, v);
+#pragma unroll
+          for (int e = 0; e < 32; ++e) s[c * 32 + e] = __uint_as_float(v[e]);
+        }
+        tmem_ld_wait();
+
+        const int k0 = j * kTileN;
+        const bool partial = (k0 + kTileN - 1 > tr[t].min_pos) || (k0 < tr[t].max_pos - w_eff);
+        if (partial) {
+#pragma unroll
+          for (int e = 0; e < kTileN; ++e) {
+            const int kp = k0 + e;
+            s[e] = (kp <= pos && kp >= pos_lo) ? s[e] : -INFINITY;
+          }
+        }
+        float mx = s[0];
+#pragma unroll
+        for (int e = 1; e < kTileN; ++e) mx = fmaxf(mx, s[e]);
+        const float m_new = fmaxf(m_use, mx * a.scale_log2);
+
+        // correction: rescale the running sum and the TMEM accumulator only when the maximum moved a lot
+        const bool need = (i == 0) ? false : (m_new - m_use > kRescaleThreshold);
+        if (i == 0) m_use = m_new;
+        if (__any_sync(0xffffffffu, need)) {
+          const float alpha = need ? fast_exp2(m_use - m_new) : 1.0f;
+          l *= alpha;
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t v[32];
+            tmem_ld32(o_addr + c * 32, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
+            tmem_st32(o_addr + c * 32, v);
+          }
+          if (need) m_use = m_new;
+        }
+        const float m_eff = (m_use == -INFINITY) ? 0.f : m_use;
+        const float neg_m = -m_eff;
+        float sum = 0.f;
+#pragma unroll
+        for (int c = 0; c < kTileN / 64; ++c) {
+          uint32_t pk[32];
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            const float p0 = fast_exp2(fmaf(s[c * 64 + 2 * e], a.scale_log2, neg_m));
+            const float p1 = fast_exp2(fmaf(s[c * 64 + 2 * e + 1], a.scale_log2, neg_m));
+            sum += p0 + p1;
+            pk[e] = pack_bf16(p0, p1);
+          }
+          tmem_st32(s_addr + c * 32, pk);
+        }
+        l += sum;
+        tmem_st_wait();
+        tc_fence_before();
+        mbar_arrive(&bar->p_full[t]);
+      }
+
+      // ---- epilogue: O / l, log-sum-exp, store (local) or scatter + combine (global)
+      if (ok && __all_sync(0xffffffffu, mbar_wait(&bar->o_final, 0, abort_flag))) {
+        tc_fence_after();
+        const float inv_l = (l > 0.f) ? 1.0f / l : 0.f;
+        if (valid && a.lse != nullptr) {
+          const float lse = (m_use + log2f(l)) * 0.6931471805599453f;
+          a.lse[((int64_t)b * a.Hq + h) * a.Lq + row] = lse;
+        }
+        const int64_t row_stride = (int64_t)a.Hq * D;
+        bf16* dst1 = nullptr;   // row-indexed destination (s rows, or compact a rows)
+        bf16* dst2 = nullptr;   // position-indexed destination
+        if (valid) {
+          if (a.out) dst1 = a.out + ((int64_t)b * a.Lq + row) * row_stride + (int64_t)h * D;
+          if (a.out2) dst2 = a.out2 + ((int64_t)b * a.Lq + seq_row) * row_stride + (int64_t)h * D;
+        }
+        const bool accumulate = a.global_mode && a.accumulate_into_out2;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t v[32];
+          tmem_ld32(o_addr + c * 32, v);
+          tmem_ld_wait();
+          float f[32];
+#pragma unroll
+          for (int e = 0; e < 32; ++e) f[e] = __uint_as_float(v[e]) * inv_l;
+          if (dst1) {
+            uint4* d4 = reinterpret_cast<uint4*>(dst1 + c * 32);
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              d4[q] = make_uint4(pack_bf16(f[8 * q], f[8 * q + 1]), pack_bf16(f[8 * q + 2], f[8 * q + 3]),
+                                 pack_bf16(f[8 * q + 4], f[8 * q + 5]), pack_bf16(f[8 * q + 6], f[8 * q + 7]));
+          }
+          if (dst2) {
+            uint4* d4 = reinterpret_cast<uint4*>(dst2 + c * 32);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              if (accumulate) {
+                const uint4 old = d4[q];
+                const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  f[8 * q + 2 * k] += __uint_as_float(ow[k] << 16);
+                  f[8 * q + 2 * k + 1] += __uint_as_float(ow[k] & 0xffff0000u);
+                }
+              }
+              d4[q] = make_uint4(pack_bf16(f[8 * q], f[8 * q + 1]), pack_bf16(f[8 * q + 2], f[8 * q + 3]),
+                                 pack_bf16(f[8 * q + 4], f[8 * q + 5]), pack_bf16(f[8 * q + 6], f[8 * q + 7]));
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // ---- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (bar->abort_flag) {
+    // a bounded wait ran out: give copies still in flight time to land before shared memory is released
+    const uint64_t t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    if (tid == 0) atomicExch(a.status, 1);
+    __syncthreads();
+  }
+  if (warp == 9) tmem_dealloc(tmem, 512);
+}
+
+}  // namespace
+
+cudaError_t launch_attn_fwd(const FwdArgs& a, const CUtensorMap& mapQ, const CUtensorMap& mapK,
+                            const CUtensorMap& mapV, cudaStream_t stream) {
+  const int n_pairs = (a.Lq + kRowsPerCta - 1) / kRowsPerCta;
+  const unsigned grid = (unsigned)n_pairs * a.Hq * a.B;
+  cudaError_t e;
+  if (a.D == 128) {
+    e = cudaFuncSetAttribute(attn_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<128>::kTotal);
+    if (e != cudaSuccess) return e;
+    attn_fwd_kernel<128><<<grid, kFwdThreads, FwdSmem<128>::kTotal, stream>>>(mapQ, mapK, mapV, a);
+  } else {
+    e = cudaFuncSetAttribute(attn_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<64>::kTotal);
+    if (e != cudaSuccess) return e;
+    attn_fwd_kernel<64><<<grid, kFwdThreads, FwdSmem<64>::kTotal, stream>>>(mapQ, mapK, mapV, a);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace l2a

@@ -1,0 +1,232 @@
+// C ABI of libl2a.so: argument validation, workspace layout, tensor-map encoding, launch order.
+// Every step of the path runs in the CUDA kernels; nothing here computes on the host and there is
+// no fallback path.
+#include <math.h>
+#include <string.h>
+
+#include "l2a_common.cuh"
+
+namespace l2a {
+
+namespace {
+
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+encode_tiled_fn get_encode() {
+  static encode_tiled_fn fn = []() -> encode_tiled_fn {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) return nullptr;
+    if (q != cudaDriverEntryPointSuccess) return nullptr;
+    return reinterpret_cast<encode_tiled_fn>(p);
+  }();
+  return fn;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+l2a_status check_params(const l2a_params* p) {
+  if (!p) return L2A_ERR_INVALID_ARG;
+  if (p->B <= 0 || p->Lq <= 0 || p->Lk <= 0 || p->Hq <= 0 || p->Hkv <= 0 || p->D <= 0) return L2A_ERR_INVALID_ARG;
+  if (p->Hq % p->Hkv != 0) return L2A_ERR_INVALID_ARG;
+  if (p->window < 0) return L2A_ERR_INVALID_ARG;
+  if (p->q_pos_offset < 0 || (int64_t)p->Lq + p->q_pos_offset > p->Lk) return L2A_ERR_INVALID_ARG;
+  if (!(p->softmax_scale >= 0.f) || isinf(p->softmax_scale)) return L2A_ERR_INVALID_ARG;
+  if ((int64_t)p->B * p->Lq >= (1ll << 31) || (int64_t)p->B * p->Lk >= (1ll << 31)) return L2A_ERR_INVALID_ARG;
+  if (p->D != 64 && p->D != 128) return L2A_ERR_UNSUPPORTED;
+  return L2A_OK;
+}
+
+float scale_of(const l2a_params* p) { return p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->D); }
+
+size_t route_ws_size(const l2a_params* p) {
+  const int nblocks = ceil_div(p->Lq, kRouteBlockElems);
+  return kWsHeaderBytes + align_up((size_t)p->B * nblocks * sizeof(int32_t), 256);
+}
+size_t qrows_bytes(const l2a_params* p) { return align_up((size_t)p->B * p->Lq * p->Hq * p->D * sizeof(bf16), 256); }
+size_t fwd_ws_size(const l2a_params* p) { return kWsHeaderBytes + qrows_bytes(p); }
+
+bool ws_ok(const void* ws, size_t have, size_t need) { return ws && aligned(ws, 256) && have >= need; }
+
+}  // namespace
+
+bool encode_rows_map(CUtensorMap* map, const void* base, int batch, int rows, int row_elems, int box_rows) {
+  encode_tiled_fn enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)row_elems, (cuuint64_t)rows, (cuuint64_t)batch};
+  cuuint64_t strides[2] = {(cuuint64_t)row_elems * 2, (cuuint64_t)rows * row_elems * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+}  // namespace l2a
+
+using namespace l2a;
+
+extern "C" {
+
+const char* l2a_version(void) { return "l2a-b200 0.1 (sm_100a; tcgen05/TMEM/TMA)"; }
+
+const char* l2a_status_string(l2a_status s) {
+  switch (s) {
+    case L2A_OK: return "ok";
+    case L2A_ERR_INVALID_ARG: return "invalid argument";
+    case L2A_ERR_UNSUPPORTED: return "unsupported configuration";
+    case L2A_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case L2A_ERR_CUDA: return "CUDA call failed";
+    case L2A_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+  }
+  return "unknown status";
+}
+
+l2a_status l2a_workspace_bytes(const l2a_params* p, size_t* route_ws_bytes, size_t* fwd_ws_bytes,
+                               size_t* bwd_ws_bytes) {
+  l2a_status st = check_params(p);
+  if (st != L2A_OK) return st;
+  if (route_ws_bytes) *route_ws_bytes = route_ws_size(p);
+  if (fwd_ws_bytes) *fwd_ws_bytes = fwd_ws_size(p);
+  if (bwd_ws_bytes) *bwd_ws_bytes = l2a::bwd_ws_size(p);
+  return L2A_OK;
+}
+
+l2a_status l2a_workspace_status(const void* ws, void* stream) {
+  if (!ws) return L2A_ERR_INVALID_ARG;
+  int word = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(&word, ws, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return L2A_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return L2A_ERR_CUDA;
+  return word == 0 ? L2A_OK : L2A_ERR_DEVICE_TIMEOUT;
+}
+
+l2a_status l2a_route_compact(const l2a_params* p, const void* router, int router_kind, float logit_threshold,
+                             uint8_t* d_mask, int32_t* q_idx, int32_t* n_routed, int32_t* prefix, void* route_ws,
+                             size_t route_ws_bytes, void* stream) {
+  l2a_status st = check_params(p);
+  if (st != L2A_OK) return st;
+  if (!router || !d_mask || !q_idx || !n_routed || !prefix) return L2A_ERR_INVALID_ARG;
+  if (router_kind != L2A_ROUTER_MASK_U8 && router_kind != L2A_ROUTER_LOGITS_F32) return L2A_ERR_INVALID_ARG;
+  if (!aligned(q_idx, 4) || !aligned(n_routed, 4) || !aligned(prefix, 4)) return L2A_ERR_INVALID_ARG;
+  if (router_kind == L2A_ROUTER_LOGITS_F32 && !aligned(router, 4)) return L2A_ERR_INVALID_ARG;
+  if (!ws_ok(route_ws, route_ws_bytes, route_ws_size(p))) return L2A_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(route_ws, 0, kWsHeaderBytes, s) != cudaSuccess) return L2A_ERR_CUDA;
+  RouteArgs a;
+  a.router = router;
+  a.router_kind = router_kind;
+  a.threshold = logit_threshold;
+  a.B = p->B;
+  a.L = p->Lq;
+  a.d_mask = d_mask;
+  a.q_idx = q_idx;
+  a.n_routed = n_routed;
+  a.prefix = prefix;
+  a.block_sums = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(route_ws) + kWsHeaderBytes);
+  a.nblocks = ceil_div(p->Lq, kRouteBlockElems);
+  return launch_route_compact(a, s) == cudaSuccess ? L2A_OK : L2A_ERR_CUDA;
+}
+
+l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const void* V, const uint8_t* d_mask,
+                       const int32_t* q_idx, const int32_t* n_routed, const int32_t* prefix, void* O, void* S_save,
+                       void* A_c, float* lse_loc, float* lse_glb, void* fwd_ws, size_t fwd_ws_bytes, void* stream) {
+  l2a_status st = check_params(p);
+  if (st != L2A_OK) return st;
+  const bool save = p->flags & L2A_FLAG_SAVE_FOR_BWD;
+  const bool skip_local = p->flags & L2A_FLAG_SKIP_LOCAL;
+  const bool skip_global = p->flags & L2A_FLAG_SKIP_GLOBAL;
+  if (skip_local && skip_global) return L2A_ERR_INVALID_ARG;
+  if (!Q || !K || !V || !O) return L2A_ERR_INVALID_ARG;
+  if (!skip_global && (!d_mask || !q_idx || !n_routed || !prefix)) return L2A_ERR_INVALID_ARG;
+  if (save && (!S_save || !A_c || !lse_loc || !lse_glb)) return L2A_ERR_INVALID_ARG;
+  if (save && (skip_local || skip_global)) return L2A_ERR_INVALID_ARG;
+  if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || !aligned(S_save, 16) ||
+      !aligned(A_c, 16) || !aligned(lse_loc, 4) || !aligned(lse_glb, 4))
+    return L2A_ERR_INVALID_ARG;
+  if (!ws_ok(fwd_ws, fwd_ws_bytes, fwd_ws_size(p))) return L2A_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(fwd_ws);
+  int* status = reinterpret_cast<int*>(ws);
+  bf16* Qc = reinterpret_cast<bf16*>(ws + kWsHeaderBytes);
+  if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, s) != cudaSuccess) return L2A_ERR_CUDA;
+
+  CUtensorMap mapQ, mapK, mapV, mapQc;
+  if (!encode_rows_map(&mapQ, Q, p->B, p->Lq, p->Hq * p->D, kTileM) ||
+      !encode_rows_map(&mapK, K, p->B, p->Lk, p->Hkv * p->D, kTileN) ||
+      !encode_rows_map(&mapV, V, p->B, p->Lk, p->Hkv * p->D, kTileN) ||
+      !encode_rows_map(&mapQc, Qc, p->B, p->Lq, p->Hq * p->D, kTileM))
+    return L2A_ERR_CUDA;
+
+  FwdArgs a;
+  a.B = p->B; a.Lq = p->Lq; a.Lk = p->Lk; a.Hq = p->Hq; a.Hkv = p->Hkv; a.D = p->D;
+  a.window = p->window;
+  a.q_pos_offset = p->q_pos_offset;
+  a.scale_log2 = scale_of(p) * 1.4426950408889634f;
+  a.q_idx = q_idx;
+  a.n_routed = n_routed;
+  a.status = status;
+
+  if (!skip_global) {
+    // consolidate routed query rows (Algorithm 1, step 1); independent of the local pass
+    if (launch_gather_rows(static_cast<const bf16*>(Q), Qc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s) !=
+        cudaSuccess)
+      return L2A_ERR_CUDA;
+  }
+  if (!skip_local) {
+    a.global_mode = 0;
+    a.accumulate_into_out2 = 0;
+    a.out = static_cast<bf16*>(save ? S_save : O);
+    a.out2 = save ? static_cast<bf16*>(O) : nullptr;
+    a.lse = lse_loc;
+    if (launch_attn_fwd(a, mapQ, mapK, mapV, s) != cudaSuccess) return L2A_ERR_CUDA;
+  } else {
+    const size_t bytes = (size_t)p->B * p->Lq * p->Hq * p->D * sizeof(bf16);
+    if (cudaMemsetAsync(O, 0, bytes, s) != cudaSuccess) return L2A_ERR_CUDA;  // Algorithm 1: O starts at zero
+  }
+  if (!skip_global) {
+    a.global_mode = 1;
+    a.accumulate_into_out2 = skip_local ? 0 : 1;
+    a.out = static_cast<bf16*>(A_c);
+    a.out2 = static_cast<bf16*>(O);
+    a.lse = lse_glb;
+    if (launch_attn_fwd(a, mapQc, mapK, mapV, s) != cudaSuccess) return L2A_ERR_CUDA;
+  }
+  return L2A_OK;
+}
+
+l2a_status l2a_forward_host(const l2a_params* p, const void* h_Q, const void* h_K, const void* h_V,
+                            const void* h_router, int router_kind, float logit_threshold, void* h_O, void* d_Q,
+                            void* d_K, void* d_V, void* d_router, uint8_t* d_mask, int32_t* d_q_idx,
+                            int32_t* d_n_routed, int32_t* d_prefix, void* d_O, void* route_ws, size_t route_ws_bytes,
+                            void* fwd_ws, size_t fwd_ws_bytes, void* stream) {
+  l2a_status st = check_params(p);
+  if (st != L2A_OK) return st;
+  if (!h_Q || !h_K || !h_V || !h_router || !h_O || !d_Q || !d_K || !d_V || !d_router || !d_O)
+    return L2A_ERR_INVALID_ARG;
+  if (router_kind != L2A_ROUTER_MASK_U8 && router_kind != L2A_ROUTER_LOGITS_F32) return L2A_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t qb = (size_t)p->B * p->Lq * p->Hq * p->D * sizeof(bf16);
+  const size_t kb = (size_t)p->B * p->Lk * p->Hkv * p->D * sizeof(bf16);
+  const size_t rb = (size_t)p->B * p->Lq * (router_kind == L2A_ROUTER_MASK_U8 ? 1 : 4);
+  if (cudaMemcpyAsync(d_router, h_router, rb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
+  if (cudaMemcpyAsync(d_Q, h_Q, qb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
+  if (cudaMemcpyAsync(d_K, h_K, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
+  if (cudaMemcpyAsync(d_V, h_V, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
+  st = l2a_route_compact(p, d_router, router_kind, logit_threshold, d_mask, d_q_idx, d_n_routed, d_prefix, route_ws,
+                         route_ws_bytes, stream);
+  if (st != L2A_OK) return st;
+  l2a_params q = *p;
+  q.flags &= ~L2A_FLAG_SAVE_FOR_BWD;
+  st = l2a_forward(&q, d_Q, d_K, d_V, d_mask, d_q_idx, d_n_routed, d_prefix, d_O, nullptr, nullptr, nullptr, nullptr,
+                   fwd_ws, fwd_ws_bytes, stream);
+  if (st != L2A_OK) return st;
+  if (cudaMemcpyAsync(h_O, d_O, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return L2A_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return L2A_ERR_CUDA;
+  return L2A_OK;
+}
+
+}  // extern "C"

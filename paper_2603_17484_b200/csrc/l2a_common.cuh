@@ -1,0 +1,66 @@
+// Internal declarations shared by the translation units of libl2a.so (not part of the C ABI).
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/l2a.h"
+
+namespace l2a {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int kTileM = 128;         // query rows per MMA tile
+constexpr int kTileN = 128;         // keys per KV block
+constexpr int kRowsPerCta = 256;    // two query tiles per CTA in the forward / dQ kernels
+constexpr size_t kWsHeaderBytes = 256;  // every workspace starts with a header; word 0 = status
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Host-side: resolved driver entry point for cuTensorMapEncodeTiled, and a helper that encodes a
+// [batch, rows, heads*D] bf16 tensor as a 3-D map with a {64 elements, box_rows, 1} box and the
+// 128-byte swizzle the MMA operand descriptors expect.  Returns false on failure.
+bool encode_rows_map(CUtensorMap* map, const void* base, int batch, int rows, int row_elems, int box_rows);
+
+// Launchers (each returns the CUDA error of its launch).  Defined in the kernel files.
+struct RouteArgs {
+  const void* router;
+  int router_kind;
+  float threshold;
+  int B, L;
+  uint8_t* d_mask;
+  int32_t* q_idx;
+  int32_t* n_routed;
+  int32_t* prefix;
+  int32_t* block_sums;  // workspace: [B, nblocks]
+  int nblocks;
+};
+constexpr int kRouteBlockElems = 4096;  // positions per CTA of the route/compact kernels
+cudaError_t launch_route_compact(const RouteArgs& a, cudaStream_t stream);
+
+// Gathers rows src[b, q_idx[b][c], :] -> dst[b, c, :] for c < n_routed[b], and zero-fills rows up to
+// the next multiple of kRowsPerCta (bounded by L) so that padded MMA tiles read zeros.
+cudaError_t launch_gather_rows(const bf16* src, bf16* dst, const int32_t* q_idx, const int32_t* n_routed,
+                               int B, int L, int row_elems, cudaStream_t stream);
+
+struct FwdArgs {
+  int B, Lq, Lk, Hq, Hkv, D;
+  int window, q_pos_offset;
+  float scale_log2;         // softmax_scale * log2(e)
+  int global_mode;          // 0: local banded attention over all rows; 1: global attention over compact rows
+  int accumulate_into_out2; // global mode: out2[row] = out2[row] + a (1) or out2[row] = a (0)
+  const int32_t* q_idx;
+  const int32_t* n_routed;
+  bf16* out;    // local: s rows [B,Lq,Hq,D];  global: compact a rows (A_c) or NULL
+  bf16* out2;   // local: optional second copy of s (NULL to skip);  global: O rows, indexed by position
+  float* lse;   // local: [B,Hq,Lq] by row;  global: [B,Hq,Lq] by compact row; may be NULL
+  int* status;  // workspace status word
+};
+size_t bwd_ws_size(const l2a_params* p);  // defined with the backward
+
+cudaError_t launch_attn_fwd(const FwdArgs& a, const CUtensorMap& mapQ, const CUtensorMap& mapK,
+                            const CUtensorMap& mapV, cudaStream_t stream);
+
+}  // namespace l2a

@@ -1,0 +1,158 @@
+// Routing decision + query compaction (Eq. 3; Section 3.2; Algorithm 1 step 1), and the row gather
+// that consolidates routed rows into a contiguous buffer.
+//
+// Two small launches, both HBM/latency bound:
+//   route_count : each CTA thresholds 4096 positions and counts its routed ones (ballot + popc)
+//   route_scan  : each CTA sums the counts of the CTAs before it, rescans its own 4096 positions
+//                 (per-thread popcount of a 16-bit flag word, warp shuffle scan, cross-warp scan)
+//                 and writes d_mask, prefix, q_idx (ascending = stable) and the -1 tail.
+// Nothing is read back by the host: the routed count stays on the device.
+#include "l2a_common.cuh"
+
+namespace l2a {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kPerThread = kRouteBlockElems / kThreads;  // 16
+
+__device__ __forceinline__ uint32_t load_flags(const void* router, int kind, float thr, int64_t row_base, int t0,
+                                               int L) {
+  uint32_t flags = 0;
+  if (kind == L2A_ROUTER_MASK_U8) {
+    const uint8_t* m = static_cast<const uint8_t*>(router) + row_base;
+    if (t0 + kPerThread <= L && ((reinterpret_cast<uintptr_t>(m + t0) & 15) == 0)) {
+      const uint4 v = *reinterpret_cast<const uint4*>(m + t0);
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if ((w[i] >> (8 * k)) & 0xffu) flags |= 1u << (4 * i + k);
+    } else {
+      for (int i = 0; i < kPerThread; ++i)
+        if (t0 + i < L && m[t0 + i]) flags |= 1u << i;
+    }
+  } else {
+    const float* z = static_cast<const float*>(router) + row_base;
+    for (int i = 0; i < kPerThread; ++i)
+      if (t0 + i < L && z[t0 + i] >= thr) flags |= 1u << i;  // NaN compares false; -0.0 >= 0.0 is true
+  }
+  return flags;
+}
+
+__global__ void __launch_bounds__(kThreads) route_count_kernel(RouteArgs a) {
+  const int b = blockIdx.y, blk = blockIdx.x;
+  const int t0 = blk * kRouteBlockElems + threadIdx.x * kPerThread;
+  const uint32_t flags = load_flags(a.router, a.router_kind, a.threshold, (int64_t)b * a.L, t0, a.L);
+  int cnt = __popc(flags);
+  __shared__ int warp_cnt[kThreads / 32];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+  if ((threadIdx.x & 31) == 0) warp_cnt[threadIdx.x >> 5] = cnt;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int s = 0;
+    for (int w = 0; w < kThreads / 32; ++w) s += warp_cnt[w];
+    a.block_sums[b * a.nblocks + blk] = s;
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) route_scan_kernel(RouteArgs a) {
+  const int b = blockIdx.y, blk = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __shared__ int red_before[kThreads / 32], red_total[kThreads / 32], warp_off[kThreads / 32];
+
+  // counts of the CTAs before this one, and the row total
+  int before = 0, total = 0;
+  for (int i = threadIdx.x; i < a.nblocks; i += kThreads) {
+    const int v = a.block_sums[b * a.nblocks + i];
+    total += v;
+    if (i < blk) before += v;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    before += __shfl_xor_sync(0xffffffffu, before, o);
+    total += __shfl_xor_sync(0xffffffffu, total, o);
+  }
+  if (lane == 0) { red_before[warp] = before; red_total[warp] = total; }
+  __syncthreads();
+  before = 0; total = 0;
+  for (int w = 0; w < kThreads / 32; ++w) { before += red_before[w]; total += red_total[w]; }
+
+  const int t0 = blk * kRouteBlockElems + threadIdx.x * kPerThread;
+  const uint32_t flags = load_flags(a.router, a.router_kind, a.threshold, (int64_t)b * a.L, t0, a.L);
+  const int cnt = __popc(flags);
+  int incl = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) warp_off[warp] = incl;
+  __syncthreads();
+  int c = before + incl - cnt;
+  for (int w = 0; w < warp; ++w) c += warp_off[w];
+
+  uint8_t* dm = a.d_mask + (int64_t)b * a.L;
+  int32_t* qi = a.q_idx + (int64_t)b * a.L;
+  int32_t* pf = a.prefix + (int64_t)b * (a.L + 1);
+#pragma unroll
+  for (int i = 0; i < kPerThread; ++i) {
+    const int t = t0 + i;
+    if (t < a.L) {
+      const int on = (flags >> i) & 1;
+      dm[t] = (uint8_t)on;
+      pf[t] = c;
+      if (on) qi[c++] = t;
+      if (t >= total) qi[t] = -1;  // compact slots past the routed count
+    }
+  }
+  if (blk == 0 && threadIdx.x == 0) {
+    a.n_routed[b] = total;
+    pf[a.L] = total;
+  }
+}
+
+// One CTA per compact row (grid-stride); 16-byte chunks.
+__global__ void __launch_bounds__(256) gather_rows_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst,
+                                                          const int32_t* __restrict__ q_idx,
+                                                          const int32_t* __restrict__ n_routed, int L,
+                                                          int row_chunks /* 16-byte chunks per row */) {
+  const int b = blockIdx.y;
+  const int n_c = n_routed[b];
+  int n_pad = (n_c + kRowsPerCta - 1) / kRowsPerCta * kRowsPerCta;
+  if (n_pad > L) n_pad = L;
+  const uint4* s = reinterpret_cast<const uint4*>(src) + (int64_t)b * L * row_chunks;
+  uint4* d = reinterpret_cast<uint4*>(dst) + (int64_t)b * L * row_chunks;
+  for (int c = blockIdx.x; c < n_pad; c += gridDim.x) {
+    if (c < n_c) {
+      const int t = q_idx[(int64_t)b * L + c];
+      for (int i = threadIdx.x; i < row_chunks; i += blockDim.x)
+        d[(int64_t)c * row_chunks + i] = __ldg(&s[(int64_t)t * row_chunks + i]);
+    } else {
+      for (int i = threadIdx.x; i < row_chunks; i += blockDim.x)
+        d[(int64_t)c * row_chunks + i] = make_uint4(0, 0, 0, 0);
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_route_compact(const RouteArgs& a, cudaStream_t stream) {
+  dim3 grid(a.nblocks, a.B);
+  route_count_kernel<<<grid, kThreads, 0, stream>>>(a);
+  route_scan_kernel<<<grid, kThreads, 0, stream>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gather_rows(const bf16* src, bf16* dst, const int32_t* q_idx, const int32_t* n_routed, int B,
+                               int L, int row_elems, cudaStream_t stream) {
+  const int row_chunks = row_elems * 2 / 16;
+  int gx = L < 148 * 16 ? L : 148 * 16;
+  dim3 grid(gx, B);
+  gather_rows_kernel<<<grid, 256, 0, stream>>>(src, dst, q_idx, n_routed, L, row_chunks);
+  return cudaGetLastError();
+}
+
+}  // namespace l2a

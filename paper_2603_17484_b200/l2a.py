@@ -1,0 +1,225 @@
+"""Thin binding over the C ABI of ``libl2a.so`` (declared in ``include/l2a.h``).
+
+Argument marshalling only: every step of the path runs in the CUDA kernels of the library.  There is
+no fallback -- if the library has not been built (``python -m paper_2603_17484_b200.build``) or
+cannot be loaded, the first call raises.  torch is used for device memory and streams.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libl2a.so")
+
+L2A_OK = 0
+FLAG_SAVE_FOR_BWD = 1
+FLAG_SKIP_LOCAL = 2
+FLAG_SKIP_GLOBAL = 4
+ROUTER_MASK_U8 = 0
+ROUTER_LOGITS_F32 = 1
+
+EXPORTS = (
+    "l2a_version", "l2a_status_string", "l2a_workspace_bytes", "l2a_workspace_status",
+    "l2a_route_compact", "l2a_forward", "l2a_backward", "l2a_forward_host",
+)
+
+
+class L2AParams(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("Lq", ctypes.c_int32), ("Lk", ctypes.c_int32),
+        ("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32), ("D", ctypes.c_int32),
+        ("window", ctypes.c_int32), ("q_pos_offset", ctypes.c_int32),
+        ("softmax_scale", ctypes.c_float), ("flags", ctypes.c_uint32),
+    ]
+
+
+class L2AError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} ({code})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libl2a.so; raises if it is missing (there is no CPU or eager fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not built: run `python -m paper_2603_17484_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        L.l2a_version.restype = ctypes.c_char_p
+        L.l2a_status_string.restype = ctypes.c_char_p
+        L.l2a_status_string.argtypes = [ctypes.c_int]
+        for name in EXPORTS[2:]:
+            getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def version() -> str:
+    return lib().l2a_version().decode()
+
+
+def status_string(code: int) -> str:
+    return lib().l2a_status_string(code).decode()
+
+
+def params(B, Lq, Lk, Hq, Hkv, D, window, q_pos_offset=None, softmax_scale=0.0, flags=0) -> L2AParams:
+    return L2AParams(B, Lq, Lk, Hq, Hkv, D, window, Lk - Lq if q_pos_offset is None else q_pos_offset,
+                     softmax_scale, flags)
+
+
+def _ptr(t):
+    if t is None:
+        return ctypes.c_void_p(0)
+    if isinstance(t, torch.Tensor):
+        assert t.is_contiguous(), "tensors passed to the C ABI must be contiguous"
+        return ctypes.c_void_p(t.data_ptr())
+    return ctypes.c_void_p(int(t))
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(code: int, where: str):
+    if code != L2A_OK:
+        raise L2AError(code, where)
+
+
+def l2a_workspace_bytes(p: L2AParams) -> tuple[int, int, int]:
+    r, f, b = ctypes.c_size_t(0), ctypes.c_size_t(0), ctypes.c_size_t(0)
+    _check(lib().l2a_workspace_bytes(ctypes.byref(p), ctypes.byref(r), ctypes.byref(f), ctypes.byref(b)),
+           "l2a_workspace_bytes")
+    return r.value, f.value, b.value
+
+
+def l2a_workspace_status(ws: torch.Tensor, stream=None) -> int:
+    return lib().l2a_workspace_status(_ptr(ws), _stream(stream))
+
+
+def l2a_route_compact(p, router, router_kind, logit_threshold, d_mask, q_idx, n_routed, prefix, route_ws,
+                      stream=None, check=True) -> int:
+    code = lib().l2a_route_compact(ctypes.byref(p), _ptr(router), ctypes.c_int(router_kind),
+                                   ctypes.c_float(logit_threshold), _ptr(d_mask), _ptr(q_idx), _ptr(n_routed),
+                                   _ptr(prefix), _ptr(route_ws),
+                                   ctypes.c_size_t(route_ws.numel() * route_ws.element_size() if route_ws is not None else 0),
+                                   _stream(stream))
+    if check:
+        _check(code, "l2a_route_compact")
+    return code
+
+
+def l2a_forward(p, Q, K, V, d_mask, q_idx, n_routed, prefix, O, S_save, A_c, lse_loc, lse_glb, fwd_ws,
+                stream=None, check=True) -> int:
+    code = lib().l2a_forward(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(d_mask), _ptr(q_idx), _ptr(n_routed),
+                             _ptr(prefix), _ptr(O), _ptr(S_save), _ptr(A_c), _ptr(lse_loc), _ptr(lse_glb),
+                             _ptr(fwd_ws),
+                             ctypes.c_size_t(fwd_ws.numel() * fwd_ws.element_size() if fwd_ws is not None else 0),
+                             _stream(stream))
+    if check:
+        _check(code, "l2a_forward")
+    return code
+
+
+def l2a_backward(p, Q, K, V, d_mask, q_idx, n_routed, prefix, dO, S_save, A_c, lse_loc, lse_glb, dQ, dK, dV,
+                 dgate, bwd_ws, stream=None, check=True) -> int:
+    code = lib().l2a_backward(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(d_mask), _ptr(q_idx),
+                              _ptr(n_routed), _ptr(prefix), _ptr(dO), _ptr(S_save), _ptr(A_c), _ptr(lse_loc),
+                              _ptr(lse_glb), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dgate), _ptr(bwd_ws),
+                              ctypes.c_size_t(bwd_ws.numel() * bwd_ws.element_size() if bwd_ws is not None else 0),
+                              _stream(stream))
+    if check:
+        _check(code, "l2a_backward")
+    return code
+
+
+def l2a_forward_host(p, h_Q, h_K, h_V, h_router, router_kind, logit_threshold, h_O, bufs: "Buffers",
+                     stream=None, check=True) -> int:
+    """Host-buffer entry point: copies in, routes, runs the forward, copies O out, synchronises."""
+    code = lib().l2a_forward_host(ctypes.byref(p), _ptr(h_Q), _ptr(h_K), _ptr(h_V), _ptr(h_router),
+                                  ctypes.c_int(router_kind), ctypes.c_float(logit_threshold), _ptr(h_O),
+                                  _ptr(bufs.Q), _ptr(bufs.K), _ptr(bufs.V), _ptr(bufs.router), _ptr(bufs.d_mask),
+                                  _ptr(bufs.q_idx), _ptr(bufs.n_routed), _ptr(bufs.prefix), _ptr(bufs.O),
+                                  _ptr(bufs.route_ws), ctypes.c_size_t(bufs.route_ws.numel()),
+                                  _ptr(bufs.fwd_ws), ctypes.c_size_t(bufs.fwd_ws.numel()), _stream(stream))
+    if check:
+        _check(code, "l2a_forward_host")
+    return code
+
+
+@dataclass
+class Buffers:
+    """Device buffers for one shape (allocation helper for tests and benchmarks; torch owns the memory)."""
+    p: L2AParams
+    Q: torch.Tensor = None
+    K: torch.Tensor = None
+    V: torch.Tensor = None
+    router: torch.Tensor = None
+    d_mask: torch.Tensor = None
+    q_idx: torch.Tensor = None
+    n_routed: torch.Tensor = None
+    prefix: torch.Tensor = None
+    O: torch.Tensor = None
+    S_save: torch.Tensor = None
+    A_c: torch.Tensor = None
+    lse_loc: torch.Tensor = None
+    lse_glb: torch.Tensor = None
+    dO: torch.Tensor = None
+    dQ: torch.Tensor = None
+    dK: torch.Tensor = None
+    dV: torch.Tensor = None
+    dgate: torch.Tensor = None
+    route_ws: torch.Tensor = None
+    fwd_ws: torch.Tensor = None
+    bwd_ws: torch.Tensor = None
+
+    @staticmethod
+    def allocate(p: L2AParams, backward: bool = False, device="cuda", router_dtype=torch.uint8) -> "Buffers":
+        B, Lq, Lk, Hq, Hkv, D = p.B, p.Lq, p.Lk, p.Hq, p.Hkv, p.D
+        bf, dev = torch.bfloat16, device
+        r, f, w = l2a_workspace_bytes(p)
+        b = Buffers(p)
+        b.Q = torch.empty((B, Lq, Hq, D), dtype=bf, device=dev)
+        b.K = torch.empty((B, Lk, Hkv, D), dtype=bf, device=dev)
+        b.V = torch.empty((B, Lk, Hkv, D), dtype=bf, device=dev)
+        b.router = torch.empty((B, Lq), dtype=router_dtype, device=dev)
+        b.d_mask = torch.empty((B, Lq), dtype=torch.uint8, device=dev)
+        b.q_idx = torch.empty((B, Lq), dtype=torch.int32, device=dev)
+        b.n_routed = torch.empty((B,), dtype=torch.int32, device=dev)
+        b.prefix = torch.empty((B, Lq + 1), dtype=torch.int32, device=dev)
+        b.O = torch.empty((B, Lq, Hq, D), dtype=bf, device=dev)
+        b.route_ws = torch.empty((r,), dtype=torch.uint8, device=dev)
+        b.fwd_ws = torch.empty((f,), dtype=torch.uint8, device=dev)
+        if backward:
+            b.S_save = torch.empty((B, Lq, Hq, D), dtype=bf, device=dev)
+            b.A_c = torch.empty((B, Lq, Hq, D), dtype=bf, device=dev)
+            b.lse_loc = torch.empty((B, Hq, Lq), dtype=torch.float32, device=dev)
+            b.lse_glb = torch.empty((B, Hq, Lq), dtype=torch.float32, device=dev)
+            b.dO = torch.empty((B, Lq, Hq, D), dtype=bf, device=dev)
+            b.dQ = torch.empty((B, Lq, Hq, D), dtype=bf, device=dev)
+            b.dK = torch.empty((B, Lk, Hkv, D), dtype=bf, device=dev)
+            b.dV = torch.empty((B, Lk, Hkv, D), dtype=bf, device=dev)
+            b.dgate = torch.empty((B, Lq), dtype=torch.float32, device=dev)
+            b.bwd_ws = torch.empty((w,), dtype=torch.uint8, device=dev)
+        return b
+
+    def route(self, router_kind=ROUTER_MASK_U8, threshold=0.0, stream=None):
+        return l2a_route_compact(self.p, self.router, router_kind, threshold, self.d_mask, self.q_idx,
+                                 self.n_routed, self.prefix, self.route_ws, stream)
+
+    def forward(self, stream=None):
+        return l2a_forward(self.p, self.Q, self.K, self.V, self.d_mask, self.q_idx, self.n_routed, self.prefix,
+                           self.O, self.S_save, self.A_c, self.lse_loc, self.lse_glb, self.fwd_ws, stream)
+
+    def backward(self, stream=None, with_dgate=False):
+        return l2a_backward(self.p, self.Q, self.K, self.V, self.d_mask, self.q_idx, self.n_routed, self.prefix,
+                            self.dO, self.S_save, self.A_c, self.lse_loc, self.lse_glb, self.dQ, self.dK, self.dV,
+                            self.dgate if with_dgate else None, self.bwd_ws, stream)

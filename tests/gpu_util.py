@@ -1,0 +1,92 @@
+"""Helpers for the GPU parity tests: run the CUDA path through the C-ABI binding and the fp64 oracle on
+the same seeded inputs and compare.  Tolerances are the ones the target states for bf16 outputs and
+gradients against the fp64 oracle: max abs error <= 2e-2, mean abs error <= 2e-3."""
+import numpy as np
+import torch
+
+import oracle
+from paper_2603_17484_b200 import l2a, synth
+
+MAX_ABS = 2e-2
+MEAN_ABS = 2e-3
+LSE_ABS = 1e-3
+
+
+def to_f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def check_close(got: np.ndarray, want: np.ndarray, what: str, max_abs=MAX_ABS, mean_abs=MEAN_ABS):
+    assert got.shape == want.shape, (what, got.shape, want.shape)
+    assert np.isfinite(got).all(), f"{what}: non-finite values in the GPU result"
+    err = np.abs(got - want)
+    i = np.unravel_index(np.argmax(err), err.shape) if err.size else ()
+    assert err.size == 0 or err.max() <= max_abs, f"{what}: max abs err {err.max():.4g} at {i} (got {got[i]}, want {want[i]})"
+    assert err.size == 0 or err.mean() <= mean_abs, f"{what}: mean abs err {err.mean():.4g}"
+
+
+class Case:
+    """One synthetic problem on the GPU, inputs shared bit-for-bit with the oracle."""
+
+    def __init__(self, B, Lq, Hq, Hkv, D, W, d, seed, Lk=None, backward=False, scale=0.0, flags=0, logits=None,
+                 threshold=0.0):
+        Lk = Lq if Lk is None else Lk
+        self.shape = oracle.Shape(B, Lq, Lk, Hq, Hkv, D, W, scale=(scale if scale > 0 else None))
+        self.backward = backward
+        t = synth.qkv(B, Lq, Hq, Hkv, D, seed, with_dO=backward, Lk=Lk)
+        self.host = t
+        self.d = np.ascontiguousarray(d, dtype=np.uint8)
+        fl = flags | (l2a.FLAG_SAVE_FOR_BWD if backward else 0)
+        self.p = l2a.params(B, Lq, Lk, Hq, Hkv, D, W, softmax_scale=scale, flags=fl)
+        self.buf = l2a.Buffers.allocate(self.p, backward=backward,
+                                        router_dtype=torch.float32 if logits is not None else torch.uint8)
+        self.buf.Q.copy_(t["Q"]); self.buf.K.copy_(t["K"]); self.buf.V.copy_(t["V"])
+        if backward:
+            self.buf.dO.copy_(t["dO"])
+        if logits is not None:
+            self.buf.router.copy_(torch.from_numpy(logits))
+            self.kind = l2a.ROUTER_LOGITS_F32
+        else:
+            self.buf.router.copy_(torch.from_numpy(self.d))
+            self.kind = l2a.ROUTER_MASK_U8
+        self.threshold = threshold
+
+    def u16(self, name):
+        return synth.as_u16(self.host[name])
+
+    def run_forward(self):
+        b = self.buf
+        # poison outputs so that rows the kernels fail to write are caught
+        b.O.fill_(float("nan"))
+        b.route(self.kind, self.threshold)
+        b.forward()
+        torch.cuda.synchronize()
+        assert l2a.l2a_workspace_status(b.fwd_ws) == 0, "device-side wait timed out in the forward"
+        return b
+
+    def check_routing(self):
+        b = self.buf
+        q_idx, n, prefix = oracle.compact(self.d)
+        assert np.array_equal(b.d_mask.cpu().numpy(), self.d), "d_mask"
+        assert np.array_equal(b.n_routed.cpu().numpy(), n), "n_routed"
+        assert np.array_equal(b.q_idx.cpu().numpy(), q_idx), "q_idx"
+        assert np.array_equal(b.prefix.cpu().numpy(), prefix), "prefix"
+        return q_idx, n, prefix
+
+    def oracle_forward(self):
+        return oracle.forward_full(self.shape, self.u16("Q"), self.u16("K"), self.u16("V"), self.d)
+
+    def check_forward_full(self, ref=None):
+        b = self.buf
+        ref = self.oracle_forward() if ref is None else ref
+        q_idx, n, _ = self.check_routing()
+        check_close(to_f64(b.O), ref["o"], "O")
+        if self.backward:
+            check_close(to_f64(b.S_save), ref["s"], "S_save")
+            check_close(to_f64(b.lse_loc), ref["lse_loc"], "lse_loc", LSE_ABS, LSE_ABS)
+            A_c, lse_glb = to_f64(b.A_c), to_f64(b.lse_glb)
+            for bi in range(self.shape.B):
+                rows = q_idx[bi, :n[bi]]
+                check_close(A_c[bi, :n[bi]], ref["a"][bi, rows], "A_c")
+                check_close(lse_glb[bi, :, :n[bi]], ref["lse_glb"][bi][:, rows], "lse_glb", LSE_ABS, LSE_ABS)
+        return ref

@@ -1,0 +1,60 @@
+"""CPU checks of the boundary: the C-ABI library builds/loads and exports every symbol include/l2a.h
+declares; host-only entry points behave (no GPU work is launched here)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2603_17484_b200 import build as l2a_build
+from paper_2603_17484_b200 import l2a
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    l2a_build.build_lib()
+    return l2a.lib()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "l2a.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(l2a_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_functions()
+    assert {"l2a_route_compact", "l2a_forward", "l2a_backward"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in include/l2a.h but not exported"
+    assert set(names) == set(l2a.EXPORTS)
+
+
+def test_version_and_status_strings(lib):
+    assert "sm_100a" in l2a.version()
+    assert l2a.status_string(0) == "ok"
+    for code in (-1, -2, -3, -4, -5):
+        assert l2a.status_string(code) not in ("ok", "unknown status")
+
+
+def test_workspace_sizes_and_validation(lib):
+    p = l2a.params(1, 131072, 131072, 32, 8, 128, 4096)
+    r, f, b = l2a.l2a_workspace_bytes(p)
+    assert r >= 256 and r % 256 == 0
+    assert f >= 131072 * 32 * 128 * 2            # room for the compact query buffer, worst case
+    assert b >= 256
+    bad = l2a.params(1, 128, 64, 2, 1, 128, 4)   # Lq + offset > Lk with offset forced to 0
+    bad.q_pos_offset = 0
+    with pytest.raises(l2a.L2AError):
+        l2a.l2a_workspace_bytes(bad)
+    with pytest.raises(l2a.L2AError):
+        l2a.l2a_workspace_bytes(l2a.params(1, 128, 128, 3, 2, 128, 4))
+    with pytest.raises(l2a.L2AError) as e:
+        l2a.l2a_workspace_bytes(l2a.params(1, 128, 128, 2, 1, 80, 4))
+    assert e.value.code == -2
+
+
+def test_params_struct_layout_matches_header():
+    assert ctypes.sizeof(l2a.L2AParams) == 40
