@@ -1,0 +1,340 @@
+#!/usr/bin/env python
+"""Benchmark of the L2A hot path on B200: one step = route/compact + forward + backward of one layer.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--density RHO] [--impl reference]
+
+Prints ONE JSON line (rank 0).  ``value`` is useful TFLOP/s with inputs resident in HBM; ``e2e`` is the
+same metric through the host-buffer C-ABI call with the transfers inside the timed region;
+``roofline`` describes the dominant kernel (timed with CUDA events at the phase boundaries the
+library records on its own stream); ``cpu_baseline`` times the fp64 oracle on a bounded sample.
+With N > 1 every rank runs an independent replica of the workload (the path has no exchange step).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2603_17484_b200 import synth  # noqa: E402
+
+METRIC = "L2A fwd+bwd useful TFLOP/s at 128K (one layer, one GPU)"
+KERNELS_PER_STEP = 11  # route: count, scan | fwd: gather, local, global | bwd: gather x2, delta, dkv, dq x2
+FWD_PHASES = ("gather_q", "attn_fwd_local", "attn_fwd_global")
+BWD_PHASES = ("gather_q_dO", "bwd_delta", "bwd_dkv", "bwd_dq_local", "bwd_dq_global")
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            m = json.load(f)
+        return {"burst": m["bf16_tflops"], "sustained": m.get("bf16_tflops_sustained", m["bf16_tflops"]),
+                "hbm_gbs": m["hbm_gbs"], "source": "measured"}
+    return {"burst": 1590.0, "sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(prefix="l2a_clocks_", suffix=".csv")
+            self.out = os.fdopen(fd, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, smax, reasons, power = [], [], set(), []
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        with open(self.path) as f:
+            for line in f:
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1])); smax.append(float(parts[2])); power.append(float(parts[3]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, parts[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+        os.unlink(self.path)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "reasons": sorted(reasons),
+                "power_w_max": float(max(power)), "samples": len(sm)}
+
+
+def make_workload(args, seed_offset=0):
+    cfg = synth.CONFIGS[args.workload]
+    idx = synth.CONFIG_INDEX[args.workload]
+    rho = cfg.density if args.density is None else args.density
+    seed = synth.seed_for(idx, int(round(rho * 10))) + 7919 * seed_offset
+    if args.routing:
+        cfg = synth.Config(**{**cfg.__dict__, "routing": args.routing})
+    d, logits = synth.routing(cfg, seed, density=rho)
+    return cfg, rho, seed, d, logits
+
+
+def cpu_oracle_sample(cfg, seed, rho, T, backward=True):
+    """fp64 oracle, forward (+ backward), on the workload truncated to its first T tokens (all heads)."""
+    import oracle
+    t = synth.qkv(cfg.B, T, cfg.Hq, cfg.Hkv, cfg.D, seed, with_dO=True)
+    d = synth.mask_bernoulli(cfg.B, T, rho, seed) if rho < 1.0 else np.ones((cfg.B, T), np.uint8)
+    sh = oracle.Shape(cfg.B, T, T, cfg.Hq, cfg.Hkv, cfg.D, cfg.W)
+    Q, K, V, dO = (synth.as_u16(t[k]) for k in ("Q", "K", "V", "dO"))
+    oracle.num_threads()  # builds/loads outside the timed region
+    t0 = time.perf_counter()
+    oracle.forward_full(sh, Q, K, V, d)
+    if backward:
+        oracle.backward_full(sh, Q, K, V, d, dO)
+    dt = time.perf_counter() - t0
+    pairs = sum(synth.pairs_local(T, cfg.W) + synth.pairs_global(d[b]) for b in range(cfg.B))
+    flops = (4.0 + (10.0 if backward else 0.0)) * cfg.D * cfg.Hq * pairs
+    return flops / dt / 1e12, dt, oracle.num_threads()
+
+
+def run_reference(args):
+    """Reference arm: the fp64 oracle as it stands on the host cores, a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg, rho, seed, d, _ = make_workload(args)
+    T = args.ref_tokens
+    for _ in range(args.warmup):
+        cpu_oracle_sample(cfg, seed, rho, min(T, 256))
+    t0 = time.perf_counter()
+    vals = [cpu_oracle_sample(cfg, seed + i, rho, T) for i in range(args.steps)]
+    total = time.perf_counter() - t0
+    value = float(np.mean([v[0] for v in vals]))
+    cores = vals[0][2]
+    sample = (f"fp64 oracle forward+backward on the workload truncated to its first {T} tokens (all heads, "
+              f"density {rho}); the backward leg parallelises over (batch, KV head) = {cfg.B * cfg.Hkv} threads")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": total / max(1, args.steps) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "B": cfg.B, "L": cfg.L, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
+                   "W": cfg.W, "density": rho, "sample_tokens": T},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="stress_128k", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--density", type=float, default=None)
+    ap.add_argument("--routing", default=None, choices=[None, "bernoulli", "clustered", "all", "none"])
+    ap.add_argument("--forward-only", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--cpu-tokens", type=int, default=2048, help="tokens of the CPU-baseline sample (0 = skip)")
+    ap.add_argument("--ref-tokens", type=int, default=1024, help="tokens per step of --impl reference")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        return run_reference(args)
+
+    from paper_2603_17484_b200 import l2a
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    cfg, rho, seed, d, logits = make_workload(args, seed_offset=rank)
+    backward = not args.forward_only
+    flags = l2a.FLAG_SAVE_FOR_BWD if backward else 0
+    p = l2a.params(cfg.B, cfg.L, cfg.L, cfg.Hq, cfg.Hkv, cfg.D, cfg.W, flags=flags)
+    use_logits = logits is not None
+    buf = l2a.Buffers.allocate(p, backward=backward, router_dtype=torch.float32 if use_logits else torch.uint8)
+    kind = l2a.ROUTER_LOGITS_F32 if use_logits else l2a.ROUTER_MASK_U8
+
+    # host inputs (pinned): the same seeded tensors the oracle would read
+    host = {k: v.pin_memory() for k, v in synth.qkv(cfg.B, cfg.L, cfg.Hq, cfg.Hkv, cfg.D, seed, with_dO=backward).items()}
+    host["router"] = torch.from_numpy(logits if use_logits else d).pin_memory()
+    host["O"] = torch.empty_like(host["Q"]).pin_memory()
+    if backward:
+        host["dQ"] = torch.empty_like(host["Q"]).pin_memory()
+        host["dK"] = torch.empty_like(host["K"]).pin_memory()
+        host["dV"] = torch.empty_like(host["V"]).pin_memory()
+    for name in ("Q", "K", "V") + (("dO",) if backward else ()):
+        getattr(buf, name).copy_(host[name], non_blocking=True)
+    buf.router.copy_(host["router"], non_blocking=True)
+    torch.cuda.synchronize()
+
+    fwd_flops, bwd_flops = synth.useful_flops(cfg, d, backward)
+    pairs = sum(synth.pairs_local(cfg.L, cfg.W) + synth.pairs_global(d[b]) for b in range(cfg.B))
+    step_flops = fwd_flops + bwd_flops
+
+    def step(profile=None):
+        buf.route(kind, 0.0)
+        if profile is not None:
+            l2a.l2a_profile_next_call([e.cuda_event for e in profile[0]])
+        buf.forward()
+        if backward:
+            if profile is not None:
+                l2a.l2a_profile_next_call([e.cuda_event for e in profile[1]])
+            buf.backward()
+
+    def new_events(n):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        for e in ev:
+            e.record()  # forces creation of the underlying handle
+        return ev
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    assert l2a.l2a_workspace_status(buf.fwd_ws) == 0, "device-side timeout in the forward"
+    if backward:
+        assert l2a.l2a_workspace_status(buf.bwd_ws) == 0, "device-side timeout in the backward"
+
+    prof = [(new_events(4), new_events(6)) for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    start.record()
+    for i in range(args.steps):
+        step(prof[i])
+    stop.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = start.elapsed_time(stop)
+    if dist is not None:
+        t = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+
+    # per-phase durations from the library's own stream events
+    phase_ms = {}
+    for names, which in ((FWD_PHASES, 0), (BWD_PHASES, 1)):
+        if which == 1 and not backward:
+            continue
+        for k, name in enumerate(names):
+            phase_ms[name] = float(np.mean([pr[which][k].elapsed_time(pr[which][k + 1]) for pr in prof]))
+
+    # ---- end to end through the host-buffer C-ABI call (transfers inside the timed region)
+    e2e = None
+    if args.e2e_steps > 0:
+        l2a.l2a_step_host(p, host, buf, kind, 0.0)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        e0.record()
+        for _ in range(args.e2e_steps):
+            l2a.l2a_step_host(p, host, buf, kind, 0.0)
+        e1.record()
+        torch.cuda.synchronize()
+        e2e_ms = e0.elapsed_time(e1) / args.e2e_steps
+        if dist is not None:
+            t = torch.tensor([e2e_ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        qb, kb = host["Q"].numel() * 2, host["K"].numel() * 2
+        h2d = qb + 2 * kb + host["router"].numel() * host["router"].element_size() + (qb if backward else 0)
+        d2h = qb + ((qb + 2 * kb) if backward else 0)
+        e2e = {"value": world * step_flops / e2e_ms / 1e9, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    # dominant kernel and its algorithmic FLOPs: forward kernels 4*D per pair (local / global pairs
+    # separately); dK/dV kernel 8*D per pair (S, dP, dV, dK); dQ kernels 2*D per pair (dQ only; their
+    # recomputation of S and dP is not algorithmic work)
+    HD = cfg.Hq * cfg.D
+    pl = sum(synth.pairs_local(cfg.L, cfg.W) for _ in range(cfg.B))
+    pg = sum(synth.pairs_global(d[b]) for b in range(cfg.B))
+    kernel_flops = {"attn_fwd_local": 4.0 * HD * pl, "attn_fwd_global": 4.0 * HD * pg,
+                    "bwd_dkv": 8.0 * HD * (pl + pg), "bwd_dq_local": 2.0 * HD * pl, "bwd_dq_global": 2.0 * HD * pg}
+    tensor_phases = {k: v for k, v in phase_ms.items() if k in kernel_flops}
+    dom = max(tensor_phases, key=tensor_phases.get)
+    achieved = kernel_flops[dom] / phase_ms[dom] / 1e9
+    roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peaks["sustained"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["sustained"], "traffic": None,
+                "peak_kind": f"sustained bf16 GEMM, {peaks['source']}", "launch_ms": phase_ms[dom],
+                "algorithmic_flops_per_launch": kernel_flops[dom]}
+
+    cpu = None
+    if args.cpu_tokens > 0 and world == 1:
+        v, dt, cores = cpu_oracle_sample(cfg, seed, min(rho, 1.0), args.cpu_tokens, backward)
+        cpu = {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "seconds": dt,
+               "sample": f"fp64 oracle {'forward+backward' if backward else 'forward'} on the workload truncated to "
+                         f"its first {args.cpu_tokens} tokens (all heads, Bernoulli density {rho}); the backward leg "
+                         f"parallelises over (batch, KV head) = {cfg.B * cfg.Hkv} threads"}
+
+    value = world * step_flops / ms_step / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "B": cfg.B, "L": cfg.L, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
+                   "W": cfg.W, "routing": args.routing or cfg.routing, "density": float(d.mean()),
+                   "pass": "fwd+bwd" if backward else "fwd", "parallelism": f"replicas x{world}",
+                   "l2_policy": "inputs larger than L2 (Q alone is %.2f GB)" % (host["Q"].numel() * 2 / 1e9),
+                   "useful_tflop_per_step": step_flops / 1e12, "pairs_per_head": pairs},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": KERNELS_PER_STEP * args.steps if backward else 5 * args.steps,
+        "roofline": roofline, "cpu_baseline": cpu,
+        "phase_ms": phase_ms,
+        "frac_of_peak": {"measured_burst_%.0f" % peaks["burst"]: value / world / peaks["burst"],
+                         "measured_sustained_%.0f" % peaks["sustained"]: value / world / peaks["sustained"],
+                         "datasheet_2250": value / world / 2250.0},
+    }
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

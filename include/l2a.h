@@ -158,18 +158,50 @@ l2a_status l2a_backward(const l2a_params* p, const void* Q, const void* K, const
                         float* dgate, void* bwd_ws, size_t bwd_ws_bytes, void* stream);
 
 /*
- * Convenience for callers that hold HOST buffers: copies Q, K, V and the router input to the
- * device buffers the caller supplies, runs l2a_route_compact + l2a_forward, copies O back, and
- * synchronises the stream.  All `h_` pointers are host memory (pinned memory gives asynchronous
- * copies), all `d_` pointers device memory of the sizes the corresponding arguments above need.
- * Exists so that end-to-end time including the transfers can be measured through the C ABI.
+ * One whole step for callers that hold HOST buffers, so that end-to-end time including the
+ * transfers can be measured through the C ABI: copies Q, K, V, the router input (and dO) to the
+ * device buffers the caller supplies, runs l2a_route_compact + l2a_forward (+ l2a_backward when
+ * host->dO is non-NULL), copies O (and dQ, dK, dV) back, and synchronises the stream.
+ * `host` holds HOST pointers (pinned memory makes the copies asynchronous); `dev` holds DEVICE
+ * pointers with the sizes the corresponding arguments of the three calls need.  With a backward,
+ * p->flags must contain L2A_FLAG_SAVE_FOR_BWD and every field of `dev` must be set; without one,
+ * dO, S_save, A_c, lse_*, dQ, dK, dV and bwd_ws may be NULL.
  */
-l2a_status l2a_forward_host(const l2a_params* p, const void* h_Q, const void* h_K, const void* h_V,
-                            const void* h_router, int router_kind, float logit_threshold, void* h_O,
-                            void* d_Q, void* d_K, void* d_V, void* d_router, uint8_t* d_mask,
-                            int32_t* d_q_idx, int32_t* d_n_routed, int32_t* d_prefix, void* d_O,
-                            void* route_ws, size_t route_ws_bytes, void* fwd_ws, size_t fwd_ws_bytes,
-                            void* stream);
+typedef struct l2a_host_io {
+  const void *Q, *K, *V;  /* bf16, layouts above                                   */
+  const void* router;     /* [B, Lq] uint8 or fp32, per router_kind                */
+  const void* dO;         /* bf16 [B, Lq, Hq, D] or NULL for a forward-only step   */
+  void* O;                /* out                                                   */
+  void *dQ, *dK, *dV;     /* out; may be NULL when dO is NULL                      */
+} l2a_host_io;
+
+typedef struct l2a_device_io {
+  void *Q, *K, *V, *router, *dO;
+  uint8_t* d_mask;
+  int32_t *q_idx, *n_routed, *prefix;
+  void *O, *S_save, *A_c;
+  float *lse_loc, *lse_glb;
+  void *dQ, *dK, *dV;
+  void* route_ws; size_t route_ws_bytes;
+  void* fwd_ws;   size_t fwd_ws_bytes;
+  void* bwd_ws;   size_t bwd_ws_bytes;
+} l2a_device_io;
+
+l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a_device_io* dev,
+                         int router_kind, float logit_threshold, void* stream);
+
+/*
+ * Profiling aid (no counterpart in the paper).  Registers up to 8 cudaEvent_t handles (host array of
+ * `n_events` handles created by the caller with timing enabled; the array is copied).  The NEXT
+ * l2a_forward or l2a_backward call made by this host thread records event k on its stream at its
+ * k-th phase boundary and then clears the registration.  Phase boundaries:
+ *   l2a_forward : 0 start | 1 after the query gather | 2 after the local kernel | 3 after the
+ *                 global kernel
+ *   l2a_backward: 0 start | 1 after the gathers | 2 after the Delta kernel | 3 after the dK/dV
+ *                 kernel | 4 after the local dQ kernel | 5 after the global dQ kernel
+ * This is the only per-thread state the library keeps.
+ */
+l2a_status l2a_profile_next_call(void* const* events, int n_events);
 
 #ifdef __cplusplus
 }

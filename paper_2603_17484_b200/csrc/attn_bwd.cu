@@ -652,12 +652,15 @@ cudaError_t launch_bwd_kernels(const BwdArgs& base, const CUtensorMap& mapQ, con
   const unsigned n_kblocks = (base.Lk + kTileN - 1) / kTileN;
   bwd_dkv_kernel<D><<<n_kblocks * base.B * base.Hkv, 192, DkvSmem<D>::kTotal, s>>>(mapQ, mapDO, mapQc, mapDOc, mapK,
                                                                                   mapV, base);
+  phase_events().mark(s);
   const unsigned n_tiles = (base.Lq + kTileM - 1) / kTileM;
   BwdArgs a = base;
   a.global_mode = 0;
   bwd_dq_kernel<D><<<n_tiles * base.B * base.Hq, 192, DqSmem<D>::kTotal, s>>>(mapQ, mapDO, mapK, mapV, a);
+  phase_events().mark(s);
   a.global_mode = 1;
   bwd_dq_kernel<D><<<n_tiles * base.B * base.Hq, 192, DqSmem<D>::kTotal, s>>>(mapQc, mapDOc, mapK, mapV, a);
+  phase_events().mark(s);
   return cudaGetLastError();
 }
 
@@ -703,11 +706,15 @@ extern "C" l2a_status l2a_backward(const l2a_params* p, const void* Q, const voi
       !encode_rows_map(&mapV, V, p->B, p->Lk, p->Hkv * p->D, kTileN))
     return L2A_ERR_CUDA;
 
+  PhaseEvents& pe = phase_events();
+  struct ClearOnExit { PhaseEvents& p; ~ClearOnExit() { p.clear(); } } clear_on_exit{pe};
+  pe.mark(s);
   if (launch_gather_rows(static_cast<const bf16*>(Q), Qc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s) != cudaSuccess)
     return L2A_ERR_CUDA;
   if (launch_gather_rows(static_cast<const bf16*>(dO), dOc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s) !=
       cudaSuccess)
     return L2A_ERR_CUDA;
+  pe.mark(s);
   {
     const int64_t warps = (int64_t)p->B * p->Lq;
     const unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
@@ -716,6 +723,7 @@ extern "C" l2a_status l2a_backward(const l2a_params* p, const void* Q, const voi
                                             p->B, p->Lq, p->Hq, p->D);
     if (cudaGetLastError() != cudaSuccess) return L2A_ERR_CUDA;
   }
+  pe.mark(s);
   BwdArgs a;
   a.B = p->B; a.Lq = p->Lq; a.Lk = p->Lk; a.Hq = p->Hq; a.Hkv = p->Hkv; a.D = p->D;
   a.window = p->window;

@@ -52,6 +52,11 @@ bool ws_ok(const void* ws, size_t have, size_t need) { return ws && aligned(ws, 
 
 }  // namespace
 
+PhaseEvents& phase_events() {
+  static thread_local PhaseEvents pe;
+  return pe;
+}
+
 bool encode_rows_map(CUtensorMap* map, const void* base, int batch, int rows, int row_elems, int box_rows) {
   encode_tiled_fn enc = get_encode();
   if (!enc) return false;
@@ -170,12 +175,16 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
   a.n_routed = n_routed;
   a.status = status;
 
+  PhaseEvents& pe = phase_events();
+  struct ClearOnExit { PhaseEvents& p; ~ClearOnExit() { p.clear(); } } clear_on_exit{pe};
+  pe.mark(s);
   if (!skip_global) {
     // consolidate routed query rows (Algorithm 1, step 1); independent of the local pass
     if (launch_gather_rows(static_cast<const bf16*>(Q), Qc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s) !=
         cudaSuccess)
       return L2A_ERR_CUDA;
   }
+  pe.mark(s);
   if (!skip_local) {
     a.global_mode = 0;
     a.accumulate_into_out2 = 0;
@@ -187,6 +196,7 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
     const size_t bytes = (size_t)p->B * p->Lq * p->Hq * p->D * sizeof(bf16);
     if (cudaMemsetAsync(O, 0, bytes, s) != cudaSuccess) return L2A_ERR_CUDA;  // Algorithm 1: O starts at zero
   }
+  pe.mark(s);
   if (!skip_global) {
     a.global_mode = 1;
     a.accumulate_into_out2 = skip_local ? 0 : 1;
@@ -195,36 +205,60 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
     a.lse = lse_glb;
     if (launch_attn_fwd(a, mapQc, mapK, mapV, s) != cudaSuccess) return L2A_ERR_CUDA;
   }
+  pe.mark(s);
   return L2A_OK;
 }
 
-l2a_status l2a_forward_host(const l2a_params* p, const void* h_Q, const void* h_K, const void* h_V,
-                            const void* h_router, int router_kind, float logit_threshold, void* h_O, void* d_Q,
-                            void* d_K, void* d_V, void* d_router, uint8_t* d_mask, int32_t* d_q_idx,
-                            int32_t* d_n_routed, int32_t* d_prefix, void* d_O, void* route_ws, size_t route_ws_bytes,
-                            void* fwd_ws, size_t fwd_ws_bytes, void* stream) {
+l2a_status l2a_profile_next_call(void* const* events, int n_events) {
+  if (n_events < 0 || n_events > 8 || (n_events > 0 && !events)) return L2A_ERR_INVALID_ARG;
+  PhaseEvents& pe = phase_events();
+  pe.clear();
+  for (int i = 0; i < n_events; ++i) pe.ev[i] = static_cast<cudaEvent_t>(events[i]);
+  pe.n = n_events;
+  return L2A_OK;
+}
+
+l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a_device_io* dev, int router_kind,
+                         float logit_threshold, void* stream) {
   l2a_status st = check_params(p);
   if (st != L2A_OK) return st;
-  if (!h_Q || !h_K || !h_V || !h_router || !h_O || !d_Q || !d_K || !d_V || !d_router || !d_O)
+  if (!host || !dev) return L2A_ERR_INVALID_ARG;
+  const bool bwd = host->dO != nullptr;
+  if (!host->Q || !host->K || !host->V || !host->router || !host->O || !dev->Q || !dev->K || !dev->V ||
+      !dev->router || !dev->O)
+    return L2A_ERR_INVALID_ARG;
+  if (bwd && (!host->dQ || !host->dK || !host->dV || !dev->dO || !dev->dQ || !dev->dK || !dev->dV ||
+              !(p->flags & L2A_FLAG_SAVE_FOR_BWD)))
     return L2A_ERR_INVALID_ARG;
   if (router_kind != L2A_ROUTER_MASK_U8 && router_kind != L2A_ROUTER_LOGITS_F32) return L2A_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t qb = (size_t)p->B * p->Lq * p->Hq * p->D * sizeof(bf16);
   const size_t kb = (size_t)p->B * p->Lk * p->Hkv * p->D * sizeof(bf16);
   const size_t rb = (size_t)p->B * p->Lq * (router_kind == L2A_ROUTER_MASK_U8 ? 1 : 4);
-  if (cudaMemcpyAsync(d_router, h_router, rb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
-  if (cudaMemcpyAsync(d_Q, h_Q, qb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
-  if (cudaMemcpyAsync(d_K, h_K, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
-  if (cudaMemcpyAsync(d_V, h_V, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
-  st = l2a_route_compact(p, d_router, router_kind, logit_threshold, d_mask, d_q_idx, d_n_routed, d_prefix, route_ws,
-                         route_ws_bytes, stream);
+  if (cudaMemcpyAsync(dev->router, host->router, rb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
+  if (cudaMemcpyAsync(dev->Q, host->Q, qb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
+  if (cudaMemcpyAsync(dev->K, host->K, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
+  if (cudaMemcpyAsync(dev->V, host->V, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
+  if (bwd && cudaMemcpyAsync(dev->dO, host->dO, qb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
+  st = l2a_route_compact(p, dev->router, router_kind, logit_threshold, dev->d_mask, dev->q_idx, dev->n_routed,
+                         dev->prefix, dev->route_ws, dev->route_ws_bytes, stream);
   if (st != L2A_OK) return st;
   l2a_params q = *p;
-  q.flags &= ~L2A_FLAG_SAVE_FOR_BWD;
-  st = l2a_forward(&q, d_Q, d_K, d_V, d_mask, d_q_idx, d_n_routed, d_prefix, d_O, nullptr, nullptr, nullptr, nullptr,
-                   fwd_ws, fwd_ws_bytes, stream);
+  if (!bwd) q.flags &= ~L2A_FLAG_SAVE_FOR_BWD;
+  st = l2a_forward(&q, dev->Q, dev->K, dev->V, dev->d_mask, dev->q_idx, dev->n_routed, dev->prefix, dev->O,
+                   bwd ? dev->S_save : nullptr, bwd ? dev->A_c : nullptr, bwd ? dev->lse_loc : nullptr,
+                   bwd ? dev->lse_glb : nullptr, dev->fwd_ws, dev->fwd_ws_bytes, stream);
   if (st != L2A_OK) return st;
-  if (cudaMemcpyAsync(h_O, d_O, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return L2A_ERR_CUDA;
+  if (cudaMemcpyAsync(host->O, dev->O, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return L2A_ERR_CUDA;
+  if (bwd) {
+    st = l2a_backward(&q, dev->Q, dev->K, dev->V, dev->d_mask, dev->q_idx, dev->n_routed, dev->prefix, dev->dO,
+                      dev->S_save, dev->A_c, dev->lse_loc, dev->lse_glb, dev->dQ, dev->dK, dev->dV, nullptr,
+                      dev->bwd_ws, dev->bwd_ws_bytes, stream);
+    if (st != L2A_OK) return st;
+    if (cudaMemcpyAsync(host->dQ, dev->dQ, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return L2A_ERR_CUDA;
+    if (cudaMemcpyAsync(host->dK, dev->dK, kb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return L2A_ERR_CUDA;
+    if (cudaMemcpyAsync(host->dV, dev->dV, kb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return L2A_ERR_CUDA;
+  }
   if (cudaStreamSynchronize(s) != cudaSuccess) return L2A_ERR_CUDA;
   return L2A_OK;
 }

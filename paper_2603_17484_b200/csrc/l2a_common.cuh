@@ -58,7 +58,19 @@ struct FwdArgs {
   float* lse;   // local: [B,Hq,Lq] by row;  global: [B,Hq,Lq] by compact row; may be NULL
   int* status;  // workspace status word
 };
-size_t bwd_ws_size(const l2a_params* p);  // defined with the backward
+size_t bwd_ws_size(const l2a_params* p);
+
+// One-shot, thread-local registration of phase-boundary events (see l2a_profile_next_call).
+struct PhaseEvents {
+  cudaEvent_t ev[8];
+  int n = 0;
+  int next = 0;
+  void mark(cudaStream_t s) {
+    if (next < n) cudaEventRecord(ev[next++], s);
+  }
+  void clear() { n = 0; next = 0; }
+};
+PhaseEvents& phase_events();  // defined with the backward
 
 cudaError_t launch_attn_fwd(const FwdArgs& a, const CUtensorMap& mapQ, const CUtensorMap& mapK,
                             const CUtensorMap& mapV, cudaStream_t stream);

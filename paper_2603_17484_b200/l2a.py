@@ -24,7 +24,7 @@ ROUTER_LOGITS_F32 = 1
 
 EXPORTS = (
     "l2a_version", "l2a_status_string", "l2a_workspace_bytes", "l2a_workspace_status",
-    "l2a_route_compact", "l2a_forward", "l2a_backward", "l2a_forward_host",
+    "l2a_route_compact", "l2a_forward", "l2a_backward", "l2a_step_host", "l2a_profile_next_call",
 )
 
 
@@ -141,17 +141,44 @@ def l2a_backward(p, Q, K, V, d_mask, q_idx, n_routed, prefix, dO, S_save, A_c, l
     return code
 
 
-def l2a_forward_host(p, h_Q, h_K, h_V, h_router, router_kind, logit_threshold, h_O, bufs: "Buffers",
-                     stream=None, check=True) -> int:
-    """Host-buffer entry point: copies in, routes, runs the forward, copies O out, synchronises."""
-    code = lib().l2a_forward_host(ctypes.byref(p), _ptr(h_Q), _ptr(h_K), _ptr(h_V), _ptr(h_router),
-                                  ctypes.c_int(router_kind), ctypes.c_float(logit_threshold), _ptr(h_O),
-                                  _ptr(bufs.Q), _ptr(bufs.K), _ptr(bufs.V), _ptr(bufs.router), _ptr(bufs.d_mask),
-                                  _ptr(bufs.q_idx), _ptr(bufs.n_routed), _ptr(bufs.prefix), _ptr(bufs.O),
-                                  _ptr(bufs.route_ws), ctypes.c_size_t(bufs.route_ws.numel()),
-                                  _ptr(bufs.fwd_ws), ctypes.c_size_t(bufs.fwd_ws.numel()), _stream(stream))
+class HostIO(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("Q", "K", "V", "router", "dO", "O", "dQ", "dK", "dV")]
+
+
+class DeviceIO(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("Q", "K", "V", "router", "dO", "d_mask", "q_idx", "n_routed", "prefix",
+                                                "O", "S_save", "A_c", "lse_loc", "lse_glb", "dQ", "dK", "dV")] + [
+        ("route_ws", ctypes.c_void_p), ("route_ws_bytes", ctypes.c_size_t),
+        ("fwd_ws", ctypes.c_void_p), ("fwd_ws_bytes", ctypes.c_size_t),
+        ("bwd_ws", ctypes.c_void_p), ("bwd_ws_bytes", ctypes.c_size_t)]
+
+
+def _addr(t):
+    return None if t is None else (t.data_ptr() if isinstance(t, torch.Tensor) else int(t))
+
+
+def l2a_step_host(p, host: dict, bufs: "Buffers", router_kind=ROUTER_MASK_U8, logit_threshold=0.0, stream=None,
+                  check=True) -> int:
+    """Whole step from HOST tensors (dict with Q, K, V, router, O and, for a backward, dO, dQ, dK, dV):
+    copies in, routes, runs forward (+ backward), copies the results out, synchronises."""
+    h = HostIO(*[_addr(host.get(n)) for n in ("Q", "K", "V", "router", "dO", "O", "dQ", "dK", "dV")])
+    names = ("Q", "K", "V", "router", "dO", "d_mask", "q_idx", "n_routed", "prefix", "O", "S_save", "A_c",
+             "lse_loc", "lse_glb", "dQ", "dK", "dV")
+    d = DeviceIO(*[_addr(getattr(bufs, n)) for n in names],
+                 _addr(bufs.route_ws), bufs.route_ws.numel(), _addr(bufs.fwd_ws), bufs.fwd_ws.numel(),
+                 _addr(bufs.bwd_ws), 0 if bufs.bwd_ws is None else bufs.bwd_ws.numel())
+    code = lib().l2a_step_host(ctypes.byref(p), ctypes.byref(h), ctypes.byref(d), ctypes.c_int(router_kind),
+                               ctypes.c_float(logit_threshold), _stream(stream))
     if check:
-        _check(code, "l2a_forward_host")
+        _check(code, "l2a_step_host")
+    return code
+
+
+def l2a_profile_next_call(events) -> int:
+    """events: sequence of raw cudaEvent_t handles (ints); see include/l2a.h for the phase boundaries."""
+    arr = (ctypes.c_void_p * len(events))(*[ctypes.c_void_p(int(e)) for e in events])
+    code = lib().l2a_profile_next_call(arr, ctypes.c_int(len(events)))
+    _check(code, "l2a_profile_next_call")
     return code
 
 
