@@ -191,6 +191,35 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
                          int router_kind, float logit_threshold, void* stream);
 
 /*
+ * l2a_route_compact without any caller-provided scratch (an addition of this library; the paper has
+ * no counterpart).  Same inputs, outputs and results as l2a_route_compact, but the per-CTA counts the
+ * two kernels exchange live in a fixed device array compiled into the library instead of in
+ * `route_ws`, and the call performs no device allocation of any kind.
+ *
+ * Who needs this: callers that cannot obtain device memory at the point of the call -- code running
+ * inside an engine whose allocator has already reserved all of HBM for its own pools, plug-ins that
+ * are handed tensors but no allocator, and latency-critical loops that must not touch cudaMalloc
+ * (which may synchronise the whole device) once they are running.
+ *
+ * Limits and rules:
+ *   - B * ceil(Lq / 4096) must not exceed L2A_STATIC_ROUTE_SLOTS (4096 counts, 16 KB; e.g. B = 1 up
+ *     to Lq = 16,777,216, or B = 128 at Lq = 131,072).  Larger shapes are rejected on the host with
+ *     L2A_ERR_UNSUPPORTED before anything is launched; use l2a_route_compact for those.
+ *   - The array is static device memory: every GPU that loads the library holds its 16 KB until the
+ *     process exits.
+ *   - The first call on each device looks up the array's device address (with that device current)
+ *     and caches it; make that first call before starting any stream capture.
+ *   - All calls on one device share the array and it keeps the previous call's contents.  Nothing in
+ *     it needs to start at zero (the first kernel overwrites every count the second one reads), but
+ *     two calls whose kernels overlap on the GPU (different streams, no dependency) race on it:
+ *     serialise them.
+ */
+#define L2A_STATIC_ROUTE_SLOTS 4096
+l2a_status l2a_route_compact_static(const l2a_params* p, const void* router, int router_kind,
+                                    float logit_threshold, uint8_t* d_mask, int32_t* q_idx,
+                                    int32_t* n_routed, int32_t* prefix, void* stream);
+
+/*
  * Profiling aid (no counterpart in the paper).  Registers up to 8 cudaEvent_t handles (host array of
  * `n_events` handles created by the caller with timing enabled; the array is copied).  The NEXT
  * l2a_forward or l2a_backward call made by this host thread records event k on its stream at its

@@ -156,3 +156,61 @@ cudaError_t launch_gather_rows(const bf16* src, bf16* dst, const int32_t* q_idx,
 }
 
 }  // namespace l2a
+
+// ------------------------------------------------------------------------------------------------
+// Variant of the routing/compaction entry point that needs no scratch from the caller and allocates
+// nothing: the per-CTA counts live in a fixed array in the library's own device image.
+//
+// In host code `g_static_route_counts` is only a handle for the runtime, not a device address, so
+// the launcher is never given the symbol itself: the address is looked up once per device with
+// cudaGetSymbolAddress (with that device current) and cached.
+static __device__ __align__(256) int32_t g_static_route_counts[L2A_STATIC_ROUTE_SLOTS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+int32_t* g_static_counts_addr[kMaxDevices] = {};
+
+// Returns the device address of the static array on the current device (nullptr on failure).
+int32_t* static_counts_for_current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  int32_t* cached = __atomic_load_n(&g_static_counts_addr[dev], __ATOMIC_ACQUIRE);
+  if (cached) return cached;
+  void* ptr = nullptr;
+  if (cudaGetSymbolAddress(&ptr, g_static_route_counts) != cudaSuccess || ptr == nullptr) return nullptr;
+  __atomic_store_n(&g_static_counts_addr[dev], static_cast<int32_t*>(ptr), __ATOMIC_RELEASE);
+  return static_cast<int32_t*>(ptr);
+}
+}  // namespace
+
+extern "C" l2a_status l2a_route_compact_static(const l2a_params* p, const void* router, int router_kind,
+                                               float logit_threshold, uint8_t* d_mask, int32_t* q_idx,
+                                               int32_t* n_routed, int32_t* prefix, void* stream) {
+  // shape checks come from the workspace query (host only, launches nothing)
+  size_t unused = 0;
+  l2a_status st = l2a_workspace_bytes(p, &unused, nullptr, nullptr);
+  if (st != L2A_OK) return st;
+  if (!router || !d_mask || !q_idx || !n_routed || !prefix) return L2A_ERR_INVALID_ARG;
+  if (router_kind != L2A_ROUTER_MASK_U8 && router_kind != L2A_ROUTER_LOGITS_F32) return L2A_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(q_idx) | reinterpret_cast<uintptr_t>(n_routed) |
+       reinterpret_cast<uintptr_t>(prefix)) & 3)
+    return L2A_ERR_INVALID_ARG;
+  if (router_kind == L2A_ROUTER_LOGITS_F32 && (reinterpret_cast<uintptr_t>(router) & 3)) return L2A_ERR_INVALID_ARG;
+  const int nblocks = l2a::ceil_div(p->Lq, l2a::kRouteBlockElems);
+  if ((int64_t)p->B * nblocks > L2A_STATIC_ROUTE_SLOTS) return L2A_ERR_UNSUPPORTED;  // beyond the fixed scratch
+  int32_t* counts = static_counts_for_current_device();
+  if (!counts) return L2A_ERR_CUDA;
+  l2a::RouteArgs a;
+  a.router = router;
+  a.router_kind = router_kind;
+  a.threshold = logit_threshold;
+  a.B = p->B;
+  a.L = p->Lq;
+  a.d_mask = d_mask;
+  a.q_idx = q_idx;
+  a.n_routed = n_routed;
+  a.prefix = prefix;
+  a.block_sums = counts;
+  a.nblocks = nblocks;
+  return l2a::launch_route_compact(a, static_cast<cudaStream_t>(stream)) == cudaSuccess ? L2A_OK : L2A_ERR_CUDA;
+}

@@ -25,6 +25,7 @@ ROUTER_LOGITS_F32 = 1
 EXPORTS = (
     "l2a_version", "l2a_status_string", "l2a_workspace_bytes", "l2a_workspace_status",
     "l2a_route_compact", "l2a_forward", "l2a_backward", "l2a_step_host", "l2a_profile_next_call",
+    "l2a_route_compact_static",
 )
 
 
@@ -114,6 +115,18 @@ def l2a_route_compact(p, router, router_kind, logit_threshold, d_mask, q_idx, n_
                                    _stream(stream))
     if check:
         _check(code, "l2a_route_compact")
+    return code
+
+
+def l2a_route_compact_static(p, router, router_kind, logit_threshold, d_mask, q_idx, n_routed, prefix, stream=None,
+                             check=True) -> int:
+    """Routing + compaction with the scratch held in the library's own fixed device array: for callers that
+    cannot hand over (or allocate) a workspace.  Limits and sharing rules are in include/l2a.h."""
+    code = lib().l2a_route_compact_static(ctypes.byref(p), _ptr(router), ctypes.c_int(router_kind),
+                                          ctypes.c_float(logit_threshold), _ptr(d_mask), _ptr(q_idx),
+                                          _ptr(n_routed), _ptr(prefix), _stream(stream))
+    if check:
+        _check(code, "l2a_route_compact_static")
     return code
 
 
