@@ -25,7 +25,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2603_17484_b200 import synth  # noqa: E402
+from paper_2603_17484_b200 import replicas, synth  # noqa: E402
 
 METRIC = "L2A fwd+bwd useful TFLOP/s at 128K (one layer, one GPU)"
 KERNELS_PER_STEP = 11  # route: count, scan | fwd: gather, local, global | bwd: gather x2, delta, dkv, dq x2
@@ -98,7 +98,7 @@ def make_workload(args, seed_offset=0):
     cfg = synth.CONFIGS[args.workload]
     idx = synth.CONFIG_INDEX[args.workload]
     rho = cfg.density if args.density is None else args.density
-    seed = synth.seed_for(idx, int(round(rho * 10))) + 7919 * seed_offset
+    seed = synth.seed_for(idx, int(round(rho * 10))) + replicas.rank_seed_offset(seed_offset)
     if args.routing:
         cfg = synth.Config(**{**cfg.__dict__, "routing": args.routing})
     d, logits = synth.routing(cfg, seed, density=rho)
@@ -245,11 +245,7 @@ def main():
     stop.record()
     torch.cuda.synchronize()
     clocks = sampler.stop() if rank == 0 else None
-    ms_total = start.elapsed_time(stop)
-    if dist is not None:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = replicas.max_over_ranks(start.elapsed_time(stop), dist, "cuda")
     ms_step = ms_total / args.steps
 
     # per-phase durations from the library's own stream events
@@ -273,15 +269,11 @@ def main():
             l2a.l2a_step_host(p, host, buf, kind, 0.0)
         e1.record()
         torch.cuda.synchronize()
-        e2e_ms = e0.elapsed_time(e1) / args.e2e_steps
-        if dist is not None:
-            t = torch.tensor([e2e_ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = replicas.max_over_ranks(e0.elapsed_time(e1) / args.e2e_steps, dist, "cuda")
         qb, kb = host["Q"].numel() * 2, host["K"].numel() * 2
         h2d = qb + 2 * kb + host["router"].numel() * host["router"].element_size() + (qb if backward else 0)
         d2h = qb + ((qb + 2 * kb) if backward else 0)
-        e2e = {"value": world * step_flops / e2e_ms / 1e9, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+        e2e = {"value": replicas.job_throughput(world, step_flops, e2e_ms) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}
 
     if rank != 0:
@@ -314,7 +306,7 @@ def main():
                          f"its first {args.cpu_tokens} tokens (all heads, Bernoulli density {rho}); the backward leg "
                          f"parallelises over (batch, KV head) = {cfg.B * cfg.Hkv} threads"}
 
-    value = world * step_flops / ms_step / 1e9
+    value = replicas.job_throughput(world, step_flops, ms_step) / 1e12
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
