@@ -14,7 +14,8 @@
 //                      then the compact routed tiles from the first one at or after the block -- and
 //                      accumulates dK, dV in TMEM (no atomics, one bf16 store).  The scores are built
 //                      transposed (keys on TMEM lanes) so P^T and dS^T feed the second pair of MMAs
-//                      straight from TMEM.
+//                      straight from TMEM.  Each tile is processed as two 64-column halves so that the
+//                      MMAs of one half overlap the exponentials of the other.
 //   bwd_dq_kernel    : query-stationary, the forward's iteration space; local mode writes dQ, global mode
 //                      adds the routed rows' global term at their positions.
 #include "l2a_common.cuh"
@@ -26,6 +27,17 @@ namespace {
 
 constexpr int kBoxBytes = 128 * 128;
 constexpr float kLog2e = 1.4426950408889634f;
+
+// Optional per-role clock tracing of one CTA of the dK/dV kernel (development builds only: -DL2A_TRACE=<block>).
+#ifdef L2A_TRACE
+__device__ long long g_trace[4][8192];
+#define L2A_TRACE_POINT(role, idx)                                                              \
+  do {                                                                                          \
+    if (blockIdx.x == (L2A_TRACE) && (idx) < 8192) g_trace[role][idx] = clock64();              \
+  } while (0)
+#else
+#define L2A_TRACE_POINT(role, idx)
+#endif
 
 // ------------------------------------------------------------------------------------------------
 // Delta / dgate preprocess: one warp per (b, t), looping over heads.
@@ -92,33 +104,51 @@ struct BwdArgs {
 };
 
 // ================================================================================================
-// dQ kernel: one 128-row query tile per CTA.
-//   warps 0-3: P / dS computation and epilogue (thread = query row); warp 4: TMA; warp 5: MMA.
-//   TMEM: S [0,128) | dP [128,256) | dQ [256,256+D).  dS (bf16) overwrites the first half of dP.
+// Thread roles of the two tensor-core kernels below:
+//   warps 0-15 : compute.  Warp w owns TMEM lanes 32*(w%4)..+31 (its thread's query row / key) and the
+//                32 score columns of quarter w/4, so that 16 warps hide each other's TMEM and MUFU latency.
+//   warp 16    : TMA producer          warp 17 : tcgen05 MMA issuer, TMEM owner
+//   warp 18    : (dK/dV kernel only) stages the row statistics of each query tile
+constexpr int kComputeWarps = 16;
+constexpr int kDqThreads = (kComputeWarps + 2) * 32;    // 576
+constexpr int kDkvThreads = (kComputeWarps + 3) * 32;   // 608
+
+__device__ __forceinline__ float bf16lo_to_f32(uint32_t packed) { return __uint_as_float(packed << 16); }
+__device__ __forceinline__ float bf16hi_to_f32(uint32_t packed) { return __uint_as_float(packed & 0xffff0000u); }
+
+// ================================================================================================
+// dQ kernel: one 128-row query tile per CTA; Q and dO stay in shared memory, K/V blocks stream.
+//   TMEM: dQ [0,D) | S (two buffers) [128,256) [256,384) | dP [384,512).
+//   dS (bf16) is written over dP: quarter q puts its 16 packed columns at the start of its own 32
+//   columns, and is the A operand of dQ += dS K.
+//   MMA order per key block j:  dQ(j-1) | dP(j) | S(j+1): the exponentials of block j run under dQ(j-1) and
+//   dP(j), the dS of block j under S(j+1), so the tensor pipe never waits for the CUDA cores.
 template <int D>
 struct DqSmem {
   static constexpr int kTileBytes = 128 * D * 2;
+  static constexpr int kKStages = 3;
+  static constexpr int kVStages = 2;
   static constexpr int kQOff = 0;
   static constexpr int kDoOff = kTileBytes;
   static constexpr int kKOff = 2 * kTileBytes;
-  static constexpr int kVOff = 4 * kTileBytes;
-  static constexpr int kBarOff = 6 * kTileBytes;
+  static constexpr int kVOff = kKOff + kKStages * kTileBytes;
+  static constexpr int kBarOff = kVOff + kVStages * kTileBytes;
   static constexpr int kTotal = kBarOff + 256 + 1024;
 };
 struct DqBarriers {
   uint64_t q_full;
-  uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
-  uint64_t sdp_full, ds_full, final_bar;
+  uint64_t k_full[3], k_empty[3], v_full[2], v_empty[2];
+  uint64_t s_full[2], dp_full, ds_full, final_bar;
   uint32_t tmem_base;
   int abort_flag;
 };
 
 template <int D>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kDqThreads, 1)
 bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapDO,
               const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, const BwdArgs a) {
   using SM = DqSmem<D>;
-  constexpr int kDBoxes = D / 64, kKSteps = D / 16;
+  constexpr int kKSteps = D / 16;
   const int n_tiles = (a.Lq + kTileM - 1) / kTileM;
   const int h = blockIdx.x % a.Hq;
   const int rest = blockIdx.x / a.Hq;
@@ -135,6 +165,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
   const int max_pos = (a.global_mode ? q_idx_b[last] : last) + a.q_pos_offset;
   const int jlo = (min_pos - w_eff > 0) ? (min_pos - w_eff) / kTileN : 0;
   const int jhi = max_pos / kTileN;
+  const int n_blocks = jhi - jlo + 1;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -148,82 +179,116 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
 
   if (tid == 0) {
     mbar_init(&bar->q_full, 1);
+    for (int s = 0; s < 3; ++s) { mbar_init(&bar->k_full[s], 1); mbar_init(&bar->k_empty[s], 1); }
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&bar->k_full[s], 1); mbar_init(&bar->k_empty[s], 1);
       mbar_init(&bar->v_full[s], 1); mbar_init(&bar->v_empty[s], 1);
+      mbar_init(&bar->s_full[s], 1);
     }
-    mbar_init(&bar->sdp_full, 1);
-    mbar_init(&bar->ds_full, 128);
+    mbar_init(&bar->dp_full, 1);
+    mbar_init(&bar->ds_full, kComputeWarps * 32);
     mbar_init(&bar->final_bar, 1);
     bar->abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 5) { tmem_alloc(&bar->tmem_base, 512); tmem_relinquish(); }
+  if (warp == 17) { tmem_alloc(&bar->tmem_base, 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bar->tmem_base;
 
-  if (warp == 4) {
+  if (warp == 16) {
+    // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&mapQ); tma_prefetch_desc(&mapDO); tma_prefetch_desc(&mapK); tma_prefetch_desc(&mapV);
       mbar_expect_tx(&bar->q_full, 2 * SM::kTileBytes);
-      for (int x = 0; x < kDBoxes; ++x) {
-        tma_load_3d(sQ + x * kBoxBytes, &mapQ, &bar->q_full, h * D + x * 64, row0, b);
-        tma_load_3d(sDO + x * kBoxBytes, &mapDO, &bar->q_full, h * D + x * 64, row0, b);
-      }
-      for (int j = jlo; j <= jhi; ++j) {
-        const int it = j - jlo, s = it & 1;
-        const uint32_t ph = (it >> 1) & 1;
-        if (!mbar_wait(&bar->k_empty[s], ph ^ 1, abort_flag)) break;
-        mbar_expect_tx(&bar->k_full[s], SM::kTileBytes);
-        for (int x = 0; x < kDBoxes; ++x)
-          tma_load_3d(sK + s * SM::kTileBytes + x * kBoxBytes, &mapK, &bar->k_full[s], g * D + x * 64, j * kTileN, b);
-        if (!mbar_wait(&bar->v_empty[s], ph ^ 1, abort_flag)) break;
-        mbar_expect_tx(&bar->v_full[s], SM::kTileBytes);
-        for (int x = 0; x < kDBoxes; ++x)
-          tma_load_3d(sV + s * SM::kTileBytes + x * kBoxBytes, &mapV, &bar->v_full[s], g * D + x * 64, j * kTileN, b);
+      tma_load_4d(sQ, &mapQ, &bar->q_full, 0, row0, h * (D / 64), b);
+      tma_load_4d(sDO, &mapDO, &bar->q_full, 0, row0, h * (D / 64), b);
+      for (int it = 0; it < n_blocks; ++it) {
+        const int j = jlo + it;
+        const int ks = it % 3, vs = it & 1;
+        if (!mbar_wait(&bar->k_empty[ks], ((it / 3) & 1) ^ 1, abort_flag)) break;
+        mbar_expect_tx(&bar->k_full[ks], SM::kTileBytes);
+        tma_load_4d(sK + ks * SM::kTileBytes, &mapK, &bar->k_full[ks], 0, j * kTileN, g * (D / 64), b);
+        if (!mbar_wait(&bar->v_empty[vs], ((it >> 1) & 1) ^ 1, abort_flag)) break;
+        mbar_expect_tx(&bar->v_full[vs], SM::kTileBytes);
+        tma_load_4d(sV + vs * SM::kTileBytes, &mapV, &bar->v_full[vs], 0, j * kTileN, g * (D / 64), b);
       }
     }
     __syncwarp();
-  } else if (warp == 5) {
-    if (lane == 0) {
+  } else if (warp == 17) {
+    // ------------------------------------------------------------------ MMA issuer
+    // (whole warp runs the loop; only the tcgen05 instructions are predicated on lane 0)
+    {
+      const uint32_t leader = (lane == 0);
       constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);
       constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 0, 1);
-      bool ok = mbar_wait(&bar->q_full, 0, abort_flag);
-      const uint32_t qa = smem_u32(sQ), doa = smem_u32(sDO);
-      for (int j = jlo; ok && j <= jhi; ++j) {
-        const int it = j - jlo, s = it & 1;
-        const uint32_t ph = (it >> 1) & 1;
-        if (!mbar_wait(&bar->k_full[s], ph, abort_flag) || !mbar_wait(&bar->v_full[s], ph, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t ka = smem_u32(sK + s * SM::kTileBytes), va = smem_u32(sV + s * SM::kTileBytes);
+      const uint64_t dq = smem_desc_sw128(smem_u32(sQ), 16, 1024), ddo = smem_desc_sw128(smem_u32(sDO), 16, 1024);
+      const uint64_t dk_base = smem_desc_sw128(smem_u32(sK), 16, 1024);            // K-major view of a K stage
+      const uint64_t dkm_base = smem_desc_sw128(smem_u32(sK), kBoxBytes, 1024);    // same bytes as MN-major B
+      const uint64_t dv_base = smem_desc_sw128(smem_u32(sV), 16, 1024);
+      constexpr uint32_t kStageStep = SM::kTileBytes >> 4;
+      auto issue_S = [&](int it) {   // S(it) = Q K^T into S buffer it&1
+        const uint64_t kd = dk_base + (it % 3) * kStageStep;
+        const uint32_t buf = tmem + 128 + (it & 1) * 128;
 #pragma unroll
         for (int kk = 0; kk < kKSteps; ++kk) {
-          const uint32_t off = (kk >> 2) * kBoxBytes + (kk & 3) * 32;
-          mma_ss(tmem, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(ka + off, 16, 1024), idesc_s, kk > 0);
+          const uint32_t c = ((kk >> 2) * kBoxBytes + (kk & 3) * 32) >> 4;
+          mma_ss(buf, dq + c, kd + c, idesc_s, kk > 0, leader);
         }
+        tc_commit(&bar->s_full[it & 1], leader);
+      };
+      auto issue_dP = [&](int it) {  // dP(it) = dO V^T
+        const uint64_t vd = dv_base + (it & 1) * kStageStep;
 #pragma unroll
         for (int kk = 0; kk < kKSteps; ++kk) {
-          const uint32_t off = (kk >> 2) * kBoxBytes + (kk & 3) * 32;
-          mma_ss(tmem + 128, smem_desc_sw128(doa + off, 16, 1024), smem_desc_sw128(va + off, 16, 1024), idesc_s, kk > 0);
+          const uint32_t c = ((kk >> 2) * kBoxBytes + (kk & 3) * 32) >> 4;
+          mma_ss(tmem + 384, ddo + c, vd + c, idesc_s, kk > 0, leader);
         }
-        tc_commit(&bar->sdp_full);
-        tc_commit(&bar->v_empty[s]);
-        if (!mbar_wait(&bar->ds_full, it & 1, abort_flag)) { ok = false; break; }
-        tc_fence_after();
+        tc_commit(&bar->dp_full, leader);
+        tc_commit(&bar->v_empty[it & 1], leader);
+      };
+      auto issue_dQ = [&](int it) {  // dQ += dS(it) K
+        const uint64_t kd = dkm_base + (it % 3) * kStageStep;
 #pragma unroll
-        for (int kk = 0; kk < kTileN / 16; ++kk)
-          mma_ts(tmem + 256, tmem + 128 + kk * 8, smem_desc_sw128(ka + kk * 2048, kBoxBytes, 1024), idesc_dq,
-                 (j > jlo) || (kk > 0));
-        tc_commit(&bar->k_empty[s]);
+        for (int kk = 0; kk < 8; ++kk)
+          mma_ts(tmem, tmem + 384 + (kk >> 1) * 32 + (kk & 1) * 8, kd + ((kk * 2048) >> 4), idesc_dq,
+                 (kk > 0 || it > 0) ? 1u : 0u, leader);
+        tc_commit(&bar->k_empty[it % 3], leader);
+      };
+      bool ok = mbar_wait_warp(&bar->q_full, 0, abort_flag) && mbar_wait_warp(&bar->k_full[0], 0, abort_flag) &&
+                mbar_wait_warp(&bar->v_full[0], 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
+        issue_S(0);
+        issue_dP(0);
+        if (n_blocks > 1) {
+          ok = mbar_wait_warp(&bar->k_full[1], 0, abort_flag);
+          if (ok) { tc_fence_after(); issue_S(1); }
+        }
       }
-      if (ok) tc_commit(&bar->final_bar);
+      for (int it = 0; ok && it < n_blocks; ++it) {
+        if (!mbar_wait_warp(&bar->ds_full, it & 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        issue_dQ(it);
+        if (it + 1 < n_blocks) {
+          if (!mbar_wait_warp(&bar->v_full[(it + 1) & 1], ((it + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          issue_dP(it + 1);
+        }
+        if (it + 2 < n_blocks) {
+          if (!mbar_wait_warp(&bar->k_full[(it + 2) % 3], ((it + 2) / 3) & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          issue_S(it + 2);
+        }
+      }
+      if (ok) tc_commit(&bar->final_bar, leader);
     }
     __syncwarp();
   } else {
-    const int r = warp * 32 + lane;
-    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+    // ------------------------------------------------------------------ P, dS and epilogue
+    const int q = warp >> 2;                        // column quarter
+    const int r = (warp & 3) * 32 + lane;           // query row == TMEM lane
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const int row = row0 + r;
     const bool valid = row < n_rows;
     const int seq_row = valid ? (a.global_mode ? q_idx_b[row] : row) : -1;
@@ -232,82 +297,73 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     const int64_t stat_idx = ((int64_t)b * a.Hq + h) * a.Lq + (valid ? row : 0);
     const float lse2 = valid ? (a.global_mode ? a.lse_glb : a.lse_loc)[stat_idx] * kLog2e : 0.f;
     const float delta = valid ? (a.global_mode ? a.delta_glb : a.delta_loc)[stat_idx] : 0.f;
+    const bool ragged = (last - row0 + 1 < kTileM);
     bool ok = true;
-    for (int j = jlo; j <= jhi; ++j) {
-      const int it = j - jlo;
-      if (!__all_sync(0xffffffffu, mbar_wait(&bar->sdp_full, it & 1, abort_flag))) { ok = false; break; }
+    for (int it = 0; it < n_blocks; ++it) {
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->s_full[it & 1], (it >> 1) & 1, abort_flag))) { ok = false; break; }
       tc_fence_after();
-      const int k0 = j * kTileN;
-      const bool partial = (k0 + kTileN - 1 > min_pos) || (k0 < max_pos - w_eff) || (last - row0 + 1 < kTileM);
+      const int k0 = (jlo + it) * kTileN + q * 32;   // first key of this quarter
+      const bool partial = (k0 + 31 > min_pos) || (k0 < max_pos - w_eff) || ragged;
+      uint32_t sv[32];
+      tmem_ld32(tmem + lane_base + 128 + (it & 1) * 128 + q * 32, sv);
+      tmem_ld_wait();
+      if (!partial) {
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {       // 64 keys at a time
-        uint32_t sv[2][32], dv[2][32];
-        tmem_ld32(tmem + lane_base + c * 64, sv[0]);
-        tmem_ld32(tmem + lane_base + c * 64 + 32, sv[1]);
-        tmem_ld32(tmem + lane_base + 128 + c * 64, dv[0]);
-        tmem_ld32(tmem + lane_base + 128 + c * 64 + 32, dv[1]);
-        tmem_ld_wait();
-        if (c == 1) {
-          // all of dP has been read: from here on the dS stores may overwrite its first half
-        }
-        uint32_t pk[32];
+        for (int e = 0; e < 32; ++e)
+          sv[e] = __float_as_uint(fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, -lse2)));
+      } else {
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
-          float ds2[2];
-#pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            const int idx = 2 * e + u;          // key within this 64-wide chunk
-            const float sc = __uint_as_float(sv[idx >> 5][idx & 31]);
-            const float dp = __uint_as_float(dv[idx >> 5][idx & 31]);
-            float p = fast_exp2(fmaf(sc, a.scale_log2, -lse2));
-            float ds = p * (dp - delta);
-            if (partial) {
-              const int kp = k0 + c * 64 + idx;
-              if (!(kp <= pos && kp >= pos_lo)) ds = 0.f;
-            }
-            ds2[u] = ds;
-          }
-          pk[e] = pack_bf16(ds2[0], ds2[1]);
+          const int kp = k0 + e;
+          const float p = fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, -lse2));
+          sv[e] = __float_as_uint((kp <= pos && kp >= pos_lo) ? p : 0.f);
         }
-        // dS chunk c -> packed columns [128 + 32c, 128 + 32c + 32).  Chunk 0 overwrites dP columns 0..31,
-        // which were read above; chunk 1 overwrites dP columns 32..63, read in chunk 0's loads as well.
-        if (c == 0) {
-          // keep chunk 0's packed values until chunk 1's dP loads (columns 64..127) are done: the stores
-          // only touch columns < 64 of dP, already consumed by this thread.
-        }
-        tmem_st32(tmem + lane_base + 128 + c * 32, pk);
       }
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->dp_full, it & 1, abort_flag))) { ok = false; break; }
+      tc_fence_after();
+      uint32_t dv[32];
+      tmem_ld32(tmem + lane_base + 384 + q * 32, dv);
+      tmem_ld_wait();
+      uint32_t pk[16];
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        const float ds0 = __uint_as_float(sv[2 * e]) * (__uint_as_float(dv[2 * e]) - delta);
+        const float ds1 = __uint_as_float(sv[2 * e + 1]) * (__uint_as_float(dv[2 * e + 1]) - delta);
+        pk[e] = pack_bf16(ds0, ds1);
+      }
+      tmem_st16(tmem + lane_base + 384 + q * 32, pk);
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(&bar->ds_full);
     }
+    // epilogue: quarter q stores D/4 columns of dQ
     if (ok && __all_sync(0xffffffffu, mbar_wait(&bar->final_bar, 0, abort_flag))) {
       tc_fence_after();
-      bf16* dst = valid ? a.dQ + (((int64_t)b * a.Lq + seq_row) * a.Hq + h) * D : nullptr;
+      constexpr int kCols = D / 4;     // 32 (D = 128) or 16 (D = 64)
+      bf16* dst = valid ? a.dQ + (((int64_t)b * a.Lq + seq_row) * a.Hq + h) * D + q * kCols : nullptr;
+      uint32_t v[32];
+      tmem_ld32(tmem + lane_base + (q * kCols & ~31), v);   // D = 64: quarters 0,1 / 2,3 share a 32-column load
+      tmem_ld_wait();
+      if (dst) {
+        constexpr int kOff = 0;
+        (void)kOff;
+        const int sub = (D == 64) ? (q & 1) * 16 : 0;
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t v[32];
-        tmem_ld32(tmem + lane_base + 256 + c * 32, v);
-        tmem_ld_wait();
-        if (dst) {
-          float f[32];
+        for (int c8 = 0; c8 < kCols / 8; ++c8) {
+          float f[8];
 #pragma unroll
-          for (int e = 0; e < 32; ++e) f[e] = __uint_as_float(v[e]) * a.scale;
-          uint4* d4 = reinterpret_cast<uint4*>(dst + c * 32);
+          for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[sub + c8 * 8 + e]) * a.scale;
+          uint4* d4 = reinterpret_cast<uint4*>(dst + c8 * 8);
+          if (a.global_mode) {
+            const uint4 old = *d4;
+            const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            if (a.global_mode) {
-              const uint4 old = d4[q];
-              const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
-#pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                f[8 * q + 2 * k] += __uint_as_float(ow[k] << 16);
-                f[8 * q + 2 * k + 1] += __uint_as_float(ow[k] & 0xffff0000u);
-              }
+            for (int k = 0; k < 4; ++k) {
+              f[2 * k] += bf16lo_to_f32(ow[k]);
+              f[2 * k + 1] += bf16hi_to_f32(ow[k]);
             }
-            d4[q] = make_uint4(pack_bf16(f[8 * q], f[8 * q + 1]), pack_bf16(f[8 * q + 2], f[8 * q + 3]),
-                               pack_bf16(f[8 * q + 4], f[8 * q + 5]), pack_bf16(f[8 * q + 6], f[8 * q + 7]));
           }
+          *d4 = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
         }
       }
     }
@@ -320,30 +376,40 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     if (tid == 0) atomicExch(a.status, 1);
     __syncthreads();
   }
-  if (warp == 5) tmem_dealloc(tmem, 512);
+  if (warp == 17) tmem_dealloc(tmem, 512);
 }
 
 // ================================================================================================
-// dK/dV kernel: one block of 128 keys of one KV head per CTA.
-//   warps 0-3: P^T / dS^T computation and epilogue (thread = key); warp 4: TMA + per-item row
-//   statistics staging; warp 5: MMA.
-//   TMEM: S^T [0,128) | dP^T [128,256) | dV [256,256+D) | dK [256+D, 256+2D).
+// dK/dV kernel: one block of 128 keys of one KV head per CTA; K and V stay in shared memory, the Q and dO
+// tiles of every query tile that can see the block stream through their own rings (Q: 3 stages, released by
+// the item's last MMA; dO: 2 stages, released earlier), so that the next tile is always resident.
+//   TMEM: dV [0,D) | dK [D,2D) | S^T [256,384) | dP^T [384,512).
+//   P^T / dS^T (bf16): quarter q puts its 16 packed columns at the start of its own 32 columns of S^T / dP^T;
+//   they are the A operands of dV += P^T dO and dK += dS^T Q.
+//   MMA order per item i:  dV(i) | S^T(i+1) | dK(i) | dP^T(i+1): the exponentials of item i+1 run under dK(i) and
+//   dP^T(i+1), its dS under dV(i+1) and S^T(i+2).
+//   Shared memory is used to the last kilobyte (7 tiles of 32 KB at D = 128): the dynamic segment must start
+//   1024-byte aligned, which the kernel checks instead of padding.
 template <int D>
 struct DkvSmem {
   static constexpr int kTileBytes = 128 * D * 2;
+  static constexpr int kQStages = 3;
+  static constexpr int kDoStages = 2;
   static constexpr int kKOff = 0;
   static constexpr int kVOff = kTileBytes;
-  static constexpr int kQOff = 2 * kTileBytes;       // 2 stages
-  static constexpr int kDoOff = 4 * kTileBytes;      // 2 stages
-  static constexpr int kStatOff = 6 * kTileBytes;    // 2 stages x {lse2[128], delta[128], pos[128], flags[4]}
-  static constexpr int kStatStage = (3 * 128 + 4) * 4;
-  static constexpr int kBarOff = kStatOff + 2 * kStatStage + 16;
-  static constexpr int kTotal = kBarOff + 256 + 1024;
+  static constexpr int kQOff = 2 * kTileBytes;
+  static constexpr int kDoOff = kQOff + kQStages * kTileBytes;
+  static constexpr int kStatOff = kDoOff + kDoStages * kTileBytes;   // 2 slots x {lse2[128], delta[128], flags[8]}
+  static constexpr int kStatSlot = (2 * 128 + 8) * 4;
+  static constexpr int kBarOff = kStatOff + 2 * kStatSlot;
+  static constexpr int kTotal = kBarOff + 256;
 };
 struct DkvBarriers {
   uint64_t kv_full;
-  uint64_t qdo_full[2], qdo_empty[2];
-  uint64_t sdp_full, pds_full, final_bar;
+  uint64_t q_full[3], q_empty[3];
+  uint64_t do_full[2], do_empty[2];
+  uint64_t st_full[2], st_empty[2];
+  uint64_t s_full, dp_full, p_full, ds_full, final_bar;
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -377,13 +443,23 @@ __device__ __forceinline__ ItemPlan make_plan(const BwdArgs& a, int b, int k0) {
   return p;
 }
 
+// Walks the items of a CTA in order without divisions: (head, local/compact, tile).
+struct ItemCursor {
+  int h, r, per_head, loc_nt, loc_t0, glb_t0;
+  __device__ __forceinline__ ItemCursor(const ItemPlan& p, int h0)
+      : h(h0), r(0), per_head(p.per_head), loc_nt(p.loc_nt), loc_t0(p.loc_t0), glb_t0(p.glb_t0) {}
+  __device__ __forceinline__ int glb() const { return r >= loc_nt; }
+  __device__ __forceinline__ int tile() const { return r < loc_nt ? loc_t0 + r : glb_t0 + (r - loc_nt); }
+  __device__ __forceinline__ void next() { if (++r == per_head) { r = 0; ++h; } }
+};
+
 template <int D>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kDkvThreads, 1)
 bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapDO,
                const __grid_constant__ CUtensorMap mapQc, const __grid_constant__ CUtensorMap mapDOc,
                const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, const BwdArgs a) {
   using SM = DkvSmem<D>;
-  constexpr int kDBoxes = D / 64, kKSteps = D / 16;
+  constexpr int kKSteps = D / 16;
   const int n_kblocks = (a.Lk + kTileN - 1) / kTileN;
   // key blocks ascending (most work first) inside one KV head; KV heads outermost so that the CTAs
   // running together share the same query tiles in L2
@@ -396,8 +472,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   const ItemPlan plan = make_plan(a, b, k0);
   const int n_c = a.n_routed[b];
 
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  extern __shared__ __align__(1024) uint8_t smem[];
   uint8_t* sK = smem + SM::kKOff;
   uint8_t* sV = smem + SM::kVOff;
   uint8_t* sQ = smem + SM::kQOff;
@@ -406,6 +481,10 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   volatile int* abort_flag = &bar->abort_flag;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
+  if ((smem_u32(smem) & 1023u) != 0) {   // the swizzled tiles need a 1024-byte aligned base: refuse to run otherwise
+    if (tid == 0) atomicExch(a.status, 2);
+    return;
+  }
   if (plan.total == 0) {
     // no query can see these keys: their gradients are zero
     for (int i = tid; i < kTileN * (D / 8); i += blockDim.x) {
@@ -421,204 +500,305 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 
   if (tid == 0) {
     mbar_init(&bar->kv_full, 1);
-    for (int s = 0; s < 2; ++s) { mbar_init(&bar->qdo_full[s], 33); mbar_init(&bar->qdo_empty[s], 1); }
-    mbar_init(&bar->sdp_full, 1);
-    mbar_init(&bar->pds_full, 128);
+    for (int s = 0; s < 3; ++s) { mbar_init(&bar->q_full[s], 1); mbar_init(&bar->q_empty[s], 1); }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&bar->do_full[s], 1); mbar_init(&bar->do_empty[s], 1);
+      mbar_init(&bar->st_full[s], 32); mbar_init(&bar->st_empty[s], kComputeWarps * 32);
+    }
+    mbar_init(&bar->s_full, 1);
+    mbar_init(&bar->dp_full, 1);
+    mbar_init(&bar->p_full, kComputeWarps * 32);
+    mbar_init(&bar->ds_full, kComputeWarps * 32);
     mbar_init(&bar->final_bar, 1);
     bar->abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 5) { tmem_alloc(&bar->tmem_base, 512); tmem_relinquish(); }
+  if (warp == 17) { tmem_alloc(&bar->tmem_base, 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bar->tmem_base;
 
-  // item i -> (head, mode, tile)
-  auto decode = [&](int i, int& h, int& glb, int& tile) {
-    const int hh = i / plan.per_head, r = i % plan.per_head;
-    h = g * G + hh;
-    if (r < plan.loc_nt) { glb = 0; tile = plan.loc_t0 + r; }
-    else { glb = 1; tile = plan.glb_t0 + (r - plan.loc_nt); }
-  };
-
-  if (warp == 4) {
-    // ------------------------------------------------------------------ producer: TMA + statistics
+  if (warp == 16) {
+    // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&mapQ); tma_prefetch_desc(&mapDO); tma_prefetch_desc(&mapQc); tma_prefetch_desc(&mapDOc);
       mbar_expect_tx(&bar->kv_full, 2 * SM::kTileBytes);
-      for (int x = 0; x < kDBoxes; ++x) {
-        tma_load_3d(sK + x * kBoxBytes, &mapK, &bar->kv_full, g * D + x * 64, k0, b);
-        tma_load_3d(sV + x * kBoxBytes, &mapV, &bar->kv_full, g * D + x * 64, k0, b);
+      tma_load_4d(sK, &mapK, &bar->kv_full, 0, k0, g * (D / 64), b);
+      tma_load_4d(sV, &mapV, &bar->kv_full, 0, k0, g * (D / 64), b);
+      ItemCursor cur(plan, g * G);
+      int qs = 0;
+      uint32_t qph = 0;
+      for (int i = 0; i < plan.total; ++i) {
+        const int glb = cur.glb(), row0 = cur.tile() * kTileM, hc = cur.h * (D / 64);
+        cur.next();
+        if (!mbar_wait(&bar->q_empty[qs], qph ^ 1, abort_flag)) break;
+        L2A_TRACE_POINT(3, 2 * i);
+        mbar_expect_tx(&bar->q_full[qs], SM::kTileBytes);
+        tma_load_4d(sQ + qs * SM::kTileBytes, glb ? &mapQc : &mapQ, &bar->q_full[qs], 0, row0, hc, b);
+        if (!mbar_wait(&bar->do_empty[i & 1], ((i >> 1) & 1) ^ 1, abort_flag)) break;
+        mbar_expect_tx(&bar->do_full[i & 1], SM::kTileBytes);
+        tma_load_4d(sDO + (i & 1) * SM::kTileBytes, glb ? &mapDOc : &mapDO, &bar->do_full[i & 1], 0, row0, hc, b);
+        L2A_TRACE_POINT(3, 2 * i + 1);
+        if (++qs == 3) { qs = 0; qph ^= 1; }
       }
     }
-    bool ok = true;
-    for (int i = 0; i < plan.total; ++i) {
-      const int s = i & 1;
-      const uint32_t ph = (i >> 1) & 1;
-      int h, glb, tile;
-      decode(i, h, glb, tile);
-      const int row0 = tile * kTileM;
-      if (!__all_sync(0xffffffffu, mbar_wait(&bar->qdo_empty[s], ph ^ 1, abort_flag))) { ok = false; break; }
-      if (lane == 0) {
-        mbar_expect_tx(&bar->qdo_full[s], 2 * SM::kTileBytes);
-        for (int x = 0; x < kDBoxes; ++x) {
-          tma_load_3d(sQ + s * SM::kTileBytes + x * kBoxBytes, glb ? &mapQc : &mapQ, &bar->qdo_full[s],
-                      h * D + x * 64, row0, b);
-          tma_load_3d(sDO + s * SM::kTileBytes + x * kBoxBytes, glb ? &mapDOc : &mapDO, &bar->qdo_full[s],
-                      h * D + x * 64, row0, b);
-        }
-      }
-      float* st_lse = reinterpret_cast<float*>(smem + SM::kStatOff + s * SM::kStatStage);
-      float* st_delta = st_lse + 128;
-      int* st_pos = reinterpret_cast<int*>(st_delta + 128);
-      int* st_flags = st_pos + 128;
+    __syncwarp();
+  } else if (warp == 18) {
+    // ------------------------------------------------------------------ row statistics of each item
+    // lse * log2(e) and Delta of the item's 128 query rows, plus per-quarter mask flags, go to shared memory.
+    // The global loads of item i+1 are issued before waiting for its slot, so their latency is hidden.
+    float r_lse[4], r_delta[4];
+    int r_pos[4], r_glb = 0, r_row0 = 0;
+    ItemCursor cur(plan, g * G);
+    auto load_item = [&]() {
+      const int h = cur.h, glb = cur.glb(), row0 = cur.tile() * kTileM;
+      cur.next();
       const int n_rows = glb ? n_c : a.Lq;
       const float* lse = glb ? a.lse_glb : a.lse_loc;
       const float* dl = glb ? a.delta_glb : a.delta_loc;
-      int pmin = 0x7fffffff, pmax = -1, all_valid = 1;
+      r_glb = glb;
+      r_row0 = row0;
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const int col = q * 32 + lane, row = row0 + col;
+        const int row = row0 + q * 32 + lane;
         const bool valid = row < n_rows;
         const int64_t si = ((int64_t)b * a.Hq + h) * a.Lq + (valid ? row : 0);
-        st_lse[col] = valid ? lse[si] * kLog2e : 0.f;
-        st_delta[col] = valid ? dl[si] : 0.f;
-        const int pos = valid ? (glb ? a.q_idx[(int64_t)b * a.Lq + row] : row) + a.q_pos_offset : -1;
-        st_pos[col] = pos;
-        if (valid) { pmin = min(pmin, pos); pmax = max(pmax, pos); } else all_valid = 0;
+        r_lse[q] = valid ? __ldg(&lse[si]) * kLog2e : 0.f;
+        r_delta[q] = valid ? __ldg(&dl[si]) : 0.f;
+        r_pos[q] = valid ? (glb ? __ldg(&a.q_idx[(int64_t)b * a.Lq + row]) : row) + a.q_pos_offset : -1;
       }
+    };
+    load_item();
+    for (int i = 0; i < plan.total; ++i) {
+      const int s = i & 1;
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->st_empty[s], ((i >> 1) & 1) ^ 1, abort_flag))) break;
+      float* st_lse = reinterpret_cast<float*>(smem + SM::kStatOff + s * SM::kStatSlot);
+      float* st_delta = st_lse + 128;
+      int* st_flags = reinterpret_cast<int*>(st_delta + 128);
+      const int w_eff = r_glb ? 0x3fffffff : a.window;
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        pmin = min(pmin, __shfl_xor_sync(0xffffffffu, pmin, o));
-        pmax = max(pmax, __shfl_xor_sync(0xffffffffu, pmax, o));
-        all_valid &= __shfl_xor_sync(0xffffffffu, all_valid, o);
+      for (int q = 0; q < 4; ++q) {
+        const int col = q * 32 + lane;
+        st_lse[col] = r_lse[q];
+        st_delta[col] = r_delta[q];
+        // quarter q needs the element mask unless every (key, query) pair of it is visible
+        const bool lane_ok = r_pos[q] >= 0 && (k0 + kTileN - 1 <= r_pos[q]) && (k0 >= r_pos[q] - w_eff);
+        const bool interior = __all_sync(0xffffffffu, lane_ok);
+        if (lane == 0) st_flags[q] = interior ? 0 : 1;
       }
-      if (lane == 0) {
-        const int w_eff = glb ? 0x3fffffff : a.window;
-        const int interior = all_valid && (k0 + kTileN - 1 <= pmin) && (k0 >= pmax - w_eff);
-        st_flags[0] = interior ? 0 : 1;     // 1 = apply the element mask
-        st_flags[1] = glb;
-      }
+      if (lane == 0) { st_flags[4] = r_glb; st_flags[5] = r_row0; }
       __syncwarp();
-      mbar_arrive(&bar->qdo_full[s]);
+      mbar_arrive(&bar->st_full[s]);
+      if (i + 1 < plan.total) load_item();
     }
-    (void)ok;
-  } else if (warp == 5) {
+  } else if (warp == 17) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // (whole warp runs the loop; only the tcgen05 instructions are predicated on lane 0)
+    {
+      const uint32_t leader = (lane == 0);
       constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);
       constexpr uint32_t idesc_acc = idesc_bf16_f32(128, D, 0, 1);
-      bool ok = mbar_wait(&bar->kv_full, 0, abort_flag);
-      const uint32_t ka = smem_u32(sK), va = smem_u32(sV);
-      for (int i = 0; ok && i < plan.total; ++i) {
-        const int s = i & 1;
-        const uint32_t ph = (i >> 1) & 1;
-        if (!mbar_wait(&bar->qdo_full[s], ph, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t qa = smem_u32(sQ + s * SM::kTileBytes), doa = smem_u32(sDO + s * SM::kTileBytes);
+      constexpr uint32_t kStageStep = SM::kTileBytes >> 4;
+      const uint64_t dk = smem_desc_sw128(smem_u32(sK), 16, 1024), dv = smem_desc_sw128(smem_u32(sV), 16, 1024);
+      const uint64_t dq_base = smem_desc_sw128(smem_u32(sQ), 16, 1024);
+      const uint64_t ddo_base = smem_desc_sw128(smem_u32(sDO), 16, 1024);
+      const uint64_t dqm_base = smem_desc_sw128(smem_u32(sQ), kBoxBytes, 1024);      // Q / dO as MN-major B
+      const uint64_t ddom_base = smem_desc_sw128(smem_u32(sDO), kBoxBytes, 1024);
+      auto issue_S = [&](int qs) {    // S^T = K Q^T
+        const uint64_t qd = dq_base + qs * kStageStep;
 #pragma unroll
-        for (int kk = 0; kk < kKSteps; ++kk) {   // S^T = K Q^T
-          const uint32_t off = (kk >> 2) * kBoxBytes + (kk & 3) * 32;
-          mma_ss(tmem, smem_desc_sw128(ka + off, 16, 1024), smem_desc_sw128(qa + off, 16, 1024), idesc_s, kk > 0);
+        for (int kk = 0; kk < kKSteps; ++kk) {
+          const uint32_t c = ((kk >> 2) * kBoxBytes + (kk & 3) * 32) >> 4;
+          mma_ss(tmem + 256, dk + c, qd + c, idesc_s, kk > 0, leader);
         }
+        tc_commit(&bar->s_full, leader);
+      };
+      auto issue_dP = [&](int ds) {   // dP^T = V dO^T
+        const uint64_t dod = ddo_base + ds * kStageStep;
 #pragma unroll
-        for (int kk = 0; kk < kKSteps; ++kk) {   // dP^T = V dO^T
-          const uint32_t off = (kk >> 2) * kBoxBytes + (kk & 3) * 32;
-          mma_ss(tmem + 128, smem_desc_sw128(va + off, 16, 1024), smem_desc_sw128(doa + off, 16, 1024), idesc_s, kk > 0);
+        for (int kk = 0; kk < kKSteps; ++kk) {
+          const uint32_t c = ((kk >> 2) * kBoxBytes + (kk & 3) * 32) >> 4;
+          mma_ss(tmem + 384, dv + c, dod + c, idesc_s, kk > 0, leader);
         }
-        tc_commit(&bar->sdp_full);
-        if (!mbar_wait(&bar->pds_full, i & 1, abort_flag)) { ok = false; break; }
+        tc_commit(&bar->dp_full, leader);
+      };
+      auto issue_dV = [&](int ds, bool first) {   // dV += P^T dO
+        const uint64_t dod = ddom_base + ds * kStageStep;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          mma_ts(tmem, tmem + 256 + (kk >> 1) * 32 + (kk & 1) * 8, dod + ((kk * 2048) >> 4), idesc_acc,
+                 (kk > 0 || !first) ? 1u : 0u, leader);
+        tc_commit(&bar->do_empty[ds], leader);
+      };
+      auto issue_dK = [&](int qs, bool first) {   // dK += dS^T Q
+        const uint64_t qd = dqm_base + qs * kStageStep;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          mma_ts(tmem + D, tmem + 384 + (kk >> 1) * 32 + (kk & 1) * 8, qd + ((kk * 2048) >> 4), idesc_acc,
+                 (kk > 0 || !first) ? 1u : 0u, leader);
+        tc_commit(&bar->q_empty[qs], leader);
+      };
+      bool ok = mbar_wait_warp(&bar->kv_full, 0, abort_flag) && mbar_wait_warp(&bar->q_full[0], 0, abort_flag) &&
+                mbar_wait_warp(&bar->do_full[0], 0, abort_flag);
+      if (ok) {
         tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < kTileM / 16; ++kk)   // dV += P^T dO
-          mma_ts(tmem + 256, tmem + kk * 8, smem_desc_sw128(doa + kk * 2048, kBoxBytes, 1024), idesc_acc,
-                 (i > 0) || (kk > 0));
-#pragma unroll
-        for (int kk = 0; kk < kTileM / 16; ++kk)   // dK += dS^T Q
-          mma_ts(tmem + 256 + D, tmem + 128 + kk * 8, smem_desc_sw128(qa + kk * 2048, kBoxBytes, 1024), idesc_acc,
-                 (i > 0) || (kk > 0));
-        tc_commit(&bar->qdo_empty[s]);
+        issue_S(0);
+        issue_dP(0);
       }
-      if (ok) tc_commit(&bar->final_bar);
+      int qs = 0;           // Q stage of item i
+      uint32_t qph = 0;     // its phase parity
+      for (int i = 0; ok && i < plan.total; ++i) {
+        const bool more = i + 1 < plan.total;
+        int qn = qs + 1;
+        uint32_t qphn = qph;
+        if (qn == 3) { qn = 0; qphn ^= 1; }
+        if (!mbar_wait_warp(&bar->p_full, i & 1, abort_flag)) { ok = false; break; }
+        if (lane == 0) L2A_TRACE_POINT(0, 4 * i);
+        tc_fence_after();
+        issue_dV(i & 1, i == 0);
+        if (lane == 0) L2A_TRACE_POINT(2, 4 * i + 3);
+        if (more) {
+          if (!mbar_wait_warp(&bar->q_full[qn], qphn, abort_flag)) { ok = false; break; }
+          if (lane == 0) L2A_TRACE_POINT(0, 4 * i + 1);
+          tc_fence_after();
+          issue_S(qn);
+        }
+        if (!mbar_wait_warp(&bar->ds_full, i & 1, abort_flag)) { ok = false; break; }
+        if (lane == 0) L2A_TRACE_POINT(0, 4 * i + 2);
+        tc_fence_after();
+        issue_dK(qs, i == 0);
+        if (more) {
+          if (!mbar_wait_warp(&bar->do_full[(i + 1) & 1], ((i + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          issue_dP((i + 1) & 1);
+        }
+        if (lane == 0) L2A_TRACE_POINT(0, 4 * i + 3);
+        qs = qn;
+        qph = qphn;
+      }
+      if (ok) tc_commit(&bar->final_bar, leader);
     }
     __syncwarp();
   } else {
     // ------------------------------------------------------------------ P^T / dS^T and epilogue
-    const int kr = warp * 32 + lane;           // key inside the block == TMEM lane
+    const int q = warp >> 2;                           // query-column quarter of this warp
+    const int kr = (warp & 3) * 32 + lane;             // key inside the block == TMEM lane
     const int kp = k0 + kr;
-    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const uint32_t s_addr = tmem + lane_base + 256 + q * 32;
+    const uint32_t dp_addr = tmem + lane_base + 384 + q * 32;
     bool ok = true;
     for (int i = 0; i < plan.total; ++i) {
       const int s = i & 1;
-      if (!__all_sync(0xffffffffu, mbar_wait(&bar->sdp_full, i & 1, abort_flag))) { ok = false; break; }
-      tc_fence_after();
-      const float* st_lse = reinterpret_cast<const float*>(smem + SM::kStatOff + s * SM::kStatStage);
-      const float* st_delta = st_lse + 128;
-      const int* st_pos = reinterpret_cast<const int*>(st_delta + 128);
-      const int* st_flags = st_pos + 128;
-      const bool masked = st_flags[0] != 0;
-      const int w_eff = st_flags[1] ? 0x3fffffff : a.window;
+      // this item's row statistics go to registers before the scores are waited for
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->st_full[s], (i >> 1) & 1, abort_flag))) { ok = false; break; }
+      const uint32_t st_base = smem_u32(smem + SM::kStatOff + s * SM::kStatSlot);
+      const int* st_flags = reinterpret_cast<const int*>(smem + SM::kStatOff + s * SM::kStatSlot) + 2 * 128;
+      float st[32];
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {   // 64 query columns at a time
-        uint32_t sv[2][32], dv[2][32];
-        tmem_ld32(tmem + lane_base + c * 64, sv[0]);
-        tmem_ld32(tmem + lane_base + c * 64 + 32, sv[1]);
-        tmem_ld32(tmem + lane_base + 128 + c * 64, dv[0]);
-        tmem_ld32(tmem + lane_base + 128 + c * 64 + 32, dv[1]);
-        tmem_ld_wait();
-        uint32_t pp[32], pd[32];
-#pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          float p2[2], ds2[2];
-#pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            const int idx = 2 * e + u, col = c * 64 + idx;
-            const float sc = __uint_as_float(sv[idx >> 5][idx & 31]);
-            const float dp = __uint_as_float(dv[idx >> 5][idx & 31]);
-            float p = fast_exp2(fmaf(sc, a.scale_log2, -st_lse[col]));
-            float ds = p * (dp - st_delta[col]);
-            if (masked) {
-              const int pos = st_pos[col];
-              if (!(kp <= pos && kp >= pos - w_eff)) { p = 0.f; ds = 0.f; }
-            }
-            p2[u] = p; ds2[u] = ds;
-          }
-          pp[e] = pack_bf16(p2[0], p2[1]);
-          pd[e] = pack_bf16(ds2[0], ds2[1]);
-        }
-        // P^T chunk c -> S^T columns [32c, 32c+32); dS^T chunk c -> dP^T columns [32c, 32c+32): both ranges
-        // lie inside the columns this thread has already loaded (chunk 0 reads 0..63, chunk 1 reads 64..127)
-        tmem_st32(tmem + lane_base + c * 32, pp);
-        tmem_st32(tmem + lane_base + 128 + c * 32, pd);
+      for (int c = 0; c < 8; ++c) {
+        const float4 v = lds128(st_base + (q * 32 + c * 4) * 4);
+        st[4 * c] = v.x; st[4 * c + 1] = v.y; st[4 * c + 2] = v.z; st[4 * c + 3] = v.w;
       }
+      const bool masked = st_flags[q] != 0;
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->s_full, i & 1, abort_flag))) { ok = false; break; }
+      if (warp == 0 && lane == 0) L2A_TRACE_POINT(1, 4 * i);
+      tc_fence_after();
+      uint32_t pp[16];
+      {
+        uint32_t sv[32];
+        tmem_ld32(s_addr, sv);
+        tmem_ld_wait();
+        if (warp == 0 && lane == 0) L2A_TRACE_POINT(2, 4 * i);
+        // the element mask is needed only for the few tiles that straddle the causal diagonal or a window edge:
+        // two loop versions, so that the common one has no branches
+        if (!masked) {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * e]), a.scale_log2, -st[2 * e]));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * e + 1]), a.scale_log2, -st[2 * e + 1]));
+            pp[e] = pack_bf16(p0, p1);
+          }
+        } else {
+          const int glb = st_flags[4], row0 = st_flags[5];
+          const int w_eff = glb ? 0x3fffffff : a.window;
+          const int n_rows = glb ? n_c : a.Lq;
+          const int32_t* qi = a.q_idx + (int64_t)b * a.Lq;
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            int pos[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+              const int row = row0 + q * 32 + e + u;
+              pos[u] = row < n_rows ? (glb ? __ldg(&qi[row]) : row) + a.q_pos_offset : -1;
+            }
+            float p0 = fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, -st[e]));
+            float p1 = fast_exp2(fmaf(__uint_as_float(sv[e + 1]), a.scale_log2, -st[e + 1]));
+            p0 = (kp <= pos[0] && kp >= pos[0] - w_eff) ? p0 : 0.f;
+            p1 = (kp <= pos[1] && kp >= pos[1] - w_eff) ? p1 : 0.f;
+            pp[e >> 1] = pack_bf16(p0, p1);
+          }
+        }
+      }
+      if (warp == 0 && lane == 0) L2A_TRACE_POINT(2, 4 * i + 1);
+      tmem_st16(s_addr, pp);     // P^T over the first half of this quarter's own S^T columns
+      tmem_st_wait();
+      if (warp == 0 && lane == 0) L2A_TRACE_POINT(2, 4 * i + 2);
+      tc_fence_before();
+      mbar_arrive(&bar->p_full);
+      if (warp == 0 && lane == 0) L2A_TRACE_POINT(1, 4 * i + 1);
+      // Delta of the same rows, again ahead of the wait; after this the statistics slot may be refilled
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const float4 v = lds128(st_base + (128 + q * 32 + c * 4) * 4);
+        st[4 * c] = v.x; st[4 * c + 1] = v.y; st[4 * c + 2] = v.z; st[4 * c + 3] = v.w;
+      }
+      mbar_arrive(&bar->st_empty[s]);
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->dp_full, i & 1, abort_flag))) { ok = false; break; }
+      if (warp == 0 && lane == 0) L2A_TRACE_POINT(1, 4 * i + 2);
+      tc_fence_after();
+      uint32_t pd[16];
+      {
+        uint32_t dv[32];
+        tmem_ld32(dp_addr, dv);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          // dS uses the bf16-rounded P, the same value the dV product sees
+          const float ds0 = bf16lo_to_f32(pp[e]) * (__uint_as_float(dv[2 * e]) - st[2 * e]);
+          const float ds1 = bf16hi_to_f32(pp[e]) * (__uint_as_float(dv[2 * e + 1]) - st[2 * e + 1]);
+          pd[e] = pack_bf16(ds0, ds1);
+        }
+      }
+      tmem_st16(dp_addr, pd);    // dS^T over the first half of this quarter's own dP^T columns
       tmem_st_wait();
       tc_fence_before();
-      mbar_arrive(&bar->pds_full);
+      mbar_arrive(&bar->ds_full);
+      if (warp == 0 && lane == 0) L2A_TRACE_POINT(1, 4 * i + 3);
     }
+    // epilogue: quarters 0,1 store the two column halves of dV, quarters 2,3 those of dK
     if (ok && __all_sync(0xffffffffu, mbar_wait(&bar->final_bar, 0, abort_flag))) {
       tc_fence_after();
       const bool valid = kp < a.Lk;
-      const int64_t o = (((int64_t)b * a.Lk + (valid ? kp : 0)) * a.Hkv + g) * D;
+      const int which = q >> 1, half = q & 1;
+      const int64_t o = (((int64_t)b * a.Lk + (valid ? kp : 0)) * a.Hkv + g) * D + half * (D / 2);
+      bf16* dst = (which == 0 ? a.dV : a.dK) + o;
+      const float mul = which == 0 ? 1.0f : a.scale;
 #pragma unroll
-      for (int which = 0; which < 2; ++which) {
-        bf16* dst = (which == 0 ? a.dV : a.dK) + o;
-        const float mul = which == 0 ? 1.0f : a.scale;
+      for (int c = 0; c < D / 64; ++c) {
+        uint32_t v[32];
+        tmem_ld32(tmem + lane_base + which * D + half * (D / 2) + c * 32, v);
+        tmem_ld_wait();
+        if (valid) {
+          uint4* d4 = reinterpret_cast<uint4*>(dst + c * 32);
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t v[32];
-          tmem_ld32(tmem + lane_base + 256 + which * D + c * 32, v);
-          tmem_ld_wait();
-          if (valid) {
-            uint4* d4 = reinterpret_cast<uint4*>(dst + c * 32);
+          for (int x = 0; x < 4; ++x) {
+            float f[8];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              float f[8];
-#pragma unroll
-              for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[8 * q + e]) * mul;
-              d4[q] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
-                                 pack_bf16(f[6], f[7]));
-            }
+            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[8 * x + e]) * mul;
+            d4[x] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
+                               pack_bf16(f[6], f[7]));
           }
         }
       }
@@ -632,7 +812,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     if (tid == 0) atomicExch(a.status, 1);
     __syncthreads();
   }
-  if (warp == 5) tmem_dealloc(tmem, 512);
+  if (warp == 17) tmem_dealloc(tmem, 512);
 }
 
 size_t rows_bytes(const l2a_params* p) { return align_up((size_t)p->B * p->Lq * p->Hq * p->D * sizeof(bf16), 256); }
@@ -650,16 +830,16 @@ cudaError_t launch_bwd_kernels(const BwdArgs& base, const CUtensorMap& mapQ, con
   e = cudaFuncSetAttribute(bwd_dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<D>::kTotal);
   if (e != cudaSuccess) return e;
   const unsigned n_kblocks = (base.Lk + kTileN - 1) / kTileN;
-  bwd_dkv_kernel<D><<<n_kblocks * base.B * base.Hkv, 192, DkvSmem<D>::kTotal, s>>>(mapQ, mapDO, mapQc, mapDOc, mapK,
+  bwd_dkv_kernel<D><<<n_kblocks * base.B * base.Hkv, kDkvThreads, DkvSmem<D>::kTotal, s>>>(mapQ, mapDO, mapQc, mapDOc, mapK,
                                                                                   mapV, base);
   phase_events().mark(s);
   const unsigned n_tiles = (base.Lq + kTileM - 1) / kTileM;
   BwdArgs a = base;
   a.global_mode = 0;
-  bwd_dq_kernel<D><<<n_tiles * base.B * base.Hq, 192, DqSmem<D>::kTotal, s>>>(mapQ, mapDO, mapK, mapV, a);
+  bwd_dq_kernel<D><<<n_tiles * base.B * base.Hq, kDqThreads, DqSmem<D>::kTotal, s>>>(mapQ, mapDO, mapK, mapV, a);
   phase_events().mark(s);
   a.global_mode = 1;
-  bwd_dq_kernel<D><<<n_tiles * base.B * base.Hq, 192, DqSmem<D>::kTotal, s>>>(mapQc, mapDOc, mapK, mapV, a);
+  bwd_dq_kernel<D><<<n_tiles * base.B * base.Hq, kDqThreads, DqSmem<D>::kTotal, s>>>(mapQc, mapDOc, mapK, mapV, a);
   phase_events().mark(s);
   return cudaGetLastError();
 }
@@ -671,6 +851,12 @@ size_t bwd_ws_size(const l2a_params* p) { return kWsHeaderBytes + 2 * rows_bytes
 }  // namespace l2a
 
 using namespace l2a;
+
+#ifdef L2A_TRACE
+extern "C" int l2a_debug_read_trace(long long* host) {
+  return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(g_trace));
+}
+#endif
 
 extern "C" l2a_status l2a_backward(const l2a_params* p, const void* Q, const void* K, const void* V,
                                    const uint8_t* d_mask, const int32_t* q_idx, const int32_t* n_routed,
@@ -698,12 +884,12 @@ extern "C" l2a_status l2a_backward(const l2a_params* p, const void* Q, const voi
   float* delta_glb = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + stat_bytes(p));
 
   CUtensorMap mapQ, mapDO, mapQc, mapDOc, mapK, mapV;
-  if (!encode_rows_map(&mapQ, Q, p->B, p->Lq, p->Hq * p->D, kTileM) ||
-      !encode_rows_map(&mapDO, dO, p->B, p->Lq, p->Hq * p->D, kTileM) ||
-      !encode_rows_map(&mapQc, Qc, p->B, p->Lq, p->Hq * p->D, kTileM) ||
-      !encode_rows_map(&mapDOc, dOc, p->B, p->Lq, p->Hq * p->D, kTileM) ||
-      !encode_rows_map(&mapK, K, p->B, p->Lk, p->Hkv * p->D, kTileN) ||
-      !encode_rows_map(&mapV, V, p->B, p->Lk, p->Hkv * p->D, kTileN))
+  if (!encode_rows_map(&mapQ, Q, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||
+      !encode_rows_map(&mapDO, dO, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||
+      !encode_rows_map(&mapQc, Qc, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||
+      !encode_rows_map(&mapDOc, dOc, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||
+      !encode_rows_map(&mapK, K, p->B, p->Lk, p->Hkv * p->D, kTileN, p->D) ||
+      !encode_rows_map(&mapV, V, p->B, p->Lk, p->Hkv * p->D, kTileN, p->D))
     return L2A_ERR_CUDA;
 
   PhaseEvents& pe = phase_events();

@@ -147,99 +147,114 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       for (int t = 0; t < kNumTiles; ++t) {
         if (!tr[t].active) continue;
         mbar_expect_tx(&bar->q_full[t], SM::kQTileBytes);
-        for (int x = 0; x < kDBoxes; ++x)
-          tma_load_3d(sQ + t * SM::kQTileBytes + x * SM::kBoxBytes, &mapQ, &bar->q_full[t], h * D + x * 64,
-                      row0 + t * kTileM, b);
+        tma_load_4d(sQ + t * SM::kQTileBytes, &mapQ, &bar->q_full[t], 0, row0 + t * kTileM, h * (D / 64), b);
       }
       for (int j = jlo; j <= jhi; ++j) {
         const int it = j - jlo, s = it % kStages;
         const uint32_t ph = (it / kStages) & 1;
         if (!mbar_wait(&bar->k_empty[s], ph ^ 1, abort_flag)) break;
         mbar_expect_tx(&bar->k_full[s], SM::kKVTileBytes);
-        for (int x = 0; x < kDBoxes; ++x)
-          tma_load_3d(sK + s * SM::kKVTileBytes + x * SM::kBoxBytes, &mapK, &bar->k_full[s], g * D + x * 64,
-                      j * kTileN, b);
+        tma_load_4d(sK + s * SM::kKVTileBytes, &mapK, &bar->k_full[s], 0, j * kTileN, g * (D / 64), b);
         if (!mbar_wait(&bar->v_empty[s], ph ^ 1, abort_flag)) break;
         mbar_expect_tx(&bar->v_full[s], SM::kKVTileBytes);
-        for (int x = 0; x < kDBoxes; ++x)
-          tma_load_3d(sV + s * SM::kKVTileBytes + x * SM::kBoxBytes, &mapV, &bar->v_full[s], g * D + x * 64,
-                      j * kTileN, b);
+        tma_load_4d(sV + s * SM::kKVTileBytes, &mapV, &bar->v_full[s], 0, j * kTileN, g * (D / 64), b);
       }
     }
     __syncwarp();
   } else if (warp == 9) {
     // =========================================================================== MMA issuer
-    if (lane == 0) {
+    // The whole warp runs this loop (uniform control flow keeps the descriptor arithmetic in uniform registers);
+    // only the tcgen05 instructions themselves are predicated on lane 0.  Operand descriptors are built once per
+    // tile / stage and advanced by compile-time constants, so that issuing stays well under the 64 clocks one
+    // 128x128x16 MMA takes.
+    {
+      const uint32_t leader = (lane == 0);
+      static_assert(kStages == 2 && kNumTiles == 2, "descriptor selects below assume two stages and two tiles");
       constexpr uint32_t idesc_qk = idesc_bf16_f32(kTileM, kTileN, 0, 0);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(kTileM, D, 0, 1);
-      uint32_t p_cnt[kNumTiles] = {0, 0};
+      const uint64_t dq0 = smem_desc_sw128(smem_u32(sQ), 16, 1024);
+      const uint64_t dq1 = smem_desc_sw128(smem_u32(sQ + SM::kQTileBytes), 16, 1024);
+      const uint64_t dk0 = smem_desc_sw128(smem_u32(sK), 16, 1024);
+      const uint64_t dk1 = smem_desc_sw128(smem_u32(sK + SM::kKVTileBytes), 16, 1024);
+      const uint64_t dv0 = smem_desc_sw128(smem_u32(sV), SM::kBoxBytes, 1024);
+      const uint64_t dv1 = smem_desc_sw128(smem_u32(sV + SM::kKVTileBytes), SM::kBoxBytes, 1024);
+      const int lo0 = tr[0].lo, hi0 = tr[0].hi, lo1 = tr[1].lo, hi1 = tr[1].hi;  // an inactive tile has lo > hi
+      uint32_t p_cnt0 = 0, p_cnt1 = 0;
       bool ok = true;
 
-      auto issue_qk = [&](int t, int j) {
-        const int s = (j - jlo) % kStages;
-        const uint32_t qa = smem_u32(sQ + t * SM::kQTileBytes);
-        const uint32_t ka = smem_u32(sK + s * SM::kKVTileBytes);
+      auto issue_qk = [&](int t, int s) {
+        const uint64_t qd = t ? dq1 : dq0, kd = s ? dk1 : dk0;
+        const uint32_t d = tmem + t * kTileN;
 #pragma unroll
         for (int kk = 0; kk < kKSteps; ++kk) {
-          const uint32_t off = (kk >> 2) * SM::kBoxBytes + (kk & 3) * 32;
-          mma_ss(tmem + t * kTileN, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(ka + off, 16, 1024),
-                 idesc_qk, kk > 0);
+          const uint32_t c = ((kk >> 2) * SM::kBoxBytes + (kk & 3) * 32) >> 4;
+          mma_ss(d, qd + c, kd + c, idesc_qk, kk > 0, leader);
         }
-        tc_commit(&bar->s_full[t]);
+        tc_commit(&bar->s_full[t], leader);
       };
-      auto in_range = [&](int t, int j) { return tr[t].active && j >= tr[t].lo && j <= tr[t].hi; };
+      auto issue_pv = [&](int t, int s, uint32_t acc) {
+        const uint64_t vd = s ? dv1 : dv0;
+        const uint32_t d = tmem + kOCol0 + t * D, p = tmem + t * kTileN;
+#pragma unroll
+        for (int kk = 0; kk < kTileN / 16; ++kk) mma_ts(d, p + kk * 8, vd + ((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc, leader);
+      };
+      auto in_range = [&](int t, int j) { return t ? (j >= lo1 && j <= hi1) : (j >= lo0 && j <= hi0); };
 
       // first key block: Q*K^T for both tiles
-      if (!mbar_wait(&bar->k_full[0], 0, abort_flag)) ok = false;
-      for (int t = 0; ok && t < kNumTiles; ++t) {
-        if (!in_range(t, jlo)) continue;
-        if (!mbar_wait(&bar->q_full[t], 0, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        issue_qk(t, jlo);
+      if (!mbar_wait_warp(&bar->k_full[0], 0, abort_flag)) ok = false;
+#pragma unroll
+      for (int t = 0; t < kNumTiles; ++t) {
+        if (ok && in_range(t, jlo)) {
+          if (!mbar_wait_warp(&bar->q_full[t], 0, abort_flag)) { ok = false; }
+          else { tc_fence_after(); issue_qk(t, 0); }
+        }
       }
-      if (ok) tc_commit(&bar->k_empty[0]);
+      if (ok) tc_commit(&bar->k_empty[0], leader);
 
       for (int j = jlo; ok && j <= jhi; ++j) {
-        const int it = j - jlo, s = it % kStages;
-        const uint32_t ph = (it / kStages) & 1;
-        const int sn = (it + 1) % kStages;
-        const uint32_t phn = ((it + 1) / kStages) & 1;
+        const int it = j - jlo, s = it & 1, sn = s ^ 1;
+        const uint32_t ph = (it >> 1) & 1;
+        const uint32_t phn = ((it + 1) >> 1) & 1;
         bool v_ready = false, k_ready = false;
-        for (int t = 0; ok && t < kNumTiles; ++t) {
-          if (in_range(t, j)) {
-            if (!mbar_wait(&bar->p_full[t], p_cnt[t] & 1, abort_flag)) { ok = false; break; }
-            ++p_cnt[t];
-            if (!v_ready) {
-              if (!mbar_wait(&bar->v_full[s], ph, abort_flag)) { ok = false; break; }
-              v_ready = true;
-            }
-            tc_fence_after();
-            const uint32_t va = smem_u32(sV + s * SM::kKVTileBytes);
 #pragma unroll
-            for (int kk = 0; kk < kTileN / 16; ++kk)
-              mma_ts(tmem + kOCol0 + t * D, tmem + t * kTileN + kk * 8,
-                     smem_desc_sw128(va + kk * 2048, SM::kBoxBytes, 1024), idesc_pv, (j > tr[t].lo) || (kk > 0));
+        for (int t = 0; t < kNumTiles; ++t) {
+          if (ok && in_range(t, j)) {
+            uint32_t& pc = t ? p_cnt1 : p_cnt0;
+            if (!mbar_wait_warp(&bar->p_full[t], pc & 1, abort_flag)) { ok = false; }
+            else {
+              ++pc;
+              if (!v_ready) {
+                if (!mbar_wait_warp(&bar->v_full[s], ph, abort_flag)) ok = false;
+                v_ready = true;
+              }
+              if (ok) {
+                tc_fence_after();
+                issue_pv(t, s, j > (t ? lo1 : lo0) ? 1u : 0u);
+              }
+            }
           }
-          if (j + 1 <= jhi && in_range(t, j + 1)) {
+          if (ok && j + 1 <= jhi && in_range(t, j + 1)) {
             if (!k_ready) {
-              if (!mbar_wait(&bar->k_full[sn], phn, abort_flag)) { ok = false; break; }
+              if (!mbar_wait_warp(&bar->k_full[sn], phn, abort_flag)) ok = false;
               k_ready = true;
             }
-            if (j + 1 == tr[t].lo && !mbar_wait(&bar->q_full[t], 0, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            issue_qk(t, j + 1);
+            if (ok && j + 1 == (t ? lo1 : lo0) && !mbar_wait_warp(&bar->q_full[t], 0, abort_flag)) ok = false;
+            if (ok) {
+              tc_fence_after();
+              issue_qk(t, sn);
+            }
           }
         }
         if (!ok) break;
         // V block j is released once both tiles' P*V have drained; K block j+1 once both Q*K^T have
-        if (!v_ready && !mbar_wait(&bar->v_full[s], ph, abort_flag)) break;
-        tc_commit(&bar->v_empty[s]);
+        if (!v_ready && !mbar_wait_warp(&bar->v_full[s], ph, abort_flag)) break;
+        tc_commit(&bar->v_empty[s], leader);
         if (j + 1 <= jhi) {
-          if (!k_ready && !mbar_wait(&bar->k_full[sn], phn, abort_flag)) break;
-          tc_commit(&bar->k_empty[sn]);
+          if (!k_ready && !mbar_wait_warp(&bar->k_full[sn], phn, abort_flag)) break;
+          tc_commit(&bar->k_empty[sn], leader);
         }
       }
-      if (ok) tc_commit(&bar->o_final);
+      if (ok) tc_commit(&bar->o_final, leader);
     }
     __syncwarp();
   } else {

@@ -57,14 +57,18 @@ PhaseEvents& phase_events() {
   return pe;
 }
 
-bool encode_rows_map(CUtensorMap* map, const void* base, int batch, int rows, int row_elems, int box_rows) {
+bool encode_rows_map(CUtensorMap* map, const void* base, int batch, int rows, int row_elems, int box_rows,
+                     int head_dim) {
   encode_tiled_fn enc = get_encode();
   if (!enc) return false;
-  cuuint64_t dims[3] = {(cuuint64_t)row_elems, (cuuint64_t)rows, (cuuint64_t)batch};
-  cuuint64_t strides[2] = {(cuuint64_t)row_elems * 2, (cuuint64_t)rows * row_elems * 2};
-  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+  // [batch, rows, row_elems] seen as {64 elements, rows, row_elems / 64 column chunks, batch}: one copy of a
+  // {64, box_rows, head_dim / 64, 1} box lands in shared memory as head_dim / 64 consecutive 128-byte-swizzled
+  // sub-tiles of box_rows x 64 elements -- the layout the MMA operand descriptors address.
+  cuuint64_t dims[4] = {64, (cuuint64_t)rows, (cuuint64_t)(row_elems / 64), (cuuint64_t)batch};
+  cuuint64_t strides[3] = {(cuuint64_t)row_elems * 2, 128, (cuuint64_t)rows * row_elems * 2};
+  cuuint32_t box[4] = {64, (cuuint32_t)box_rows, (cuuint32_t)(head_dim / 64), 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
@@ -160,10 +164,10 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
   if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, s) != cudaSuccess) return L2A_ERR_CUDA;
 
   CUtensorMap mapQ, mapK, mapV, mapQc;
-  if (!encode_rows_map(&mapQ, Q, p->B, p->Lq, p->Hq * p->D, kTileM) ||
-      !encode_rows_map(&mapK, K, p->B, p->Lk, p->Hkv * p->D, kTileN) ||
-      !encode_rows_map(&mapV, V, p->B, p->Lk, p->Hkv * p->D, kTileN) ||
-      !encode_rows_map(&mapQc, Qc, p->B, p->Lq, p->Hq * p->D, kTileM))
+  if (!encode_rows_map(&mapQ, Q, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||
+      !encode_rows_map(&mapK, K, p->B, p->Lk, p->Hkv * p->D, kTileN, p->D) ||
+      !encode_rows_map(&mapV, V, p->B, p->Lk, p->Hkv * p->D, kTileN, p->D) ||
+      !encode_rows_map(&mapQc, Qc, p->B, p->Lq, p->Hq * p->D, kTileM, p->D))
     return L2A_ERR_CUDA;
 
   FwdArgs a;

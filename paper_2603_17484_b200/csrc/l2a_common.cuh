@@ -20,9 +20,10 @@ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Host-side: resolved driver entry point for cuTensorMapEncodeTiled, and a helper that encodes a
-// [batch, rows, heads*D] bf16 tensor as a 3-D map with a {64 elements, box_rows, 1} box and the
-// 128-byte swizzle the MMA operand descriptors expect.  Returns false on failure.
-bool encode_rows_map(CUtensorMap* map, const void* base, int batch, int rows, int row_elems, int box_rows);
+// [batch, rows, heads*D] bf16 tensor so that ONE copy brings a box_rows x head_dim tile into shared memory in
+// the 128-byte-swizzled layout the MMA operand descriptors expect.  Returns false on failure.
+bool encode_rows_map(CUtensorMap* map, const void* base, int batch, int rows, int row_elems, int box_rows,
+                     int head_dim);
 
 // Launchers (each returns the CUDA error of its launch).  Defined in the kernel files.
 struct RouteArgs {
