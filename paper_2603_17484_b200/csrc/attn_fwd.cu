@@ -9,9 +9,12 @@
 //          the compact output O_c and log-sum-exp L_c.
 //
 // Structure (per CTA: two 128-row query tiles of one head, sharing the K/V stream):
-//   warps 0-3 / 4-7 : soft-max + correction + epilogue of tile 0 / 1 (one thread per query row)
-//   warp 8          : TMA producer (Q once; K and V blocks through 2-stage rings)
-//   warp 9          : tcgen05 MMA issuer and TMEM owner
+//   warps 0-15      : soft-max + correction + epilogue.  Warpgroup 2t+hf (4 warps) owns the 64 score columns of
+//                     half hf of tile t; the two threads that share a query row exchange their row maxima (and,
+//                     at the end, their row sums) through shared memory.  Sixteen warps hide each other's TMEM
+//                     and special-function latency.
+//   warp 16         : TMA producer (Q once; K and V blocks through 2-stage rings)
+//   warp 17         : tcgen05 MMA issuer and TMEM owner
 //   TMEM (512 cols) : S0 | S1 | O0 | O1 (fp32); the bf16 probabilities P overwrite the first half
 //                     of their own S columns and are consumed from TMEM as the A operand of P*V.
 // While one tile's soft-max runs on the CUDA cores, the tensor core works on the other tile.
@@ -26,7 +29,8 @@ namespace {
 
 constexpr int kNumTiles = 2;
 constexpr int kStages = 2;
-constexpr int kFwdThreads = 320;
+constexpr int kSoftmaxWarps = 16;
+constexpr int kFwdThreads = (kSoftmaxWarps + 2) * 32;   // 576
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
 template <int D>
@@ -38,7 +42,8 @@ struct FwdSmem {
   static constexpr int kKOff = kQOff + kNumTiles * kQTileBytes;
   static constexpr int kVOff = kKOff + kStages * kKVTileBytes;
   static constexpr int kBarOff = kVOff + kStages * kKVTileBytes;
-  static constexpr int kTotal = kBarOff + 256 + 1024 /* alignment slack */;
+  static constexpr int kXchOff = kBarOff + 256;                 // row-statistics exchange: [2][tile][half][128] fp32
+  static constexpr int kTotal = kXchOff + 2 * kNumTiles * 2 * kTileM * 4 + 1024 /* alignment slack */;
 };
 
 struct Barriers {
@@ -47,6 +52,7 @@ struct Barriers {
   uint64_t v_full[kStages], v_empty[kStages];
   uint64_t s_full[kNumTiles];
   uint64_t p_full[kNumTiles];
+  uint64_t xch[kNumTiles];     // the two halves of a tile meet here after publishing their row maxima
   uint64_t o_final;
   uint32_t tmem_base;
   int abort_flag;
@@ -63,7 +69,6 @@ __global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                 const __grid_constant__ CUtensorMap mapV, const FwdArgs a) {
   using SM = FwdSmem<D>;
-  constexpr int kDBoxes = D / 64;      // 64-element boxes per row
   constexpr int kKSteps = D / 16;      // MMA k-steps of Q*K^T
   constexpr int kOCol0 = 2 * kTileN;   // first TMEM column of the O accumulators
 
@@ -117,7 +122,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     for (int t = 0; t < kNumTiles; ++t) {
       mbar_init(&bar->q_full[t], 1);
       mbar_init(&bar->s_full[t], 1);
-      mbar_init(&bar->p_full[t], kTileM);
+      mbar_init(&bar->p_full[t], 2 * kTileM);
+      mbar_init(&bar->xch[t], 2 * kTileM);
     }
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&bar->k_full[s], 1);
@@ -129,7 +135,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     bar->abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 9) {
+  if (warp == 17) {
     tmem_alloc(&bar->tmem_base, 512);
     tmem_relinquish();
   }
@@ -138,7 +144,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem = bar->tmem_base;
 
-  if (warp == 8) {
+  if (warp == 16) {
     // =========================================================================== TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&mapQ);
@@ -161,7 +167,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       }
     }
     __syncwarp();
-  } else if (warp == 9) {
+  } else if (warp == 17) {
     // =========================================================================== MMA issuer
     // The whole warp runs this loop (uniform control flow keeps the descriptor arithmetic in uniform registers);
     // only the tcgen05 instructions themselves are predicated on lane 0.  Operand descriptors are built once per
@@ -196,7 +202,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         const uint64_t vd = s ? dv1 : dv0;
         const uint32_t d = tmem + kOCol0 + t * D, p = tmem + t * kTileN;
 #pragma unroll
-        for (int kk = 0; kk < kTileN / 16; ++kk) mma_ts(d, p + kk * 8, vd + ((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc, leader);
+        for (int kk = 0; kk < kTileN / 16; ++kk)
+          mma_ts(d, p + (kk >> 2) * 64 + (kk & 3) * 8, vd + ((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc, leader);
       };
       auto in_range = [&](int t, int j) { return t ? (j >= lo1 && j <= hi1) : (j >= lo0 && j <= hi0); };
 
@@ -259,49 +266,57 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     __syncwarp();
   } else {
     // =========================================================================== soft-max warpgroups
-    const int t = warp >> 2;                 // tile of this warpgroup
+    const int t = warp >> 3;                 // tile of this warpgroup
+    const int hf = (warp >> 2) & 1;          // which 64 score columns (and which half of the output columns)
     const int r = (warp & 3) * 32 + lane;    // row inside the tile == TMEM lane
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    const uint32_t s_addr = tmem + lane_base + t * kTileN;
-    const uint32_t o_addr = tmem + lane_base + kOCol0 + t * D;
-    if (tr[t].active) {
+    const uint32_t s_addr = tmem + lane_base + t * kTileN + hf * 64;        // this thread's 64 score columns
+    const uint32_t o_addr = tmem + lane_base + kOCol0 + t * D + hf * (D / 2);  // its D/2 accumulator columns
+    float* xch = reinterpret_cast<float*>(smem + SM::kXchOff);
+    const TileRange my = t ? tr[1] : tr[0];
+    if (my.active) {
       const int row = row0 + t * kTileM + r;           // sequence row (local) or compact row (global)
       const bool valid = row < n_rows;
       const int seq_row = valid ? (a.global_mode ? q_idx_b[row] : row) : -1;
       const int pos = valid ? seq_row + a.q_pos_offset : -1;
       const int pos_lo = valid ? (pos - w_eff) : 0x7fffffff;   // smallest visible key position
-      float m_use = -INFINITY;   // reference maximum, exp2 domain
-      float l = 0.f;
+      float m_use = -INFINITY;   // reference maximum, exp2 domain (identical in both threads of a row)
+      float l = 0.f;             // this thread's part of the row sum
       bool ok = true;
-      const int n_my = tr[t].hi - tr[t].lo + 1;
+      const int n_my = my.hi - my.lo + 1;
 
       for (int i = 0; i < n_my; ++i) {
-        const int j = tr[t].lo + i;
+        const int j = my.lo + i;
         // warp-uniform outcome: the TMEM loads/stores below are warp-collective
         if (!__all_sync(0xffffffffu, mbar_wait(&bar->s_full[t], i & 1, abort_flag))) { ok = false; break; }
         tc_fence_after();
-        float s[kTileN];
+        const int k0 = j * kTileN + hf * 64;
+        const bool partial = (k0 + 63 > my.min_pos) || (k0 < my.max_pos - w_eff);
+        // pass 1: row maximum of this half (32 columns at a time: the scores are re-read from TMEM in pass 2
+        // rather than kept in 64 registers)
+        float mx = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < kTileN / 32; ++c) {
+        for (int c = 0; c < 2; ++c) {
           uint32_t v[32];
           tmem_ld32(s_addr + c * 32, v);
+          tmem_ld_wait();
+          if (partial) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) s[c * 32 + e] = __uint_as_float(v[e]);
-        }
-        tmem_ld_wait();
-
-        const int k0 = j * kTileN;
-        const bool partial = (k0 + kTileN - 1 > tr[t].min_pos) || (k0 < tr[t].max_pos - w_eff);
-        if (partial) {
+            for (int e = 0; e < 32; ++e) {
+              const int kp = k0 + c * 32 + e;
+              if (kp <= pos && kp >= pos_lo) mx = fmaxf(mx, __uint_as_float(v[e]));
+            }
+          } else {
 #pragma unroll
-          for (int e = 0; e < kTileN; ++e) {
-            const int kp = k0 + e;
-            s[e] = (kp <= pos && kp >= pos_lo) ? s[e] : -INFINITY;
+            for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(v[e]));
           }
         }
-        float mx = s[0];
-#pragma unroll
-        for (int e = 1; e < kTileN; ++e) mx = fmaxf(mx, s[e]);
+        // row maximum over both halves: publish mine, meet the other half, read theirs
+        float* slot = xch + (((i & 1) * kNumTiles + t) * 2) * kTileM;
+        slot[hf * kTileM + r] = mx;
+        mbar_arrive(&bar->xch[t]);
+        if (!__all_sync(0xffffffffu, mbar_wait(&bar->xch[t], i & 1, abort_flag))) { ok = false; break; }
+        mx = fmaxf(mx, slot[(hf ^ 1) * kTileM + r]);
         const float m_new = fmaxf(m_use, mx * a.scale_log2);
 
         // correction: rescale the running sum and the TMEM accumulator only when the maximum moved a lot
@@ -311,7 +326,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
           const float alpha = need ? fast_exp2(m_use - m_new) : 1.0f;
           l *= alpha;
 #pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
+          for (int c = 0; c < D / 64; ++c) {
             uint32_t v[32];
             tmem_ld32(o_addr + c * 32, v);
             tmem_ld_wait();
@@ -323,18 +338,35 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         }
         const float m_eff = (m_use == -INFINITY) ? 0.f : m_use;
         const float neg_m = -m_eff;
+        // pass 2: probabilities, 32 columns at a time; P overwrites the first 32 of this half's 64 columns
         float sum = 0.f;
 #pragma unroll
-        for (int c = 0; c < kTileN / 64; ++c) {
-          uint32_t pk[32];
+        for (int c = 0; c < 2; ++c) {
+          uint32_t v[32];
+          tmem_ld32(s_addr + c * 32, v);
+          tmem_ld_wait();
+          uint32_t pk[16];
+          if (partial) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            const float p0 = fast_exp2(fmaf(s[c * 64 + 2 * e], a.scale_log2, neg_m));
-            const float p1 = fast_exp2(fmaf(s[c * 64 + 2 * e + 1], a.scale_log2, neg_m));
-            sum += p0 + p1;
-            pk[e] = pack_bf16(p0, p1);
+            for (int e = 0; e < 16; ++e) {
+              const int kp = k0 + c * 32 + 2 * e;
+              float p0 = fast_exp2(fmaf(__uint_as_float(v[2 * e]), a.scale_log2, neg_m));
+              float p1 = fast_exp2(fmaf(__uint_as_float(v[2 * e + 1]), a.scale_log2, neg_m));
+              p0 = (kp <= pos && kp >= pos_lo) ? p0 : 0.f;
+              p1 = (kp + 1 <= pos && kp + 1 >= pos_lo) ? p1 : 0.f;
+              sum += p0 + p1;
+              pk[e] = pack_bf16(p0, p1);
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              const float p0 = fast_exp2(fmaf(__uint_as_float(v[2 * e]), a.scale_log2, neg_m));
+              const float p1 = fast_exp2(fmaf(__uint_as_float(v[2 * e + 1]), a.scale_log2, neg_m));
+              sum += p0 + p1;
+              pk[e] = pack_bf16(p0, p1);
+            }
           }
-          tmem_st32(s_addr + c * 32, pk);
+          tmem_st16(s_addr + c * 16, pk);
         }
         l += sum;
         tmem_st_wait();
@@ -345,49 +377,56 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       // ---- epilogue: O / l, log-sum-exp, store (local) or scatter + combine (global)
       if (ok && __all_sync(0xffffffffu, mbar_wait(&bar->o_final, 0, abort_flag))) {
         tc_fence_after();
-        const float inv_l = (l > 0.f) ? 1.0f / l : 0.f;
-        if (valid && a.lse != nullptr) {
-          const float lse = (m_use + log2f(l)) * 0.6931471805599453f;
-          a.lse[((int64_t)b * a.Hq + h) * a.Lq + row] = lse;
-        }
-        const int64_t row_stride = (int64_t)a.Hq * D;
-        bf16* dst1 = nullptr;   // row-indexed destination (s rows, or compact a rows)
-        bf16* dst2 = nullptr;   // position-indexed destination
-        if (valid) {
-          if (a.out) dst1 = a.out + ((int64_t)b * a.Lq + row) * row_stride + (int64_t)h * D;
-          if (a.out2) dst2 = a.out2 + ((int64_t)b * a.Lq + seq_row) * row_stride + (int64_t)h * D;
-        }
-        const bool accumulate = a.global_mode && a.accumulate_into_out2;
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t v[32];
-          tmem_ld32(o_addr + c * 32, v);
-          tmem_ld_wait();
-          float f[32];
-#pragma unroll
-          for (int e = 0; e < 32; ++e) f[e] = __uint_as_float(v[e]) * inv_l;
-          if (dst1) {
-            uint4* d4 = reinterpret_cast<uint4*>(dst1 + c * 32);
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-              d4[q] = make_uint4(pack_bf16(f[8 * q], f[8 * q + 1]), pack_bf16(f[8 * q + 2], f[8 * q + 3]),
-                                 pack_bf16(f[8 * q + 4], f[8 * q + 5]), pack_bf16(f[8 * q + 6], f[8 * q + 7]));
+        // total row sum: exchange the two partial sums (the slot of parity n_my & 1 is free by now)
+        float* slot = xch + (((n_my & 1) * kNumTiles + t) * 2) * kTileM;
+        slot[hf * kTileM + r] = l;
+        mbar_arrive(&bar->xch[t]);
+        if (__all_sync(0xffffffffu, mbar_wait(&bar->xch[t], n_my & 1, abort_flag))) {
+          l += slot[(hf ^ 1) * kTileM + r];
+          const float inv_l = (l > 0.f) ? 1.0f / l : 0.f;
+          if (valid && hf == 0 && a.lse != nullptr) {
+            const float lse = (m_use + log2f(l)) * 0.6931471805599453f;
+            a.lse[((int64_t)b * a.Hq + h) * a.Lq + row] = lse;
           }
-          if (dst2) {
-            uint4* d4 = reinterpret_cast<uint4*>(dst2 + c * 32);
+          const int64_t row_stride = (int64_t)a.Hq * D;
+          bf16* dst1 = nullptr;   // row-indexed destination (s rows, or compact a rows)
+          bf16* dst2 = nullptr;   // position-indexed destination
+          if (valid) {
+            if (a.out) dst1 = a.out + ((int64_t)b * a.Lq + row) * row_stride + (int64_t)h * D + hf * (D / 2);
+            if (a.out2) dst2 = a.out2 + ((int64_t)b * a.Lq + seq_row) * row_stride + (int64_t)h * D + hf * (D / 2);
+          }
+          const bool accumulate = a.global_mode && a.accumulate_into_out2;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              if (accumulate) {
-                const uint4 old = d4[q];
-                const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
+          for (int c = 0; c < D / 64; ++c) {
+            uint32_t v[32];
+            tmem_ld32(o_addr + c * 32, v);
+            tmem_ld_wait();
+            float f[32];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                  f[8 * q + 2 * k] += __uint_as_float(ow[k] << 16);
-                  f[8 * q + 2 * k + 1] += __uint_as_float(ow[k] & 0xffff0000u);
+            for (int e = 0; e < 32; ++e) f[e] = __uint_as_float(v[e]) * inv_l;
+            if (dst1) {
+              uint4* d4 = reinterpret_cast<uint4*>(dst1 + c * 32);
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+                d4[q] = make_uint4(pack_bf16(f[8 * q], f[8 * q + 1]), pack_bf16(f[8 * q + 2], f[8 * q + 3]),
+                                   pack_bf16(f[8 * q + 4], f[8 * q + 5]), pack_bf16(f[8 * q + 6], f[8 * q + 7]));
+            }
+            if (dst2) {
+              uint4* d4 = reinterpret_cast<uint4*>(dst2 + c * 32);
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                if (accumulate) {
+                  const uint4 old = d4[q];
+                  const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
+#pragma unroll
+                  for (int k = 0; k < 4; ++k) {
+                    f[8 * q + 2 * k] += __uint_as_float(ow[k] << 16);
+                    f[8 * q + 2 * k + 1] += __uint_as_float(ow[k] & 0xffff0000u);
+                  }
                 }
+                d4[q] = make_uint4(pack_bf16(f[8 * q], f[8 * q + 1]), pack_bf16(f[8 * q + 2], f[8 * q + 3]),
+                                   pack_bf16(f[8 * q + 4], f[8 * q + 5]), pack_bf16(f[8 * q + 6], f[8 * q + 7]));
               }
-              d4[q] = make_uint4(pack_bf16(f[8 * q], f[8 * q + 1]), pack_bf16(f[8 * q + 2], f[8 * q + 3]),
-                                 pack_bf16(f[8 * q + 4], f[8 * q + 5]), pack_bf16(f[8 * q + 6], f[8 * q + 7]));
             }
           }
         }
@@ -405,7 +444,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     if (tid == 0) atomicExch(a.status, 1);
     __syncthreads();
   }
-  if (warp == 9) tmem_dealloc(tmem, 512);
+  if (warp == 17) tmem_dealloc(tmem, 512);
 }
 
 }  // namespace
