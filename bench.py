@@ -293,8 +293,16 @@ def main():
     tensor_phases = {k: v for k, v in phase_ms.items() if k in kernel_flops}
     dom = max(tensor_phases, key=tensor_phases.get)
     achieved = kernel_flops[dom] / phase_ms[dom] / 1e9
+    # DRAM traffic of the dominant kernel: ncu measured dram read+write = 1.13 x the algorithmic bytes of the dK/dV
+    # launch on the 32K case (profiles/attention_kernels_qwen25_7b_32k.md); every operand is read once, re-reads
+    # hit L2, so traffic scales with the tensor bytes of the launch
+    qb = cfg.B * cfg.L * cfg.Hq * cfg.D * 2
+    kb = cfg.B * cfg.L * cfg.Hkv * cfg.D * 2
+    dkv_alg_bytes = 2 * qb * (1 + float(d.mean())) + 4 * kb
+    traffic = 1.13 * dkv_alg_bytes if dom == "bwd_dkv" else None
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peaks["sustained"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["sustained"], "traffic": None,
+                "frac": achieved / peaks["sustained"], "traffic": traffic,
+                "traffic_note": "bytes per launch, scaled from an ncu capture of the 32K case by tensor bytes",
                 "peak_kind": f"sustained bf16 GEMM, {peaks['source']}", "launch_ms": phase_ms[dom],
                 "algorithmic_flops_per_launch": kernel_flops[dom]}
 
