@@ -309,8 +309,12 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
       tmem_ld_wait();
       if (!partial) {
 #pragma unroll
-        for (int e = 0; e < 32; ++e)
-          sv[e] = __float_as_uint(fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, -lse2)));
+        for (int e = 0; e < 32; e += 2) {
+          const float2 x = __ffma2_rn(make_float2(__uint_as_float(sv[e]), __uint_as_float(sv[e + 1])),
+                                      make_float2(a.scale_log2, a.scale_log2), make_float2(-lse2, -lse2));
+          sv[e] = __float_as_uint(fast_exp2(x.x));
+          sv[e + 1] = __float_as_uint(fast_exp2(x.y));
+        }
       } else {
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
@@ -327,9 +331,10 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
       uint32_t pk[16];
 #pragma unroll
       for (int e = 0; e < 16; ++e) {
-        const float ds0 = __uint_as_float(sv[2 * e]) * (__uint_as_float(dv[2 * e]) - delta);
-        const float ds1 = __uint_as_float(sv[2 * e + 1]) * (__uint_as_float(dv[2 * e + 1]) - delta);
-        pk[e] = pack_bf16(ds0, ds1);
+        const float2 t = __fadd2_rn(make_float2(__uint_as_float(dv[2 * e]), __uint_as_float(dv[2 * e + 1])),
+                                    make_float2(-delta, -delta));
+        const float2 ds = __fmul2_rn(make_float2(__uint_as_float(sv[2 * e]), __uint_as_float(sv[2 * e + 1])), t);
+        pk[e] = pack_bf16(ds.x, ds.y);
       }
       tmem_st16(tmem + lane_base + 384 + q * 32, pk);
       tmem_st_wait();
@@ -581,7 +586,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       for (int q = 0; q < 4; ++q) {
         const int col = q * 32 + lane;
         st_lse[col] = r_lse[q];
-        st_delta[col] = r_delta[q];
+        st_delta[col] = -r_delta[q];   // negated: dS = P * (dP + (-Delta)) with packed f32x2 arithmetic
         // quarter q needs the element mask unless every (key, query) pair of it is visible
         const bool lane_ok = r_pos[q] >= 0 && (k0 + kTileN - 1 <= r_pos[q]) && (k0 >= r_pos[q] - w_eff);
         const bool interior = __all_sync(0xffffffffu, lane_ok);
@@ -716,9 +721,9 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         if (!masked) {
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
-            const float p0 = fast_exp2(fmaf(__uint_as_float(sv[2 * e]), a.scale_log2, -st[2 * e]));
-            const float p1 = fast_exp2(fmaf(__uint_as_float(sv[2 * e + 1]), a.scale_log2, -st[2 * e + 1]));
-            pp[e] = pack_bf16(p0, p1);
+            const float2 x = __ffma2_rn(make_float2(__uint_as_float(sv[2 * e]), __uint_as_float(sv[2 * e + 1])),
+                                        make_float2(a.scale_log2, a.scale_log2), make_float2(-st[2 * e], -st[2 * e + 1]));
+            pp[e] = pack_bf16(fast_exp2(x.x), fast_exp2(x.y));
           }
         } else {
           const int glb = st_flags[4], row0 = st_flags[5];
@@ -765,10 +770,11 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         tmem_ld_wait();
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
-          // dS uses the bf16-rounded P, the same value the dV product sees
-          const float ds0 = bf16lo_to_f32(pp[e]) * (__uint_as_float(dv[2 * e]) - st[2 * e]);
-          const float ds1 = bf16hi_to_f32(pp[e]) * (__uint_as_float(dv[2 * e + 1]) - st[2 * e + 1]);
-          pd[e] = pack_bf16(ds0, ds1);
+          // dS uses the bf16-rounded P, the same value the dV product sees; st[] holds -Delta
+          const float2 t = __fadd2_rn(make_float2(__uint_as_float(dv[2 * e]), __uint_as_float(dv[2 * e + 1])),
+                                      make_float2(st[2 * e], st[2 * e + 1]));
+          const float2 ds = __fmul2_rn(make_float2(bf16lo_to_f32(pp[e]), bf16hi_to_f32(pp[e])), t);
+          pd[e] = pack_bf16(ds.x, ds.y);
         }
       }
       tmem_st16(dp_addr, pd);    // dS^T over the first half of this quarter's own dP^T columns

@@ -308,7 +308,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             }
           } else {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(v[e]));
+            for (int e = 0; e < 32; e += 2) mx = fmax3(mx, __uint_as_float(v[e]), __uint_as_float(v[e + 1]));
           }
         }
         // row maximum over both halves: publish mine, meet the other half, read theirs
@@ -358,13 +358,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
               pk[e] = pack_bf16(p0, p1);
             }
           } else {
+            float2 sum2 = make_float2(0.f, 0.f);
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
-              const float p0 = fast_exp2(fmaf(__uint_as_float(v[2 * e]), a.scale_log2, neg_m));
-              const float p1 = fast_exp2(fmaf(__uint_as_float(v[2 * e + 1]), a.scale_log2, neg_m));
-              sum += p0 + p1;
-              pk[e] = pack_bf16(p0, p1);
+              const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1])),
+                                          make_float2(a.scale_log2, a.scale_log2), make_float2(neg_m, neg_m));
+              const float2 p = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+              sum2 = __fadd2_rn(sum2, p);
+              pk[e] = pack_bf16(p.x, p.y);
             }
+            sum += sum2.x + sum2.y;
           }
           tmem_st16(s_addr + c * 16, pk);
         }

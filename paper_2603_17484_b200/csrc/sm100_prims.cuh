@@ -35,6 +35,13 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return r;
 }
 
+// three-input maximum (one instruction on sm_100)
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 // 16-byte load from shared memory by 32-bit shared address (all lanes may read the same address: broadcast)
 __device__ __forceinline__ float4 lds128(uint32_t saddr) {
   float4 v;
