@@ -195,6 +195,14 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bar->tmem_base;
+  if (tmem != 0) {
+    // all 512 columns were requested, so the allocation must start at column 0; the MMA warp relies on it to
+    // keep its TMEM operand addresses compile-time constants
+    __syncthreads();
+    if (warp == 17) tmem_dealloc(tmem, 512);
+    if (tid == 0) atomicExch(a.status, 3);
+    return;
+  }
 
   if (warp == 16) {
     // ------------------------------------------------------------------ TMA producer
@@ -220,6 +228,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     // (whole warp runs the loop; only the tcgen05 instructions are predicated on lane 0)
     {
       const uint32_t leader = (lane == 0);
+      constexpr uint32_t tmem = 0;   // checked above: TMEM operand addresses are immediates in this loop
       constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);
       constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 0, 1);
       const uint64_t dq = smem_desc_sw128(smem_u32(sQ), 16, 1024), ddo = smem_desc_sw128(smem_u32(sDO), 16, 1024);
@@ -523,6 +532,14 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bar->tmem_base;
+  if (tmem != 0) {
+    // all 512 columns were requested, so the allocation must start at column 0; the MMA warp relies on it to
+    // keep its TMEM operand addresses compile-time constants
+    __syncthreads();
+    if (warp == 17) tmem_dealloc(tmem, 512);
+    if (tid == 0) atomicExch(a.status, 3);
+    return;
+  }
 
   if (warp == 16) {
     // ------------------------------------------------------------------ TMA producer
@@ -602,6 +619,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     // (whole warp runs the loop; only the tcgen05 instructions are predicated on lane 0)
     {
       const uint32_t leader = (lane == 0);
+      constexpr uint32_t tmem = 0;   // checked above: TMEM operand addresses are immediates in this loop
       constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);
       constexpr uint32_t idesc_acc = idesc_bf16_f32(128, D, 0, 1);
       constexpr uint32_t kStageStep = SM::kTileBytes >> 4;

@@ -143,6 +143,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bar->tmem_base;
+  if (tmem != 0) {
+    // all 512 columns were requested, so the allocation must start at column 0; the MMA warp relies on it to
+    // keep its TMEM operand addresses compile-time constants
+    __syncthreads();
+    if (warp == 17) tmem_dealloc(tmem, 512);
+    if (tid == 0) atomicExch(a.status, 3);
+    return;
+  }
 
   if (warp == 16) {
     // =========================================================================== TMA producer
@@ -175,6 +183,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     // 128x128x16 MMA takes.
     {
       const uint32_t leader = (lane == 0);
+      constexpr uint32_t tmem = 0;   // checked above: TMEM operand addresses are immediates in this loop
       static_assert(kStages == 2 && kNumTiles == 2, "descriptor selects below assume two stages and two tiles");
       constexpr uint32_t idesc_qk = idesc_bf16_f32(kTileM, kTileN, 0, 0);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(kTileM, D, 0, 1);
