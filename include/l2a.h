@@ -49,6 +49,13 @@ typedef enum {
 #define L2A_FLAG_SKIP_LOCAL 2u    /* forward: no local module; O = d * A (the "SWA-0" ablation)   */
 #define L2A_FLAG_SKIP_GLOBAL 4u   /* forward: local module only; O = S (first phase of the layer, */
                                   /* before the router has seen S)                                */
+#define L2A_FLAG_FORCE_ALL_GLOBAL 8u /* training iterations that invoke Global Attention for every    */
+                                  /* token regardless of d_t (Section 3.3: done with a small       */
+                                  /* probability so that masked tokens' routers get a gradient).   */
+                                  /* O is unchanged (a_t is still multiplied by d_t), but A_c and   */
+                                  /* lse_glb are then indexed by ROW t and hold a_t for every t,    */
+                                  /* and l2a_backward's dgate covers every token.  Pass the flag to */
+                                  /* both calls.  Needs L2A_FLAG_SAVE_FOR_BWD.                      */
 
 /* router_kind of l2a_route_compact */
 #define L2A_ROUTER_MASK_U8 0     /* router = uint8 [B, Lq], non-zero => routed                    */
@@ -146,9 +153,10 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
  *               in : as written by l2a_forward with L2A_FLAG_SAVE_FOR_BWD.
  *   dQ          out: bf16 [B, Lq, Hq, D].
  *   dK, dV      out: bf16 [B, Lk, Hkv, D].
- *   dgate       out: optional fp32 [B, Lq] (may be NULL): sum over heads of dO_t . a_t for routed
- *                    rows, 0 elsewhere -- the loss-dependent term of the straight-through router
- *                    gradient (Eq. 7) for the rows whose global output was computed.
+ *   dgate       out: optional fp32 [B, Lq] (may be NULL): sum over heads of dO_t . a_t -- the
+ *                    loss-dependent term of the straight-through router gradient (Eq. 7) -- for
+ *                    the rows whose global output was computed: routed rows (0 elsewhere), or
+ *                    every row with L2A_FLAG_FORCE_ALL_GLOBAL.
  *   bwd_ws         : workspace of at least bwd_ws_bytes.
  */
 l2a_status l2a_backward(const l2a_params* p, const void* Q, const void* K, const void* V,

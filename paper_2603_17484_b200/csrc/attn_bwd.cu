@@ -46,14 +46,15 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const bf16* __restrict__
                                                         const uint8_t* __restrict__ d_mask,
                                                         const int32_t* __restrict__ prefix, float* __restrict__ delta_loc,
                                                         float* __restrict__ delta_glb, float* __restrict__ dgate, int B,
-                                                        int L, int Hq, int D) {
+                                                        int L, int Hq, int D, int a_by_row) {
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (warp >= B * L) return;
   const int b = warp / L, t = warp % L;
   const bool routed = d_mask[(int64_t)b * L + t] != 0;
   const int c = routed ? prefix[(int64_t)b * (L + 1) + t] : 0;
   const int64_t row = ((int64_t)b * L + t) * Hq * D;
-  const int64_t crow = ((int64_t)b * L + c) * Hq * D;
+  // a_by_row: the global output was computed for every token and A is indexed by row (forced-global iterations)
+  const int64_t crow = ((int64_t)b * L + (a_by_row ? t : c)) * Hq * D;
   const int per_lane = D / 32;  // 2 or 4 elements
   float gate = 0.f;
   for (int h = 0; h < Hq; ++h) {
@@ -65,7 +66,7 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const bf16* __restrict__
       const float2 o2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(po + e));
       const float2 s2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(ps + e));
       dl += o2.x * s2.x + o2.y * s2.y;
-      if (routed) {
+      if (routed || a_by_row) {
         const float2 a2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(pa + e));
         dg += o2.x * a2.x + o2.y * a2.y;
       }
@@ -81,7 +82,19 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const bf16* __restrict__
     }
     gate += dg;
   }
-  if (dgate != nullptr && lane == 0) dgate[(int64_t)b * L + t] = routed ? gate : 0.f;
+  if (dgate != nullptr && lane == 0) dgate[(int64_t)b * L + t] = (routed || a_by_row) ? gate : 0.f;
+}
+
+// lse by row -> lse by compact row (forced-global iterations store the global log-sum-exp for every row)
+__global__ void __launch_bounds__(256) compact_stat_kernel(const float* __restrict__ by_row, float* __restrict__ by_c,
+                                                           const int32_t* __restrict__ q_idx,
+                                                           const int32_t* __restrict__ n_routed, int L, int Hq) {
+  const int b = blockIdx.z, h = blockIdx.y;
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c < n_routed[b]) {
+    const int64_t base = ((int64_t)b * Hq + h) * L;
+    by_c[base + c] = by_row[base + q_idx[(int64_t)b * L + c]];
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -870,7 +883,7 @@ cudaError_t launch_bwd_kernels(const BwdArgs& base, const CUtensorMap& mapQ, con
 
 }  // namespace
 
-size_t bwd_ws_size(const l2a_params* p) { return kWsHeaderBytes + 2 * rows_bytes(p) + 2 * stat_bytes(p); }
+size_t bwd_ws_size(const l2a_params* p) { return kWsHeaderBytes + 2 * rows_bytes(p) + 3 * stat_bytes(p); }
 
 }  // namespace l2a
 
@@ -892,6 +905,7 @@ extern "C" l2a_status l2a_backward(const l2a_params* p, const void* Q, const voi
   l2a_status st = l2a_workspace_bytes(p, nullptr, nullptr, &need);
   if (st != L2A_OK) return st;
   if (p->flags & (L2A_FLAG_SKIP_LOCAL | L2A_FLAG_SKIP_GLOBAL)) return L2A_ERR_UNSUPPORTED;
+  const bool force_all = p->flags & L2A_FLAG_FORCE_ALL_GLOBAL;
   if (!Q || !K || !V || !d_mask || !q_idx || !n_routed || !prefix || !dO || !S_save || !A_c || !lse_loc || !lse_glb ||
       !dQ || !dK || !dV)
     return L2A_ERR_INVALID_ARG;
@@ -906,6 +920,7 @@ extern "C" l2a_status l2a_backward(const l2a_params* p, const void* Q, const voi
   bf16* dOc = reinterpret_cast<bf16*>(ws + kWsHeaderBytes + rows_bytes(p));
   float* delta_loc = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p));
   float* delta_glb = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + stat_bytes(p));
+  float* lse_c = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + 2 * stat_bytes(p));
 
   CUtensorMap mapQ, mapDO, mapQc, mapDOc, mapK, mapV;
   if (!encode_rows_map(&mapQ, Q, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||
@@ -930,8 +945,13 @@ extern "C" l2a_status l2a_backward(const l2a_params* p, const void* Q, const voi
     const unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
     bwd_delta_kernel<<<blocks, 256, 0, s>>>(static_cast<const bf16*>(dO), static_cast<const bf16*>(S_save),
                                             static_cast<const bf16*>(A_c), d_mask, prefix, delta_loc, delta_glb, dgate,
-                                            p->B, p->Lq, p->Hq, p->D);
+                                            p->B, p->Lq, p->Hq, p->D, force_all ? 1 : 0);
     if (cudaGetLastError() != cudaSuccess) return L2A_ERR_CUDA;
+    if (force_all) {
+      dim3 grid((p->Lq + 255) / 256, p->Hq, p->B);
+      compact_stat_kernel<<<grid, 256, 0, s>>>(lse_glb, lse_c, q_idx, n_routed, p->Lq, p->Hq);
+      if (cudaGetLastError() != cudaSuccess) return L2A_ERR_CUDA;
+    }
   }
   pe.mark(s);
   BwdArgs a;
@@ -942,7 +962,7 @@ extern "C" l2a_status l2a_backward(const l2a_params* p, const void* Q, const voi
   a.scale_log2 = a.scale * kLog2e;
   a.global_mode = 0;
   a.q_idx = q_idx; a.n_routed = n_routed; a.prefix = prefix;
-  a.lse_loc = lse_loc; a.lse_glb = lse_glb; a.delta_loc = delta_loc; a.delta_glb = delta_glb;
+  a.lse_loc = lse_loc; a.lse_glb = force_all ? lse_c : lse_glb; a.delta_loc = delta_loc; a.delta_glb = delta_glb;
   a.dQ = static_cast<bf16*>(dQ); a.dK = static_cast<bf16*>(dK); a.dV = static_cast<bf16*>(dV);
   a.status = reinterpret_cast<int*>(ws);
   cudaError_t e = p->D == 128 ? launch_bwd_kernels<128>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, s)

@@ -79,7 +79,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   const int b = rest % a.B;
   const int pi = n_pairs - 1 - rest / a.B;
   const int g = h / (a.Hq / a.Hkv);
-  const int n_rows = a.global_mode ? a.n_routed[b] : a.Lq;  // valid (compact) rows of this batch entry
+  const bool compact = a.global_mode && !a.all_rows;           // rows are compact indices into q_idx
+  const int n_rows = compact ? a.n_routed[b] : a.Lq;           // valid (compact) rows of this batch entry
   const int row0 = pi * kRowsPerCta;
   if (row0 >= n_rows) return;
 
@@ -95,8 +96,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     if (last > n_rows - 1) last = n_rows - 1;
     tr[t].active = first < n_rows;
     if (tr[t].active) {
-      tr[t].min_pos = (a.global_mode ? q_idx_b[first] : first) + a.q_pos_offset;
-      tr[t].max_pos = (a.global_mode ? q_idx_b[last] : last) + a.q_pos_offset;
+      tr[t].min_pos = (compact ? q_idx_b[first] : first) + a.q_pos_offset;
+      tr[t].max_pos = (compact ? q_idx_b[last] : last) + a.q_pos_offset;
       const int lo_pos = tr[t].min_pos - w_eff;
       tr[t].lo = lo_pos > 0 ? lo_pos / kTileN : 0;
       tr[t].hi = tr[t].max_pos / kTileN;
@@ -286,7 +287,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     if (my.active) {
       const int row = row0 + t * kTileM + r;           // sequence row (local) or compact row (global)
       const bool valid = row < n_rows;
-      const int seq_row = valid ? (a.global_mode ? q_idx_b[row] : row) : -1;
+      const int seq_row = valid ? (compact ? q_idx_b[row] : row) : -1;
       const int pos = valid ? seq_row + a.q_pos_offset : -1;
       const int pos_lo = valid ? (pos - w_eff) : 0x7fffffff;   // smallest visible key position
       float m_use = -INFINITY;   // reference maximum, exp2 domain (identical in both threads of a row)
@@ -405,7 +406,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
           bf16* dst2 = nullptr;   // position-indexed destination
           if (valid) {
             if (a.out) dst1 = a.out + ((int64_t)b * a.Lq + row) * row_stride + (int64_t)h * D + hf * (D / 2);
-            if (a.out2) dst2 = a.out2 + ((int64_t)b * a.Lq + seq_row) * row_stride + (int64_t)h * D + hf * (D / 2);
+            if (a.out2 && (a.combine_mask == nullptr || a.combine_mask[(int64_t)b * a.Lq + seq_row]))
+              dst2 = a.out2 + ((int64_t)b * a.Lq + seq_row) * row_stride + (int64_t)h * D + hf * (D / 2);
           }
           const bool accumulate = a.global_mode && a.accumulate_into_out2;
 #pragma unroll

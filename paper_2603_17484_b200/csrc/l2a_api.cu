@@ -148,7 +148,9 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
   const bool save = p->flags & L2A_FLAG_SAVE_FOR_BWD;
   const bool skip_local = p->flags & L2A_FLAG_SKIP_LOCAL;
   const bool skip_global = p->flags & L2A_FLAG_SKIP_GLOBAL;
+  const bool force_all = p->flags & L2A_FLAG_FORCE_ALL_GLOBAL;
   if (skip_local && skip_global) return L2A_ERR_INVALID_ARG;
+  if (force_all && (!save || skip_local || skip_global)) return L2A_ERR_INVALID_ARG;
   if (!Q || !K || !V || !O) return L2A_ERR_INVALID_ARG;
   if (!skip_global && (!d_mask || !q_idx || !n_routed || !prefix)) return L2A_ERR_INVALID_ARG;
   if (save && (!S_save || !A_c || !lse_loc || !lse_glb)) return L2A_ERR_INVALID_ARG;
@@ -178,11 +180,13 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
   a.q_idx = q_idx;
   a.n_routed = n_routed;
   a.status = status;
+  a.all_rows = 0;
+  a.combine_mask = nullptr;
 
   PhaseEvents& pe = phase_events();
   struct ClearOnExit { PhaseEvents& p; ~ClearOnExit() { p.clear(); } } clear_on_exit{pe};
   pe.mark(s);
-  if (!skip_global) {
+  if (!skip_global && !force_all) {
     // consolidate routed query rows (Algorithm 1, step 1); independent of the local pass
     if (launch_gather_rows(static_cast<const bf16*>(Q), Qc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s) !=
         cudaSuccess)
@@ -207,7 +211,13 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
     a.out = static_cast<bf16*>(A_c);
     a.out2 = static_cast<bf16*>(O);
     a.lse = lse_glb;
-    if (launch_attn_fwd(a, mapQc, mapK, mapV, s) != cudaSuccess) return L2A_ERR_CUDA;
+    if (force_all) {
+      // Global Attention for every token (Section 3.3): same kernel over all rows in place; a_t is stored for
+      // every row, and still only enters O where d_t = 1
+      a.all_rows = 1;
+      a.combine_mask = d_mask;
+    }
+    if (launch_attn_fwd(a, force_all ? mapQ : mapQc, mapK, mapV, s) != cudaSuccess) return L2A_ERR_CUDA;
   }
   pe.mark(s);
   return L2A_OK;

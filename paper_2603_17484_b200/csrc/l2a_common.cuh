@@ -52,6 +52,8 @@ struct FwdArgs {
   float scale_log2;         // softmax_scale * log2(e)
   int global_mode;          // 0: local banded attention over all rows; 1: global attention over compact rows
   int accumulate_into_out2; // global mode: out2[row] = out2[row] + a (1) or out2[row] = a (0)
+  int all_rows;             // global mode over EVERY row (identity index list) instead of the compacted ones
+  const uint8_t* combine_mask;  // when set, out2 is touched only for rows with a non-zero mask entry
   const int32_t* q_idx;
   const int32_t* n_routed;
   bf16* out;    // local: s rows [B,Lq,Hq,D];  global: compact a rows (A_c) or NULL

@@ -19,6 +19,7 @@ L2A_OK = 0
 FLAG_SAVE_FOR_BWD = 1
 FLAG_SKIP_LOCAL = 2
 FLAG_SKIP_GLOBAL = 4
+FLAG_FORCE_ALL_GLOBAL = 8
 ROUTER_MASK_U8 = 0
 ROUTER_LOGITS_F32 = 1
 
