@@ -169,7 +169,9 @@ l2a_status l2a_backward(const l2a_params* p, const void* Q, const void* K, const
  * One whole step for callers that hold HOST buffers, so that end-to-end time including the
  * transfers can be measured through the C ABI: copies Q, K, V, the router input (and dO) to the
  * device buffers the caller supplies, runs l2a_route_compact + l2a_forward (+ l2a_backward when
- * host->dO is non-NULL), copies O (and dQ, dK, dV) back, and synchronises the stream.
+ * host->dO is non-NULL), copies O (and dQ, dK, dV) back, and synchronises the stream.  The transfers overlap
+ * the kernels on two helper streams the library creates once per host thread (dO goes up during the
+ * forward, O / dK / dV come down during the backward); this is the one call that keeps such state.
  * `host` holds HOST pointers (pinned memory makes the copies asynchronous); `dev` holds DEVICE
  * pointers with the sizes the corresponding arguments of the three calls need.  With a backward,
  * p->flags must contain L2A_FLAG_SAVE_FOR_BWD and every field of `dev` must be set; without one,

@@ -249,11 +249,38 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
   const size_t qb = (size_t)p->B * p->Lq * p->Hq * p->D * sizeof(bf16);
   const size_t kb = (size_t)p->B * p->Lk * p->Hkv * p->D * sizeof(bf16);
   const size_t rb = (size_t)p->B * p->Lq * (router_kind == L2A_ROUTER_MASK_U8 ? 1 : 4);
-  if (cudaMemcpyAsync(dev->router, host->router, rb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
-  if (cudaMemcpyAsync(dev->Q, host->Q, qb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
-  if (cudaMemcpyAsync(dev->K, host->K, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
-  if (cudaMemcpyAsync(dev->V, host->V, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
-  if (bwd && cudaMemcpyAsync(dev->dO, host->dO, qb, cudaMemcpyHostToDevice, s) != cudaSuccess) return L2A_ERR_CUDA;
+  // Two helper streams (created once per host thread and device) overlap the transfers with the kernels:
+  // dO is uploaded while the forward runs, O is downloaded while the backward runs, dK / dV while the dQ
+  // kernels run.  With pageable host memory the copies simply serialise.
+  struct Aux {
+    int device = -1;
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, up = nullptr, fwd = nullptr, phase[6] = {}, down = nullptr;
+  };
+  static thread_local Aux aux;
+  int dev_id = 0;
+  if (cudaGetDevice(&dev_id) != cudaSuccess) return L2A_ERR_CUDA;
+  if (aux.device != dev_id) {
+    if (cudaStreamCreateWithFlags(&aux.in, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&aux.out, cudaStreamNonBlocking) != cudaSuccess)
+      return L2A_ERR_CUDA;
+    cudaEvent_t* evs[] = {&aux.start, &aux.up, &aux.fwd, &aux.down, &aux.phase[0], &aux.phase[1], &aux.phase[2],
+                          &aux.phase[3], &aux.phase[4], &aux.phase[5]};
+    for (cudaEvent_t* e : evs)
+      if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return L2A_ERR_CUDA;
+    aux.device = dev_id;
+  }
+#define L2A_TRY(x) do { if ((x) != cudaSuccess) return L2A_ERR_CUDA; } while (0)
+  L2A_TRY(cudaEventRecord(aux.start, s));
+  L2A_TRY(cudaMemcpyAsync(dev->router, host->router, rb, cudaMemcpyHostToDevice, s));
+  L2A_TRY(cudaMemcpyAsync(dev->Q, host->Q, qb, cudaMemcpyHostToDevice, s));
+  L2A_TRY(cudaMemcpyAsync(dev->K, host->K, kb, cudaMemcpyHostToDevice, s));
+  L2A_TRY(cudaMemcpyAsync(dev->V, host->V, kb, cudaMemcpyHostToDevice, s));
+  if (bwd) {   // dO rides the second stream, behind whatever the caller had queued before this call
+    L2A_TRY(cudaStreamWaitEvent(aux.in, aux.start, 0));
+    L2A_TRY(cudaMemcpyAsync(dev->dO, host->dO, qb, cudaMemcpyHostToDevice, aux.in));
+    L2A_TRY(cudaEventRecord(aux.up, aux.in));
+  }
   st = l2a_route_compact(p, dev->router, router_kind, logit_threshold, dev->d_mask, dev->q_idx, dev->n_routed,
                          dev->prefix, dev->route_ws, dev->route_ws_bytes, stream);
   if (st != L2A_OK) return st;
@@ -263,17 +290,29 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
                    bwd ? dev->S_save : nullptr, bwd ? dev->A_c : nullptr, bwd ? dev->lse_loc : nullptr,
                    bwd ? dev->lse_glb : nullptr, dev->fwd_ws, dev->fwd_ws_bytes, stream);
   if (st != L2A_OK) return st;
-  if (cudaMemcpyAsync(host->O, dev->O, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return L2A_ERR_CUDA;
+  L2A_TRY(cudaEventRecord(aux.fwd, s));
+  L2A_TRY(cudaStreamWaitEvent(aux.out, aux.fwd, 0));
+  L2A_TRY(cudaMemcpyAsync(host->O, dev->O, qb, cudaMemcpyDeviceToHost, aux.out));
   if (bwd) {
+    L2A_TRY(cudaStreamWaitEvent(s, aux.up, 0));
+    // phase boundary 3 of the backward = the dK/dV kernel has finished: its results can leave while dQ is computed
+    void* phase_events[6];
+    for (int i = 0; i < 6; ++i) phase_events[i] = aux.phase[i];
+    st = l2a_profile_next_call(phase_events, 6);
+    if (st != L2A_OK) return st;
     st = l2a_backward(&q, dev->Q, dev->K, dev->V, dev->d_mask, dev->q_idx, dev->n_routed, dev->prefix, dev->dO,
                       dev->S_save, dev->A_c, dev->lse_loc, dev->lse_glb, dev->dQ, dev->dK, dev->dV, nullptr,
                       dev->bwd_ws, dev->bwd_ws_bytes, stream);
     if (st != L2A_OK) return st;
-    if (cudaMemcpyAsync(host->dQ, dev->dQ, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return L2A_ERR_CUDA;
-    if (cudaMemcpyAsync(host->dK, dev->dK, kb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return L2A_ERR_CUDA;
-    if (cudaMemcpyAsync(host->dV, dev->dV, kb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return L2A_ERR_CUDA;
+    L2A_TRY(cudaStreamWaitEvent(aux.out, aux.phase[3], 0));
+    L2A_TRY(cudaMemcpyAsync(host->dK, dev->dK, kb, cudaMemcpyDeviceToHost, aux.out));
+    L2A_TRY(cudaMemcpyAsync(host->dV, dev->dV, kb, cudaMemcpyDeviceToHost, aux.out));
+    L2A_TRY(cudaMemcpyAsync(host->dQ, dev->dQ, qb, cudaMemcpyDeviceToHost, s));
   }
-  if (cudaStreamSynchronize(s) != cudaSuccess) return L2A_ERR_CUDA;
+  L2A_TRY(cudaEventRecord(aux.down, aux.out));
+  L2A_TRY(cudaStreamWaitEvent(s, aux.down, 0));   // the caller's stream ends the step with every result delivered
+  L2A_TRY(cudaStreamSynchronize(s));
+#undef L2A_TRY
   return L2A_OK;
 }
 
