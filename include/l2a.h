@@ -49,6 +49,11 @@ typedef enum {
 #define L2A_FLAG_SKIP_LOCAL 2u    /* forward: no local module; O = d * A (the "SWA-0" ablation)   */
 #define L2A_FLAG_SKIP_GLOBAL 4u   /* forward: local module only; O = S (first phase of the layer, */
                                   /* before the router has seen S)                                */
+#define L2A_FLAG_GLOBAL_PHASE 16u  /* forward: second phase of the layer.  O (and S_save) already hold   */
+                                  /* the local output from an earlier L2A_FLAG_SKIP_GLOBAL call; only  */
+                                  /* the routed rows' global attention runs and is added into O.       */
+                                  /* Lets the caller compute the router decision from S in between     */
+                                  /* (Eq. 2 -> 3 -> 4 -> 5 in the order the layer defines them).       */
 #define L2A_FLAG_FORCE_ALL_GLOBAL 8u /* training iterations that invoke Global Attention for every    */
                                   /* token regardless of d_t (Section 3.3: done with a small       */
                                   /* probability so that masked tokens' routers get a gradient).   */
@@ -112,6 +117,23 @@ l2a_status l2a_workspace_status(const void* ws, void* stream);
 l2a_status l2a_route_compact(const l2a_params* p, const void* router, int router_kind, float logit_threshold,
                              uint8_t* d_mask, int32_t* q_idx, int32_t* n_routed, int32_t* prefix,
                              void* route_ws, size_t route_ws_bytes, void* stream);
+
+/*
+ * Router logits from the local output (Eq. 3: d_hat_t = sigmoid(W s_t), one scalar per token), with the
+ * sparsity regulariser's sum (Eq. 6) as a by-product.
+ *
+ *   S           in : bf16 [B, Lq, Hq, D], the local output s_t (as written by l2a_forward); the router sees
+ *                    the Hq * D values of a token as one vector.
+ *   w           in : fp32 [Hq * D] router weights; bias: scalar added to every logit.
+ *   logits      out: fp32 [B, Lq], z_t = w . s_t + bias (fp32 accumulation), ready for
+ *                    l2a_route_compact(..., L2A_ROUTER_LOGITS_F32, threshold 0).
+ *   sum_sq      out: optional fp32 [B] (may be NULL): sum_t sigmoid(z_t)^2, the un-normalised regulariser
+ *                    of Eq. 6 (the caller multiplies by lambda / (n L)).  Accumulated with atomics: the
+ *                    last bits depend on the order of addition.
+ * HBM-bound: one pass over S.
+ */
+l2a_status l2a_router_logits(const l2a_params* p, const void* S, const float* w, float bias, float* logits,
+                             float* sum_sq, void* stream);
 
 /*
  * Forward of the layer (Eq. 2, 4, 5; Algorithm 1 for the global part).

@@ -20,4 +20,6 @@ from .binding import (  # noqa: F401
     dgate_rows,
     num_threads,
     f64_inputs,
+    router_logits,
+    gate_regulariser_sum,
 )

@@ -186,3 +186,18 @@ def dgate_rows(sh: Shape, Q, K, V, dO, rb, rt):
     _load().l2a_oracle_dgate_rows(ctypes.byref(cs), _p(Q), _p(K), _p(V), _p(dO), ctypes.c_int64(rb.size),
                                   _p(rb), _p(rt), _p(out))
     return out
+
+
+def router_logits(S, w, bias: float = 0.0):
+    """Eq. 3 before the sigmoid: z_t = W s_t + bias with s_t the Hq*D local-output values of token t.
+    S: bf16 bit patterns (uint16) [B, L, Hq, D]; w: [Hq*D].  Plain fp64 dot products."""
+    S = np.ascontiguousarray(S)
+    s64 = (S.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    B, L = S.shape[0], S.shape[1]
+    return s64.reshape(B, L, -1) @ np.asarray(w, np.float64) + float(bias)
+
+
+def gate_regulariser_sum(z):
+    """Sum over tokens of sigmoid(z_t)^2 per batch entry (Eq. 6 without its lambda / (n L) factor)."""
+    g = 1.0 / (1.0 + np.exp(-np.asarray(z, np.float64)))
+    return (g * g).sum(axis=1)

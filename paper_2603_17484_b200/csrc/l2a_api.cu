@@ -149,12 +149,14 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
   const bool skip_local = p->flags & L2A_FLAG_SKIP_LOCAL;
   const bool skip_global = p->flags & L2A_FLAG_SKIP_GLOBAL;
   const bool force_all = p->flags & L2A_FLAG_FORCE_ALL_GLOBAL;
+  const bool global_phase = p->flags & L2A_FLAG_GLOBAL_PHASE;   // O already holds S: add the global part only
   if (skip_local && skip_global) return L2A_ERR_INVALID_ARG;
+  if (global_phase && (skip_local || skip_global)) return L2A_ERR_INVALID_ARG;
   if (force_all && (!save || skip_local || skip_global)) return L2A_ERR_INVALID_ARG;
   if (!Q || !K || !V || !O) return L2A_ERR_INVALID_ARG;
   if (!skip_global && (!d_mask || !q_idx || !n_routed || !prefix)) return L2A_ERR_INVALID_ARG;
   if (save && (!S_save || !A_c || !lse_loc || !lse_glb)) return L2A_ERR_INVALID_ARG;
-  if (save && (skip_local || skip_global)) return L2A_ERR_INVALID_ARG;
+  if (save && skip_local) return L2A_ERR_INVALID_ARG;
   if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || !aligned(S_save, 16) ||
       !aligned(A_c, 16) || !aligned(lse_loc, 4) || !aligned(lse_glb, 4))
     return L2A_ERR_INVALID_ARG;
@@ -193,14 +195,14 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
       return L2A_ERR_CUDA;
   }
   pe.mark(s);
-  if (!skip_local) {
+  if (!skip_local && !global_phase) {
     a.global_mode = 0;
     a.accumulate_into_out2 = 0;
     a.out = static_cast<bf16*>(save ? S_save : O);
     a.out2 = save ? static_cast<bf16*>(O) : nullptr;
     a.lse = lse_loc;
     if (launch_attn_fwd(a, mapQ, mapK, mapV, s) != cudaSuccess) return L2A_ERR_CUDA;
-  } else {
+  } else if (skip_local) {
     const size_t bytes = (size_t)p->B * p->Lq * p->Hq * p->D * sizeof(bf16);
     if (cudaMemsetAsync(O, 0, bytes, s) != cudaSuccess) return L2A_ERR_CUDA;  // Algorithm 1: O starts at zero
   }
@@ -221,6 +223,20 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
   }
   pe.mark(s);
   return L2A_OK;
+}
+
+l2a_status l2a_router_logits(const l2a_params* p, const void* S, const float* w, float bias, float* logits,
+                             float* sum_sq, void* stream) {
+  l2a_status st = check_params(p);
+  if (st != L2A_OK) return st;
+  if (!S || !w || !logits) return L2A_ERR_INVALID_ARG;
+  if (!aligned(S, 16) || !aligned(w, 16) || !aligned(logits, 4)) return L2A_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (sum_sq && cudaMemsetAsync(sum_sq, 0, sizeof(float) * p->B, s) != cudaSuccess) return L2A_ERR_CUDA;
+  return launch_router_logits(static_cast<const bf16*>(S), w, bias, logits, sum_sq, p->B, p->Lq, p->Hq * p->D, s) ==
+                 cudaSuccess
+             ? L2A_OK
+             : L2A_ERR_CUDA;
 }
 
 l2a_status l2a_profile_next_call(void* const* events, int n_events) {

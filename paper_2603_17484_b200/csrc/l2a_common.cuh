@@ -46,6 +46,10 @@ cudaError_t launch_route_compact(const RouteArgs& a, cudaStream_t stream);
 cudaError_t launch_gather_rows(const bf16* src, bf16* dst, const int32_t* q_idx, const int32_t* n_routed,
                                int B, int L, int row_elems, cudaStream_t stream);
 
+// z[b,t] = w . S[b,t,:] + bias (fp32 accumulation); optional sum over t of sigmoid(z)^2 per batch entry
+cudaError_t launch_router_logits(const bf16* S, const float* w, float bias, float* logits, float* sum_sq, int B,
+                                 int L, int row_elems, cudaStream_t stream);
+
 struct FwdArgs {
   int B, Lq, Lk, Hq, Hkv, D;
   int window, q_pos_offset;

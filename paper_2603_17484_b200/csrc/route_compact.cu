@@ -137,7 +137,47 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const bf16* __restrict
   }
 }
 
+// Router logit (Eq. 3): one warp per token, 16-byte loads of the token's Hq*D values, fp32 accumulation.
+__global__ void __launch_bounds__(256) router_logits_kernel(const bf16* __restrict__ S, const float* __restrict__ w,
+                                                            float bias, float* __restrict__ logits,
+                                                            float* __restrict__ sum_sq, int B, int L, int row_elems) {
+  const int64_t token = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (token >= (int64_t)B * L) return;
+  const uint4* row = reinterpret_cast<const uint4*>(S + token * row_elems);
+  const float4* w4 = reinterpret_cast<const float4*>(w);
+  float acc = 0.f;
+  for (int i = lane; i < row_elems / 8; i += 32) {
+    const uint4 v = __ldg(&row[i]);
+    const float4 wa = __ldg(&w4[2 * i]), wb = __ldg(&w4[2 * i + 1]);
+    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+    const float ww[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      acc = fmaf(__uint_as_float(u[k] << 16), ww[2 * k], acc);
+      acc = fmaf(__uint_as_float(u[k] & 0xffff0000u), ww[2 * k + 1], acc);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) {
+    const float z = acc + bias;
+    logits[token] = z;
+    if (sum_sq != nullptr) {
+      const float g = 1.0f / (1.0f + __expf(-z));
+      atomicAdd(&sum_sq[token / L], g * g);
+    }
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_router_logits(const bf16* S, const float* w, float bias, float* logits, float* sum_sq, int B, int L,
+                                 int row_elems, cudaStream_t stream) {
+  const int64_t threads = (int64_t)B * L * 32;
+  router_logits_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(S, w, bias, logits, sum_sq, B, L, row_elems);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_route_compact(const RouteArgs& a, cudaStream_t stream) {
   dim3 grid(a.nblocks, a.B);

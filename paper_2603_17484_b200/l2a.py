@@ -20,13 +20,14 @@ FLAG_SAVE_FOR_BWD = 1
 FLAG_SKIP_LOCAL = 2
 FLAG_SKIP_GLOBAL = 4
 FLAG_FORCE_ALL_GLOBAL = 8
+FLAG_GLOBAL_PHASE = 16
 ROUTER_MASK_U8 = 0
 ROUTER_LOGITS_F32 = 1
 
 EXPORTS = (
     "l2a_version", "l2a_status_string", "l2a_workspace_bytes", "l2a_workspace_status",
     "l2a_route_compact", "l2a_forward", "l2a_backward", "l2a_step_host", "l2a_profile_next_call",
-    "l2a_route_compact_static",
+    "l2a_route_compact_static", "l2a_router_logits",
 )
 
 
@@ -128,6 +129,15 @@ def l2a_route_compact_static(p, router, router_kind, logit_threshold, d_mask, q_
                                           _ptr(n_routed), _ptr(prefix), _stream(stream))
     if check:
         _check(code, "l2a_route_compact_static")
+    return code
+
+
+def l2a_router_logits(p, S, w, bias, logits, sum_sq=None, stream=None, check=True) -> int:
+    """Router logits z_t = w . s_t + bias from the local output (Eq. 3); optional sum of sigmoid(z)^2 per batch entry."""
+    code = lib().l2a_router_logits(ctypes.byref(p), _ptr(S), _ptr(w), ctypes.c_float(bias), _ptr(logits), _ptr(sum_sq),
+                                   _stream(stream))
+    if check:
+        _check(code, "l2a_router_logits")
     return code
 
 

@@ -258,3 +258,16 @@ def test_dgate_matches_definition():
     want = (ref["a"] * bf16_bits_to_f64(dO)).sum(axis=(2, 3))[0]
     got = oracle.dgate_rows(sh, Q, K, V, dO, np.zeros(L, np.int32), np.arange(L))
     np.testing.assert_allclose(got, want, atol=1e-12)
+
+
+def test_router_logits_closed_forms():
+    # a one-hot router weight picks one coordinate of s_t; a zero router gives the bias for every token, and a
+    # zero-initialised router (bias 0) sits exactly on the threshold, which routes every token (Section 3.1)
+    B, L, Hq, D = 2, 9, 2, 4
+    S = rand_bf16((B, L, Hq, D))
+    s = bf16_bits_to_f64(S).reshape(B, L, Hq * D)
+    w = np.zeros(Hq * D); w[5] = 2.0
+    np.testing.assert_allclose(oracle.router_logits(S, w, 0.25), 2.0 * s[:, :, 5] + 0.25, atol=1e-15)
+    z0 = oracle.router_logits(S, np.zeros(Hq * D), 0.0)
+    assert (z0 == 0).all() and oracle.route(z0.astype(np.float32), 0.0).all()
+    np.testing.assert_allclose(oracle.gate_regulariser_sum(z0), np.full(B, L * 0.25), atol=1e-15)   # sigmoid(0)^2 = 1/4
