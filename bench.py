@@ -152,6 +152,49 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def run_decode(args):
+    """Decode-step measurement (not the headline metric): one new token per sequence against a 128K-token cache,
+    local window always, whole cache for the routed sequences.  HBM roofline."""
+    from paper_2603_17484_b200 import l2a
+    torch.cuda.set_device(0)
+    cfg = synth.CONFIGS["qwen3_8b_128k"]
+    B, Lk = args.decode_batch, cfg.L
+    rho = 0.2 if args.density is None else args.density
+    p = l2a.params(B, 1, Lk, cfg.Hq, cfg.Hkv, cfg.D, cfg.W)
+    g = torch.Generator(device="cuda"); g.manual_seed(7)
+    q = torch.randn((B, 1, cfg.Hq, cfg.D), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    K = torch.randn((B, Lk, cfg.Hkv, cfg.D), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    V = torch.randn((B, Lk, cfg.Hkv, cfg.D), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    d_host = (np.random.default_rng(11).random(B) < rho).astype(np.uint8)
+    d = torch.from_numpy(d_host).cuda()
+    O = torch.empty((B, 1, cfg.Hq, cfg.D), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(l2a.l2a_decode_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    for _ in range(max(3, args.warmup)):
+        l2a.l2a_decode(p, q, K, V, d, O, ws)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(args.steps):
+        l2a.l2a_decode(p, q, K, V, d, O, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    row = cfg.Hkv * cfg.D * 2 * 2                                   # K and V bytes of one cached position
+    alg_bytes = float(B * (cfg.W + 1) * row + int(d_host.sum()) * Lk * row)
+    peaks = measured_peaks()
+    gbs = alg_bytes / ms / 1e6
+    print(json.dumps({
+        "metric": "L2A decode step, achieved HBM GB/s", "value": gbs, "unit": "GB/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "decode_128k", "B": B, "Lk": Lk, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D, "W": cfg.W,
+                   "routed_sequences": int(d_host.sum()),
+                   "l2_policy": "K/V cache of %.1f GB exceeds L2" % (2 * K.numel() * 2 / 1e9)},
+        "roofline": {"bound": "hbm", "kernel": "decode_split_kernel", "achieved": gbs, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                     "algorithmic_bytes_per_launch": alg_bytes},
+        "gpu_launches": 2 * args.steps}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -165,11 +208,15 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-tokens", type=int, default=2048, help="tokens of the CPU-baseline sample (0 = skip)")
     ap.add_argument("--ref-tokens", type=int, default=1024, help="tokens per step of --impl reference")
+    ap.add_argument("--decode", action="store_true", help="measure the decode step instead (HBM roofline)")
+    ap.add_argument("--decode-batch", type=int, default=16)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     if args.impl == "reference":
         return run_reference(args)
+    if args.decode:
+        return run_decode(args)
 
     from paper_2603_17484_b200 import l2a
 

@@ -188,6 +188,24 @@ l2a_status l2a_backward(const l2a_params* p, const void* Q, const void* K, const
                         float* dgate, void* bwd_ws, size_t bwd_ws_bytes, void* stream);
 
 /*
+ * Decode step (Section 3.4): one new token per sequence.  The token attends to the last `window` + 1 keys of
+ * the cache (Local Attention) and, only when its routing decision is 1, to the whole cache (Global
+ * Attention, skipped entirely otherwise); o = s + d * a.  The full K/V cache is kept either way, because a
+ * later routed token may need it.
+ *
+ *   p           : Lq must be 1; Lk = number of cached tokens INCLUDING the new one; q_pos_offset = position of
+ *                 the new token (normally Lk - 1); Hq / Hkv <= 8.
+ *   q           in : bf16 [B, 1, Hq, D];  K, V in: bf16 [B, Lk, Hkv, D] (the cache).
+ *   d           in : uint8 [B] routing decision of the new token (NULL = not routed); device memory.
+ *   O           out: bf16 [B, 1, Hq, D].
+ *   ws             : workspace of l2a_decode_workspace_bytes (partial soft-max results of the key chunks).
+ * HBM-bound: reads the local window once and, for routed tokens, the cache once.
+ */
+l2a_status l2a_decode_workspace_bytes(const l2a_params* p, size_t* ws_bytes);
+l2a_status l2a_decode(const l2a_params* p, const void* q, const void* K, const void* V, const uint8_t* d,
+                      void* O, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * One whole step for callers that hold HOST buffers, so that end-to-end time including the
  * transfers can be measured through the C ABI: copies Q, K, V, the router input (and dO) to the
  * device buffers the caller supplies, runs l2a_route_compact + l2a_forward (+ l2a_backward when

@@ -27,7 +27,7 @@ ROUTER_LOGITS_F32 = 1
 EXPORTS = (
     "l2a_version", "l2a_status_string", "l2a_workspace_bytes", "l2a_workspace_status",
     "l2a_route_compact", "l2a_forward", "l2a_backward", "l2a_step_host", "l2a_profile_next_call",
-    "l2a_route_compact_static", "l2a_router_logits",
+    "l2a_route_compact_static", "l2a_router_logits", "l2a_decode_workspace_bytes", "l2a_decode",
 )
 
 
@@ -129,6 +129,21 @@ def l2a_route_compact_static(p, router, router_kind, logit_threshold, d_mask, q_
                                           _ptr(n_routed), _ptr(prefix), _stream(stream))
     if check:
         _check(code, "l2a_route_compact_static")
+    return code
+
+
+def l2a_decode_workspace_bytes(p) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().l2a_decode_workspace_bytes(ctypes.byref(p), ctypes.byref(n)), "l2a_decode_workspace_bytes")
+    return n.value
+
+
+def l2a_decode(p, q, K, V, d, O, ws, stream=None, check=True) -> int:
+    """Decode step: one new token per sequence against the K/V cache (local window always, whole cache if d = 1)."""
+    code = lib().l2a_decode(ctypes.byref(p), _ptr(q), _ptr(K), _ptr(V), _ptr(d), _ptr(O), _ptr(ws),
+                            ctypes.c_size_t(ws.numel() if ws is not None else 0), _stream(stream))
+    if check:
+        _check(code, "l2a_decode")
     return code
 
 

@@ -1,0 +1,36 @@
+"""Decode step against the oracle: the layer with a single query row placed at the end of the cache."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2603_17484_b200 import l2a, synth
+from tests.gpu_util import check_close, to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("B,Lk,Hq,Hkv,D,W", [
+    (3, 1, 2, 1, 128, 16),          # cache of one token
+    (4, 700, 4, 1, 128, 200),       # G = 4
+    (2, 5000, 28, 4, 128, 4096),    # Qwen2.5-7B heads (G = 7), window larger than most of the cache
+    (3, 9001, 32, 8, 128, 4096),    # Qwen3-8B heads
+    (2, 3000, 4, 4, 64, 100),       # head dim 64, no grouping
+])
+def test_decode_matches_oracle(B, Lk, Hq, Hkv, D, W):
+    t = synth.qkv(B, 1, Hq, Hkv, D, seed=Lk + Hq, Lk=Lk)
+    d = (np.arange(B) % 2).astype(np.uint8)[:, None]          # alternate routed / not routed, shape [B, 1]
+    p = l2a.params(B, 1, Lk, Hq, Hkv, D, W)
+    ws = torch.empty(l2a.l2a_decode_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    q, K, V = (t[k].cuda() for k in ("Q", "K", "V"))
+    O = torch.full((B, 1, Hq, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    l2a.l2a_decode(p, q, K, V, torch.from_numpy(d[:, 0].copy()).cuda(), O, ws)
+    torch.cuda.synchronize()
+    sh = oracle.Shape(B, 1, Lk, Hq, Hkv, D, W)
+    ref = oracle.forward_full(sh, synth.as_u16(t["Q"]), synth.as_u16(t["K"]), synth.as_u16(t["V"]), d)
+    check_close(to_f64(O), ref["o"], "decode O")
+    # a not-routed token equals the sliding-window output exactly as computed for d == 0
+    O0 = torch.empty_like(O)
+    l2a.l2a_decode(p, q, K, V, None, O0, ws)
+    torch.cuda.synchronize()
+    check_close(to_f64(O0), ref["s"], "decode O with no routing (local only)")
