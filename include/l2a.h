@@ -198,8 +198,12 @@ l2a_status l2a_backward(const l2a_params* p, const void* Q, const void* K, const
  *   q           in : bf16 [B, 1, Hq, D];  K, V in: bf16 [B, Lk, Hkv, D] (the cache).
  *   d           in : uint8 [B] routing decision of the new token (NULL = not routed); device memory.
  *   O           out: bf16 [B, 1, Hq, D].
- *   ws             : workspace of l2a_decode_workspace_bytes (partial soft-max results of the key chunks).
- * HBM-bound: reads the local window once and, for routed tokens, the cache once.
+ *   ws             : device workspace of l2a_decode_workspace_bytes, 256-byte aligned: a status header (read it
+ *                    with l2a_workspace_status) and the partial soft-max results of the key chunks.
+ * Keys after q_pos_offset are never used, whatever they hold.  HBM-bound: reads the local window once and, for
+ * routed tokens, the cache once.  Errors: L2A_ERR_INVALID_ARG (Lq != 1, NULL or unaligned pointers),
+ * L2A_ERR_UNSUPPORTED (Hq / Hkv > 8), L2A_ERR_WORKSPACE, L2A_ERR_CUDA; a bounded device wait that runs out is
+ * reported by the status header, not by the return value.
  */
 l2a_status l2a_decode_workspace_bytes(const l2a_params* p, size_t* ws_bytes);
 l2a_status l2a_decode(const l2a_params* p, const void* q, const void* K, const void* V, const uint8_t* d,

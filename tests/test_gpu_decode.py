@@ -34,3 +34,27 @@ def test_decode_matches_oracle(B, Lk, Hq, Hkv, D, W):
     l2a.l2a_decode(p, q, K, V, None, O0, ws)
     torch.cuda.synchronize()
     check_close(to_f64(O0), ref["s"], "decode O with no routing (local only)")
+
+
+@pytest.mark.parametrize("B,Lk,pos,Hq,Hkv,D,W", [
+    (2, 4096, 3000, 8, 2, 128, 512),     # cache allocated ahead of the sequence
+    (1, 70000, 69990, 32, 8, 128, 4096), # one sequence: the chunk plan shrinks its chunks to fill the SMs
+    (2, 1000, 63, 4, 2, 64, 31),         # position on a tile boundary, window smaller than a tile
+])
+def test_decode_ignores_cache_past_the_position(B, Lk, pos, Hq, Hkv, D, W):
+    """Rows of the cache after the new token's position are not part of the sequence yet: whatever they hold (NaN
+    here) must not reach the output."""
+    t = synth.qkv(B, 1, Hq, Hkv, D, seed=pos, Lk=Lk)
+    d = np.ones((B, 1), dtype=np.uint8)
+    p = l2a.params(B, 1, Lk, Hq, Hkv, D, W, q_pos_offset=pos)
+    ws = torch.empty(l2a.l2a_decode_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    q, K, V = (t[k].cuda() for k in ("Q", "K", "V"))
+    K[:, pos + 1:] = float("nan")
+    V[:, pos + 1:] = float("nan")
+    O = torch.full((B, 1, Hq, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    l2a.l2a_decode(p, q, K, V, torch.from_numpy(d[:, 0].copy()).cuda(), O, ws)
+    torch.cuda.synchronize()
+    assert l2a.l2a_workspace_status(ws) == 0
+    sh = oracle.Shape(B, 1, Lk, Hq, Hkv, D, W, q_pos_offset=pos)
+    ref = oracle.forward_full(sh, synth.as_u16(t["Q"]), synth.as_u16(t["K"]), synth.as_u16(t["V"]), d)
+    check_close(to_f64(O), ref["o"], "decode O, position before the end of the cache")
