@@ -200,7 +200,9 @@ l2a_status l2a_backward(const l2a_params* p, const void* Q, const void* K, const
  *   O           out: bf16 [B, 1, Hq, D].
  *   ws             : device workspace of l2a_decode_workspace_bytes, 256-byte aligned: a status header (read it
  *                    with l2a_workspace_status) and the partial soft-max results of the key chunks.
- * Keys after q_pos_offset are never used, whatever they hold.  HBM-bound: reads the local window once and, for
+ * Keys after q_pos_offset are never used, whatever they hold.  A layer whose Global Attention was pruned keeps
+ * only its last window + 1 keys: call with d = NULL, Lk = window + 1 slots (q_pos_offset = Lk - 1); the result
+ * does not depend on the order of the slots, so the cache may be a ring buffer.  HBM-bound: reads the local window once and, for
  * routed tokens, the cache once.  Errors: L2A_ERR_INVALID_ARG (Lq != 1, NULL or unaligned pointers),
  * L2A_ERR_UNSUPPORTED (Hq / Hkv > 8), L2A_ERR_WORKSPACE, L2A_ERR_CUDA; a bounded device wait that runs out is
  * reported by the status header, not by the return value.

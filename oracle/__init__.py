@@ -22,4 +22,5 @@ from .binding import (  # noqa: F401
     f64_inputs,
     router_logits,
     gate_regulariser_sum,
+    router_backward,
 )

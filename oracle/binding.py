@@ -197,6 +197,34 @@ def router_logits(S, w, bias: float = 0.0):
     return s64.reshape(B, L, -1) @ np.asarray(w, np.float64) + float(bias)
 
 
+def router_backward(S, w, z, dgate, reg_coeff: float, dO=None):
+    """Backward of the router under the straight-through estimator (Section 3.3).
+
+    The decision d_t is replaced by its relaxation d_hat_t = sigmoid(z_t) in the backward pass, so (Eq. 7)
+        dL/dd_hat_t = dgate_t + 2 * reg_coeff * d_hat_t,       dgate_t = (dL_NTP/do_t) . a_t,  reg_coeff = lambda / (n L),
+        dL/dz_t     = dL/dd_hat_t * d_hat_t * (1 - d_hat_t)    (derivative of the sigmoid),
+        dL/dW       = sum over tokens of dL/dz_t * s_t,        dL/dbias = sum over tokens of dL/dz_t,
+        dL/ds_t    += dL/dz_t * W                              (on top of dL/do_t, since o_t = s_t + d_t a_t).
+    S, dO: bf16 bit patterns (uint16) [B, L, Hq, D]; w: [Hq*D]; z, dgate: [B, L].  Returns fp64
+    dz [B, L], dw [Hq*D], dbias (scalar), dS [B, L, Hq, D] (= dO + dz * W; None when dO is None)."""
+    S = np.ascontiguousarray(S)
+    s64 = (S.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    B, L = S.shape[0], S.shape[1]
+    s64 = s64.reshape(B, L, -1)
+    w = np.asarray(w, np.float64)
+    d_hat = 1.0 / (1.0 + np.exp(-np.asarray(z, np.float64)))
+    dd_hat = np.asarray(dgate, np.float64) + 2.0 * float(reg_coeff) * d_hat
+    dz = dd_hat * d_hat * (1.0 - d_hat)
+    dw = np.einsum("bt,btk->k", dz, s64)
+    dbias = dz.sum()
+    dS = None
+    if dO is not None:
+        dO = np.ascontiguousarray(dO)
+        do64 = (dO.astype(np.uint32) << 16).view(np.float32).astype(np.float64).reshape(B, L, -1)
+        dS = (do64 + dz[:, :, None] * w[None, None, :]).reshape(S.shape)
+    return dz, dw, dbias, dS
+
+
 def gate_regulariser_sum(z):
     """Sum over tokens of sigmoid(z_t)^2 per batch entry (Eq. 6 without its lambda / (n L) factor)."""
     g = 1.0 / (1.0 + np.exp(-np.asarray(z, np.float64)))

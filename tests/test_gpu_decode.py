@@ -58,3 +58,26 @@ def test_decode_ignores_cache_past_the_position(B, Lk, pos, Hq, Hkv, D, W):
     sh = oracle.Shape(B, 1, Lk, Hq, Hkv, D, W, q_pos_offset=pos)
     ref = oracle.forward_full(sh, synth.as_u16(t["Q"]), synth.as_u16(t["K"]), synth.as_u16(t["V"]), d)
     check_close(to_f64(O), ref["o"], "decode O, position before the end of the cache")
+
+
+def test_decode_pruned_layer_ring_cache():
+    """A layer whose Global Attention was pruned (Section 3.4, sparsity-based layer pruning) keeps only the last
+    W + 1 keys.  Attention does not depend on the order of the keys, so the cache can be a ring buffer: the decode
+    call with d = NULL over the W + 1 slots, in whatever rotation they are, gives the sliding-window output."""
+    B, L, Hq, Hkv, D, W = 2, 3000, 8, 2, 128, 511
+    t = synth.qkv(B, 1, Hq, Hkv, D, seed=99, Lk=L)
+    sh = oracle.Shape(B, 1, L, Hq, Hkv, D, W)
+    ref = oracle.forward_full(sh, synth.as_u16(t["Q"]), synth.as_u16(t["K"]), synth.as_u16(t["V"]),
+                              np.zeros((B, 1), dtype=np.uint8))
+    # ring buffer of W + 1 slots: position j lives in slot j % (W + 1)
+    slots = W + 1
+    order = torch.tensor([(L - slots + i) for i in range(slots)])
+    ring = torch.empty(slots, dtype=torch.long)
+    ring[order % slots] = order
+    Kr, Vr = t["K"][:, ring].contiguous().cuda(), t["V"][:, ring].contiguous().cuda()
+    p = l2a.params(B, 1, slots, Hq, Hkv, D, W)
+    ws = torch.empty(l2a.l2a_decode_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    O = torch.empty((B, 1, Hq, D), dtype=torch.bfloat16, device="cuda")
+    l2a.l2a_decode(p, t["Q"].cuda(), Kr, Vr, None, O, ws)
+    torch.cuda.synchronize()
+    check_close(to_f64(O), ref["s"], "decode over a ring-buffer local cache")

@@ -271,3 +271,38 @@ def test_router_logits_closed_forms():
     z0 = oracle.router_logits(S, np.zeros(Hq * D), 0.0)
     assert (z0 == 0).all() and oracle.route(z0.astype(np.float32), 0.0).all()
     np.testing.assert_allclose(oracle.gate_regulariser_sum(z0), np.full(B, L * 0.25), atol=1e-15)   # sigmoid(0)^2 = 1/4
+
+
+def test_router_backward_is_the_gradient_of_the_relaxed_loss():
+    # Under the straight-through estimator the loss seen by the router is, with a_t and dL/do_t held fixed,
+    #   F(W, bias, s) = sum_t g_t * sigmoid(z_t) + c * sum_t sigmoid(z_t)^2,   z_t = W s_t + bias,  g_t = dL/do_t . a_t
+    # (Eq. 5 with d_t -> d_hat_t, plus the regulariser of Eq. 6).  Central differences of F pin dW, dbias and the
+    # router's contribution to dL/ds_t: a dropped factor 2, a missing sigmoid derivative or a wrong sign fails.
+    B, L, Hq, D = 2, 7, 2, 4
+    rng = np.random.default_rng(17)
+    S = rand_bf16((B, L, Hq, D))
+    s = bf16_bits_to_f64(S).reshape(B, L, Hq * D)
+    w = rng.standard_normal(Hq * D) * 0.4
+    bias, c = -0.2, 0.37
+    g = rng.standard_normal((B, L))
+
+    def F(w_, bias_, s_):
+        d_hat = 1.0 / (1.0 + np.exp(-(s_ @ w_ + bias_)))
+        return float((g * d_hat).sum() + c * (d_hat ** 2).sum())
+
+    z = oracle.router_logits(S, w, bias)
+    dO = rand_bf16((B, L, Hq, D))
+    dz, dw, dbias, dS = oracle.router_backward(S, w, z, g, c, dO)
+    eps = 1e-6
+    for k in range(Hq * D):
+        e = np.zeros(Hq * D); e[k] = eps
+        assert abs((F(w + e, bias, s) - F(w - e, bias, s)) / (2 * eps) - dw[k]) < 1e-7
+    assert abs((F(w, bias + eps, s) - F(w, bias - eps, s)) / (2 * eps) - dbias) < 1e-7
+    ds_router = dS.reshape(B, L, Hq * D) - bf16_bits_to_f64(dO).reshape(B, L, Hq * D)
+    for (b, t, k) in [(0, 0, 0), (1, 3, 5), (1, 6, 7)]:
+        sp, sm = s.copy(), s.copy()
+        sp[b, t, k] += eps; sm[b, t, k] -= eps
+        assert abs((F(w, bias, sp) - F(w, bias, sm)) / (2 * eps) - ds_router[b, t, k]) < 1e-7
+    # closed form on the threshold: z = 0 gives d_hat = 1/2, so dz = (g + c) / 4
+    dz0, _, _, _ = oracle.router_backward(S, w, np.zeros((B, L)), g, c)
+    np.testing.assert_allclose(dz0, (g + c) / 4.0, atol=1e-15)
