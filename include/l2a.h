@@ -188,6 +188,57 @@ l2a_status l2a_backward(const l2a_params* p, const void* Q, const void* K, const
                         float* dgate, void* bwd_ws, size_t bwd_ws_bytes, void* stream);
 
 /*
+ * l2a_backward with a separate gradient for the local output.  o_t = s_t + d_t a_t, but s_t also feeds the
+ * router (z_t = W s_t + bias, Eq. 3), so in a trained layer dL/ds_t = dL/do_t + dz_t W (Section 3.3, straight-
+ * through estimator).  dS_loc (bf16 [B, Lq, Hq, D], e.g. written by l2a_router_backward) drives the Local
+ * Attention backward; dO drives the Global Attention backward (da_t = d_t dO_t) and dgate.  Everything else is as
+ * in l2a_backward, which is this call with dS_loc = dO.
+ */
+l2a_status l2a_backward_split(const l2a_params* p, const void* Q, const void* K, const void* V,
+                              const uint8_t* d_mask, const int32_t* q_idx, const int32_t* n_routed,
+                              const int32_t* prefix, const void* dO, const void* dS_loc, const void* S_save,
+                              const void* A_c, const float* lse_loc, const float* lse_glb, void* dQ, void* dK,
+                              void* dV, float* dgate, void* bwd_ws, size_t bwd_ws_bytes, void* stream);
+
+/*
+ * Router backward under the straight-through estimator (Section 3.3, Eq. 7, with the gradient of the sparsity
+ * regulariser of Eq. 6).  With d_hat_t = sigmoid(z_t):
+ *     dL/dd_hat_t = dgate_t + 2 reg_coeff d_hat_t,     dz_t = dL/dd_hat_t d_hat_t (1 - d_hat_t),
+ *     dw = sum_t dz_t s_t,   dbias = sum_t dz_t,   dS_loc_t = dO_t + dz_t w.
+ *
+ *   S           in : bf16 [B, Lq, Hq, D] local output (S_save of l2a_forward);  w in: fp32 [Hq * D].
+ *   logits      in : fp32 [B, Lq], z_t as written by l2a_router_logits.
+ *   dgate       in : optional fp32 [B, Lq] from l2a_backward (NULL = 0: regulariser only).
+ *   reg_coeff      : lambda / (n L) of Eq. 6 (n tokens, L layers); 0 disables the regulariser term.
+ *   dO, dS_loc     : optional pair (both or neither): bf16 [B, Lq, Hq, D] in / out, dS_loc = dO + dz w rounded to
+ *                    bf16 once; dS_loc may alias dO.
+ *   dz          out: optional fp32 [B, Lq].
+ *   dw, dbias   out: optional fp32 [Hq * D] and [1]; zeroed by this call, then accumulated with atomics (the last
+ *                    bits depend on the order of addition).
+ * All pointers are device memory.  HBM-bound: one pass over S (and over dO, dS_loc when given).
+ */
+l2a_status l2a_router_backward(const l2a_params* p, const void* S, const float* w, const float* logits,
+                               const float* dgate, float reg_coeff, const void* dO, float* dz, float* dw,
+                               float* dbias, void* dS_loc, void* stream);
+
+/*
+ * The whole layer forward in its defining order, without the caller in between: Local Attention (Eq. 2) ->
+ * router logits z_t = router_w . s_t + router_bias on the local output (Eq. 3) -> d_t = (z_t >= logit_threshold),
+ * compaction -> Global Attention of the routed tokens added into O (Eq. 4, 5).  Equal, bit for bit, to
+ * l2a_forward(L2A_FLAG_SKIP_GLOBAL), l2a_router_logits, l2a_route_compact, l2a_forward(L2A_FLAG_GLOBAL_PHASE).
+ *
+ *   p->flags       : L2A_FLAG_SAVE_FOR_BWD and L2A_FLAG_FORCE_ALL_GLOBAL allowed; the SKIP and PHASE flags are not.
+ *   logits      out: fp32 [B, Lq];  sum_sq out: optional fp32 [B] (see l2a_router_logits).
+ *   d_mask, q_idx, n_routed, prefix: outputs, as in l2a_route_compact; the remaining arguments as in l2a_forward.
+ * Nothing is read back to the host: the routed count stays on the device.
+ */
+l2a_status l2a_forward_routed(const l2a_params* p, const void* Q, const void* K, const void* V,
+                              const float* router_w, float router_bias, float logit_threshold, float* logits,
+                              float* sum_sq, uint8_t* d_mask, int32_t* q_idx, int32_t* n_routed, int32_t* prefix,
+                              void* O, void* S_save, void* A_c, float* lse_loc, float* lse_glb, void* route_ws,
+                              size_t route_ws_bytes, void* fwd_ws, size_t fwd_ws_bytes, void* stream);
+
+/*
  * Decode step (Section 3.4): one new token per sequence.  The token attends to the last `window` + 1 keys of
  * the cache (Local Attention) and, only when its routing decision is 1, to the whole cache (Global
  * Attention, skipped entirely otherwise); o = s + d * a.  The full K/V cache is kept either way, because a

@@ -41,7 +41,8 @@ __device__ long long g_trace[4][8192];
 
 // ------------------------------------------------------------------------------------------------
 // Delta / dgate preprocess: one warp per (b, t), looping over heads.
-__global__ void __launch_bounds__(256) bwd_delta_kernel(const bf16* __restrict__ dO, const bf16* __restrict__ S,
+__global__ void __launch_bounds__(256) bwd_delta_kernel(const bf16* __restrict__ dO, const bf16* __restrict__ dO_loc,
+                                                        const bf16* __restrict__ S,
                                                         const bf16* __restrict__ A_c,
                                                         const uint8_t* __restrict__ d_mask,
                                                         const int32_t* __restrict__ prefix, float* __restrict__ delta_loc,
@@ -60,12 +61,14 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const bf16* __restrict__
   for (int h = 0; h < Hq; ++h) {
     float dl = 0.f, dg = 0.f;
     const bf16* po = dO + row + (int64_t)h * D + lane * per_lane;
+    const bf16* pl = dO_loc + row + (int64_t)h * D + lane * per_lane;   // gradient of s_t (== dO unless split)
     const bf16* ps = S + row + (int64_t)h * D + lane * per_lane;
     const bf16* pa = A_c + crow + (int64_t)h * D + lane * per_lane;
     for (int e = 0; e < per_lane; e += 2) {
       const float2 o2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(po + e));
       const float2 s2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(ps + e));
-      dl += o2.x * s2.x + o2.y * s2.y;
+      const float2 l2 = dO_loc == dO ? o2 : __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(pl + e));
+      dl += l2.x * s2.x + l2.y * s2.y;
       if (routed || a_by_row) {
         const float2 a2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(pa + e));
         dg += o2.x * a2.x + o2.y * a2.y;
@@ -900,7 +903,18 @@ extern "C" l2a_status l2a_backward(const l2a_params* p, const void* Q, const voi
                                    const int32_t* prefix, const void* dO, const void* S_save, const void* A_c,
                                    const float* lse_loc, const float* lse_glb, void* dQ, void* dK, void* dV,
                                    float* dgate, void* bwd_ws, size_t bwd_ws_bytes, void* stream) {
+  return l2a_backward_split(p, Q, K, V, d_mask, q_idx, n_routed, prefix, dO, dO, S_save, A_c, lse_loc, lse_glb, dQ, dK,
+                            dV, dgate, bwd_ws, bwd_ws_bytes, stream);
+}
+
+extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, const void* K, const void* V,
+                                         const uint8_t* d_mask, const int32_t* q_idx, const int32_t* n_routed,
+                                         const int32_t* prefix, const void* dO, const void* dS_loc,
+                                         const void* S_save, const void* A_c, const float* lse_loc,
+                                         const float* lse_glb, void* dQ, void* dK, void* dV, float* dgate,
+                                         void* bwd_ws, size_t bwd_ws_bytes, void* stream) {
   if (!p) return L2A_ERR_INVALID_ARG;
+  if (!dS_loc || !aligned16(dS_loc)) return L2A_ERR_INVALID_ARG;
   size_t need = 0;
   l2a_status st = l2a_workspace_bytes(p, nullptr, nullptr, &need);
   if (st != L2A_OK) return st;
@@ -924,7 +938,7 @@ extern "C" l2a_status l2a_backward(const l2a_params* p, const void* Q, const voi
 
   CUtensorMap mapQ, mapDO, mapQc, mapDOc, mapK, mapV;
   if (!encode_rows_map(&mapQ, Q, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||
-      !encode_rows_map(&mapDO, dO, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||
+      !encode_rows_map(&mapDO, dS_loc, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||   // local items: dL/ds_t
       !encode_rows_map(&mapQc, Qc, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||
       !encode_rows_map(&mapDOc, dOc, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||
       !encode_rows_map(&mapK, K, p->B, p->Lk, p->Hkv * p->D, kTileN, p->D) ||
@@ -943,7 +957,8 @@ extern "C" l2a_status l2a_backward(const l2a_params* p, const void* Q, const voi
   {
     const int64_t warps = (int64_t)p->B * p->Lq;
     const unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
-    bwd_delta_kernel<<<blocks, 256, 0, s>>>(static_cast<const bf16*>(dO), static_cast<const bf16*>(S_save),
+    bwd_delta_kernel<<<blocks, 256, 0, s>>>(static_cast<const bf16*>(dO), static_cast<const bf16*>(dS_loc),
+                                            static_cast<const bf16*>(S_save),
                                             static_cast<const bf16*>(A_c), d_mask, prefix, delta_loc, delta_glb, dgate,
                                             p->B, p->Lq, p->Hq, p->D, force_all ? 1 : 0);
     if (cudaGetLastError() != cudaSuccess) return L2A_ERR_CUDA;

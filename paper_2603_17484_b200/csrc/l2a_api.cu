@@ -239,6 +239,58 @@ l2a_status l2a_router_logits(const l2a_params* p, const void* S, const float* w,
              : L2A_ERR_CUDA;
 }
 
+l2a_status l2a_router_backward(const l2a_params* p, const void* S, const float* w, const float* logits,
+                               const float* dgate, float reg_coeff, const void* dO, float* dz, float* dw, float* dbias,
+                               void* dS_loc, void* stream) {
+  l2a_status st = check_params(p);
+  if (st != L2A_OK) return st;
+  if (!S || !w || !logits) return L2A_ERR_INVALID_ARG;
+  if ((dO == nullptr) != (dS_loc == nullptr)) return L2A_ERR_INVALID_ARG;   // the combined gradient needs both
+  if (!aligned(S, 16) || !aligned(w, 16) || !aligned(dO, 16) || !aligned(dS_loc, 16) || !aligned(logits, 4) ||
+      !aligned(dgate, 4) || !aligned(dz, 4) || !aligned(dw, 4) || !aligned(dbias, 4))
+    return L2A_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (dw && cudaMemsetAsync(dw, 0, sizeof(float) * p->Hq * p->D, s) != cudaSuccess) return L2A_ERR_CUDA;
+  if (dbias && cudaMemsetAsync(dbias, 0, sizeof(float), s) != cudaSuccess) return L2A_ERR_CUDA;
+  return launch_router_backward(static_cast<const bf16*>(S), w, logits, dgate, reg_coeff,
+                                static_cast<const bf16*>(dO), dz, dw, dbias, static_cast<bf16*>(dS_loc), p->B, p->Lq,
+                                p->Hq * p->D, s) == cudaSuccess
+             ? L2A_OK
+             : L2A_ERR_CUDA;
+}
+
+l2a_status l2a_forward_routed(const l2a_params* p, const void* Q, const void* K, const void* V, const float* router_w,
+                              float router_bias, float logit_threshold, float* logits, float* sum_sq, uint8_t* d_mask,
+                              int32_t* q_idx, int32_t* n_routed, int32_t* prefix, void* O, void* S_save, void* A_c,
+                              float* lse_loc, float* lse_glb, void* route_ws, size_t route_ws_bytes, void* fwd_ws,
+                              size_t fwd_ws_bytes, void* stream) {
+  l2a_status st = check_params(p);
+  if (st != L2A_OK) return st;
+  if (p->flags & (L2A_FLAG_SKIP_LOCAL | L2A_FLAG_SKIP_GLOBAL | L2A_FLAG_GLOBAL_PHASE)) return L2A_ERR_INVALID_ARG;
+  if (!router_w || !logits || !d_mask || !q_idx || !n_routed || !prefix) return L2A_ERR_INVALID_ARG;
+  // every argument is checked before the first launch: the later stages would otherwise fail half-way
+  if (!aligned(router_w, 16) || !aligned(logits, 4)) return L2A_ERR_INVALID_ARG;
+  if (!ws_ok(route_ws, route_ws_bytes, route_ws_size(p)) || !ws_ok(fwd_ws, fwd_ws_bytes, fwd_ws_size(p)))
+    return L2A_ERR_WORKSPACE;
+  const bool save = p->flags & L2A_FLAG_SAVE_FOR_BWD;
+  // Eq. 2: local attention for every token
+  l2a_params ph = *p;
+  ph.flags = (p->flags & ~L2A_FLAG_FORCE_ALL_GLOBAL) | L2A_FLAG_SKIP_GLOBAL;
+  st = l2a_forward(&ph, Q, K, V, d_mask, q_idx, n_routed, prefix, O, S_save, A_c, lse_loc, lse_glb, fwd_ws,
+                   fwd_ws_bytes, stream);
+  if (st != L2A_OK) return st;
+  // Eq. 3: router on the local output, threshold, compaction
+  st = l2a_router_logits(p, save ? S_save : O, router_w, router_bias, logits, sum_sq, stream);
+  if (st != L2A_OK) return st;
+  st = l2a_route_compact(p, logits, L2A_ROUTER_LOGITS_F32, logit_threshold, d_mask, q_idx, n_routed, prefix, route_ws,
+                         route_ws_bytes, stream);
+  if (st != L2A_OK) return st;
+  // Eq. 4 and 5: global attention of the routed tokens, added into O
+  ph.flags = p->flags | L2A_FLAG_GLOBAL_PHASE;
+  return l2a_forward(&ph, Q, K, V, d_mask, q_idx, n_routed, prefix, O, S_save, A_c, lse_loc, lse_glb, fwd_ws,
+                     fwd_ws_bytes, stream);
+}
+
 l2a_status l2a_profile_next_call(void* const* events, int n_events) {
   if (n_events < 0 || n_events > 8 || (n_events > 0 && !events)) return L2A_ERR_INVALID_ARG;
   PhaseEvents& pe = phase_events();

@@ -50,6 +50,12 @@ cudaError_t launch_gather_rows(const bf16* src, bf16* dst, const int32_t* q_idx,
 cudaError_t launch_router_logits(const bf16* S, const float* w, float bias, float* logits, float* sum_sq, int B,
                                  int L, int row_elems, cudaStream_t stream);
 
+// Router backward (Eq. 7 with the regulariser's gradient): dz [B,L], dW [row_elems] and dbias [1] (both added with
+// atomics to buffers the caller zeroed), dS = dO + dz * w (bf16 rows); dgate, dO/dS, dz, dw, dbias may be NULL.
+cudaError_t launch_router_backward(const bf16* S, const float* w, const float* logits, const float* dgate, float coeff,
+                                   const bf16* dO, float* dz, float* dw, float* dbias, bf16* dS, int B, int L,
+                                   int row_elems, cudaStream_t stream);
+
 struct FwdArgs {
   int B, Lq, Lk, Hq, Hkv, D;
   int window, q_pos_offset;

@@ -28,6 +28,7 @@ EXPORTS = (
     "l2a_version", "l2a_status_string", "l2a_workspace_bytes", "l2a_workspace_status",
     "l2a_route_compact", "l2a_forward", "l2a_backward", "l2a_step_host", "l2a_profile_next_call",
     "l2a_route_compact_static", "l2a_router_logits", "l2a_decode_workspace_bytes", "l2a_decode",
+    "l2a_backward_split", "l2a_router_backward", "l2a_forward_routed",
 )
 
 
@@ -177,6 +178,45 @@ def l2a_backward(p, Q, K, V, d_mask, q_idx, n_routed, prefix, dO, S_save, A_c, l
                               _stream(stream))
     if check:
         _check(code, "l2a_backward")
+    return code
+
+
+def l2a_backward_split(p, Q, K, V, d_mask, q_idx, n_routed, prefix, dO, dS_loc, S_save, A_c, lse_loc, lse_glb, dQ,
+                       dK, dV, dgate, bwd_ws, stream=None, check=True) -> int:
+    """l2a_backward with a separate gradient dS_loc for the local output (dO + the router path)."""
+    code = lib().l2a_backward_split(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(d_mask), _ptr(q_idx),
+                                    _ptr(n_routed), _ptr(prefix), _ptr(dO), _ptr(dS_loc), _ptr(S_save), _ptr(A_c),
+                                    _ptr(lse_loc), _ptr(lse_glb), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dgate),
+                                    _ptr(bwd_ws),
+                                    ctypes.c_size_t(bwd_ws.numel() * bwd_ws.element_size() if bwd_ws is not None else 0),
+                                    _stream(stream))
+    if check:
+        _check(code, "l2a_backward_split")
+    return code
+
+
+def l2a_router_backward(p, S, w, logits, dgate, reg_coeff, dO=None, dz=None, dw=None, dbias=None, dS_loc=None,
+                        stream=None, check=True) -> int:
+    """Router backward (Eq. 7 + regulariser gradient): dz, dw, dbias and dS_loc = dO + dz * w."""
+    code = lib().l2a_router_backward(ctypes.byref(p), _ptr(S), _ptr(w), _ptr(logits), _ptr(dgate),
+                                     ctypes.c_float(reg_coeff), _ptr(dO), _ptr(dz), _ptr(dw), _ptr(dbias),
+                                     _ptr(dS_loc), _stream(stream))
+    if check:
+        _check(code, "l2a_router_backward")
+    return code
+
+
+def l2a_forward_routed(p, Q, K, V, router_w, router_bias, logit_threshold, logits, sum_sq, d_mask, q_idx, n_routed,
+                       prefix, O, S_save, A_c, lse_loc, lse_glb, route_ws, fwd_ws, stream=None, check=True) -> int:
+    """Layer forward in its defining order in one call: local -> router -> route/compact -> global (Eq. 2-5)."""
+    nbytes = lambda t: ctypes.c_size_t(t.numel() * t.element_size() if t is not None else 0)
+    code = lib().l2a_forward_routed(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(router_w),
+                                    ctypes.c_float(router_bias), ctypes.c_float(logit_threshold), _ptr(logits),
+                                    _ptr(sum_sq), _ptr(d_mask), _ptr(q_idx), _ptr(n_routed), _ptr(prefix), _ptr(O),
+                                    _ptr(S_save), _ptr(A_c), _ptr(lse_loc), _ptr(lse_glb), _ptr(route_ws),
+                                    nbytes(route_ws), _ptr(fwd_ws), nbytes(fwd_ws), _stream(stream))
+    if check:
+        _check(code, "l2a_forward_routed")
     return code
 
 
