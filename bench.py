@@ -197,6 +197,54 @@ def run_decode(args):
         "gpu_launches": 2 * args.steps}), flush=True)
 
 
+def run_router(args):
+    """Router kernels on the headline shape (not the headline metric): logits from the local output (Eq. 3) and
+    the backward of Eq. 7 with dS_loc = dO + dz w.  HBM roofline; S, dO and dS_loc are 1.07 GB each (exceed L2)."""
+    from paper_2603_17484_b200 import l2a
+    torch.cuda.set_device(0)
+    cfg = synth.CONFIGS[args.workload]
+    B, L, E = cfg.B, cfg.L, cfg.Hq * cfg.D
+    p = l2a.params(B, L, L, cfg.Hq, cfg.Hkv, cfg.D, cfg.W)
+    g = torch.Generator(device="cuda"); g.manual_seed(3)
+    S = torch.randn((B, L, cfg.Hq, cfg.D), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    dO = torch.randn((B, L, cfg.Hq, cfg.D), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    dS = torch.empty_like(dO)
+    w = torch.randn((E,), generator=g, device="cuda", dtype=torch.float32) * 0.02
+    dgate = torch.randn((B, L), generator=g, device="cuda", dtype=torch.float32)
+    logits = torch.empty((B, L), dtype=torch.float32, device="cuda")
+    sum_sq = torch.empty((B,), dtype=torch.float32, device="cuda")
+    dz = torch.empty_like(logits)
+    dw = torch.empty((E,), dtype=torch.float32, device="cuda")
+    dbias = torch.empty((1,), dtype=torch.float32, device="cuda")
+    steps, warm = args.steps, max(3, args.warmup)
+    def timed(fn):
+        for _ in range(warm):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+    ms_fwd = timed(lambda: l2a.l2a_router_logits(p, S, w, 0.0, logits, sum_sq))
+    ms_bwd = timed(lambda: l2a.l2a_router_backward(p, S, w, logits, dgate, 1e-3, dO, dz, dw, dbias, dS))
+    row = E * 2
+    bytes_fwd, bytes_bwd = float(B * L * (row + 4)), float(B * L * (3 * row + 12))
+    peak = measured_peaks()["hbm_gbs"]
+    print(json.dumps({
+        "metric": "L2A router kernels, achieved HBM GB/s", "value": bytes_bwd / ms_bwd / 1e6, "unit": "GB/s", "n_gpus": 1,
+        "steps": steps, "warmup": warm, "ms_per_step": ms_bwd, "higher_is_better": True, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload + "_router", "B": B, "L": L, "row_elems": E,
+                   "l2_policy": "S, dO and dS_loc of %.2f GB each exceed L2" % (B * L * row / 1e9)},
+        "router_logits": {"ms": ms_fwd, "GB/s": bytes_fwd / ms_fwd / 1e6, "frac": bytes_fwd / ms_fwd / 1e6 / peak},
+        "roofline": {"bound": "hbm", "kernel": "router_backward_kernel", "achieved": bytes_bwd / ms_bwd / 1e6, "peak": peak,
+                     "unit": "GB/s", "frac": bytes_bwd / ms_bwd / 1e6 / peak, "traffic": None,
+                     "algorithmic_bytes_per_launch": bytes_bwd},
+        "gpu_launches": steps}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -212,6 +260,7 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=1024, help="tokens per step of --impl reference")
     ap.add_argument("--decode", action="store_true", help="measure the decode step instead (HBM roofline)")
     ap.add_argument("--decode-batch", type=int, default=16)
+    ap.add_argument("--router", action="store_true", help="measure the router kernels instead (HBM roofline)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -219,6 +268,8 @@ def main():
         return run_reference(args)
     if args.decode:
         return run_decode(args)
+    if args.router:
+        return run_router(args)
 
     from paper_2603_17484_b200 import l2a
 

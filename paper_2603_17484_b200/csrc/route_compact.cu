@@ -137,45 +137,86 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const bf16* __restrict
   }
 }
 
-// Router logit (Eq. 3): one warp per token, 16-byte loads of the token's Hq*D values, fp32 accumulation.
+// Router logit (Eq. 3).  The grid is sized to the machine: every warp owns a contiguous range of tokens and takes
+// four of them at a time, so that each 32-byte piece of w fetched (from L1) serves four 16-byte loads of S and
+// several rows are in flight per warp; fp32 accumulation.
+constexpr int kRlTokens = 4;
 __global__ void __launch_bounds__(256) router_logits_kernel(const bf16* __restrict__ S, const float* __restrict__ w,
                                                             float bias, float* __restrict__ logits,
                                                             float* __restrict__ sum_sq, int B, int L, int row_elems) {
-  const int64_t token = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t n_tokens = (int64_t)B * L;
+  const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+  const int64_t gw = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
-  if (token >= (int64_t)B * L) return;
-  const uint4* row = reinterpret_cast<const uint4*>(S + token * row_elems);
+  const int64_t t_begin = n_tokens * gw / n_warps, t_end = n_tokens * (gw + 1) / n_warps;
+  const int n_chunks = row_elems / 8;
   const float4* w4 = reinterpret_cast<const float4*>(w);
-  float acc = 0.f;
-  for (int i = lane; i < row_elems / 8; i += 32) {
-    const uint4 v = __ldg(&row[i]);
-    const float4 wa = __ldg(&w4[2 * i]), wb = __ldg(&w4[2 * i + 1]);
-    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
-    const float ww[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+  // sum of sigmoid^2 of this warp's tokens, flushed with one atomic per batch entry the range touches
+  float reg_sum = 0.f;
+  int64_t reg_b = t_begin / L;
+  for (int64_t token0 = t_begin; token0 < t_end; token0 += kRlTokens) {
+    const uint4* rows[kRlTokens];
+    float acc[kRlTokens];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      acc = fmaf(__uint_as_float(u[k] << 16), ww[2 * k], acc);
-      acc = fmaf(__uint_as_float(u[k] & 0xffff0000u), ww[2 * k + 1], acc);
+    for (int r = 0; r < kRlTokens; ++r) {
+      // rows past the range re-read its last token; their result is not stored
+      const int64_t tok = token0 + r < t_end ? token0 + r : t_end - 1;
+      rows[r] = reinterpret_cast<const uint4*>(S) + tok * n_chunks;
+      acc[r] = 0.f;
+    }
+#pragma unroll 2
+    for (int i = lane; i < n_chunks; i += 32) {
+      uint4 v[kRlTokens];
+#pragma unroll
+      for (int r = 0; r < kRlTokens; ++r) v[r] = __ldg(&rows[r][i]);
+      const float4 wa = __ldg(&w4[2 * i]), wb = __ldg(&w4[2 * i + 1]);
+      const float ww[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+      for (int r = 0; r < kRlTokens; ++r) {
+        const uint32_t u[4] = {v[r].x, v[r].y, v[r].z, v[r].w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          acc[r] = fmaf(__uint_as_float(u[k] << 16), ww[2 * k], acc[r]);
+          acc[r] = fmaf(__uint_as_float(u[k] & 0xffff0000u), ww[2 * k + 1], acc[r]);
+        }
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < kRlTokens; ++r) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc[r] += __shfl_xor_sync(0xffffffffu, acc[r], o);
+      if (lane == 0 && token0 + r < t_end) {
+        const float z = acc[r] + bias;
+        logits[token0 + r] = z;
+        if (sum_sq != nullptr) {
+          const float g = 1.0f / (1.0f + __expf(-z));
+          const int64_t bb = (token0 + r) / L;
+          if (bb != reg_b) {
+            atomicAdd(&sum_sq[reg_b], reg_sum);
+            reg_sum = 0.f;
+            reg_b = bb;
+          }
+          reg_sum += g * g;
+        }
+      }
     }
   }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-  if (lane == 0) {
-    const float z = acc + bias;
-    logits[token] = z;
-    if (sum_sq != nullptr) {
-      const float g = 1.0f / (1.0f + __expf(-z));
-      atomicAdd(&sum_sq[token / L], g * g);
-    }
-  }
+  if (sum_sq != nullptr && lane == 0 && t_end > t_begin) atomicAdd(&sum_sq[reg_b], reg_sum);
 }
 
 }  // namespace
 
 cudaError_t launch_router_logits(const bf16* S, const float* w, float bias, float* logits, float* sum_sq, int B, int L,
                                  int row_elems, cudaStream_t stream) {
-  const int64_t threads = (int64_t)B * L * 32;
-  router_logits_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(S, w, bias, logits, sum_sq, B, L, row_elems);
+  int device = 0, sms = 148;
+  if (cudaGetDevice(&device) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+  int per_sm = 0;   // one resident wave: every CTA of the grid runs at once and owns an equal share
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, router_logits_kernel, 256, 0) != cudaSuccess || per_sm < 1)
+    per_sm = 1;
+  int64_t blocks = (int64_t)sms * per_sm;
+  const int64_t max_blocks = ((int64_t)B * L + 8 * kRlTokens - 1) / (8 * kRlTokens);
+  if (blocks > max_blocks) blocks = max_blocks;
+  router_logits_kernel<<<(unsigned)blocks, 256, 0, stream>>>(S, w, bias, logits, sum_sq, B, L, row_elems);
   return cudaGetLastError();
 }
 
