@@ -40,52 +40,77 @@ __device__ long long g_trace[4][8192];
 #endif
 
 // ------------------------------------------------------------------------------------------------
-// Delta / dgate preprocess: one warp per (b, t), looping over heads.
+// Delta / dgate preprocess.  The grid is one resident wave; every warp owns a contiguous range of tokens.  A token's
+// Hq*D values are read with 16-byte loads: D/8 lanes per head, 32/(D/8) heads per pass, several passes in flight.
+__device__ __forceinline__ float dot8(const uint4& x, const uint4& y) {
+  const uint32_t a[4] = {x.x, x.y, x.z, x.w}, b[4] = {y.x, y.y, y.z, y.w};
+  float acc = 0.f;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    acc = fmaf(__uint_as_float(a[k] << 16), __uint_as_float(b[k] << 16), acc);
+    acc = fmaf(__uint_as_float(a[k] & 0xffff0000u), __uint_as_float(b[k] & 0xffff0000u), acc);
+  }
+  return acc;
+}
+
+template <int D>
 __global__ void __launch_bounds__(256) bwd_delta_kernel(const bf16* __restrict__ dO, const bf16* __restrict__ dO_loc,
                                                         const bf16* __restrict__ S,
                                                         const bf16* __restrict__ A_c,
                                                         const uint8_t* __restrict__ d_mask,
                                                         const int32_t* __restrict__ prefix, float* __restrict__ delta_loc,
                                                         float* __restrict__ delta_glb, float* __restrict__ dgate, int B,
-                                                        int L, int Hq, int D, int a_by_row) {
-  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (warp >= B * L) return;
-  const int b = warp / L, t = warp % L;
-  const bool routed = d_mask[(int64_t)b * L + t] != 0;
-  const int c = routed ? prefix[(int64_t)b * (L + 1) + t] : 0;
-  const int64_t row = ((int64_t)b * L + t) * Hq * D;
-  // a_by_row: the global output was computed for every token and A is indexed by row (forced-global iterations)
-  const int64_t crow = ((int64_t)b * L + (a_by_row ? t : c)) * Hq * D;
-  const int per_lane = D / 32;  // 2 or 4 elements
-  float gate = 0.f;
-  for (int h = 0; h < Hq; ++h) {
-    float dl = 0.f, dg = 0.f;
-    const bf16* po = dO + row + (int64_t)h * D + lane * per_lane;
-    const bf16* pl = dO_loc + row + (int64_t)h * D + lane * per_lane;   // gradient of s_t (== dO unless split)
-    const bf16* ps = S + row + (int64_t)h * D + lane * per_lane;
-    const bf16* pa = A_c + crow + (int64_t)h * D + lane * per_lane;
-    for (int e = 0; e < per_lane; e += 2) {
-      const float2 o2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(po + e));
-      const float2 s2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(ps + e));
-      const float2 l2 = dO_loc == dO ? o2 : __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(pl + e));
-      dl += l2.x * s2.x + l2.y * s2.y;
-      if (routed || a_by_row) {
-        const float2 a2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(pa + e));
-        dg += o2.x * a2.x + o2.y * a2.y;
+                                                        int L, int Hq, int a_by_row) {
+  constexpr int kLanesPerHead = D / 8;                 // 16-byte chunks per head row
+  constexpr int kHeadsPerPass = 32 / kLanesPerHead;
+  const int lane = threadIdx.x & 31;
+  const int64_t n_tokens = (int64_t)B * L;
+  const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+  const int64_t gw = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int64_t t_begin = n_tokens * gw / n_warps, t_end = n_tokens * (gw + 1) / n_warps;
+  const bool split = dO_loc != dO;                     // separate gradient for the local output
+  const int sub = lane / kLanesPerHead;                // head inside the pass
+  const int n_pass = (Hq + kHeadsPerPass - 1) / kHeadsPerPass;
+  for (int64_t token = t_begin; token < t_end; ++token) {
+    const int b = (int)(token / L), t = (int)(token % L);
+    const bool routed = d_mask[token] != 0;
+    const int c = routed ? prefix[(int64_t)b * (L + 1) + t] : 0;
+    // a_by_row: the global output was computed for every token and A is indexed by row (forced-global iterations)
+    const bool with_a = routed || a_by_row;
+    const int64_t row = token * Hq * D;
+    const int64_t crow = ((int64_t)b * L + (a_by_row ? t : c)) * Hq * D;
+    const uint4* po = reinterpret_cast<const uint4*>(dO + row) + lane;
+    const uint4* pl = reinterpret_cast<const uint4*>(dO_loc + row) + lane;
+    const uint4* ps = reinterpret_cast<const uint4*>(S + row) + lane;
+    const uint4* pa = reinterpret_cast<const uint4*>(A_c + crow) + lane;
+    float gate = 0.f;
+#pragma unroll 4
+    for (int p = 0; p < n_pass; ++p) {
+      const int h = p * kHeadsPerPass + sub;
+      float dl = 0.f, dg = 0.f;
+      if (h < Hq) {
+        const uint4 o = __ldg(po + p * 32);
+        const uint4 sv = __ldg(ps + p * 32);
+        dl = dot8(split ? __ldg(pl + p * 32) : o, sv);
+        if (with_a) dg = dot8(o, __ldg(pa + p * 32));
+      }
+#pragma unroll
+      for (int off = kLanesPerHead / 2; off > 0; off >>= 1) {
+        dl += __shfl_xor_sync(0xffffffffu, dl, off);
+        dg += __shfl_xor_sync(0xffffffffu, dg, off);
+      }
+      if (h < Hq && (lane % kLanesPerHead) == 0) {
+        delta_loc[((int64_t)b * Hq + h) * L + t] = dl;
+        if (routed) delta_glb[((int64_t)b * Hq + h) * L + c] = dg;
+        gate += dg;
       }
     }
+    if (dgate != nullptr) {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      dl += __shfl_xor_sync(0xffffffffu, dl, o);
-      dg += __shfl_xor_sync(0xffffffffu, dg, o);
+      for (int off = 16; off >= kLanesPerHead; off >>= 1) gate += __shfl_xor_sync(0xffffffffu, gate, off);
+      if (lane == 0) dgate[token] = with_a ? gate : 0.f;
     }
-    if (lane == 0) {
-      delta_loc[((int64_t)b * Hq + h) * L + t] = dl;
-      if (routed) delta_glb[((int64_t)b * Hq + h) * L + c] = dg;
-    }
-    gate += dg;
   }
-  if (dgate != nullptr && lane == 0) dgate[(int64_t)b * L + t] = (routed || a_by_row) ? gate : 0.f;
 }
 
 // lse by row -> lse by compact row (forced-global iterations store the global log-sum-exp for every row)
@@ -955,12 +980,18 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
     return L2A_ERR_CUDA;
   pe.mark(s);
   {
-    const int64_t warps = (int64_t)p->B * p->Lq;
-    const unsigned blocks = (unsigned)((warps * 32 + 255) / 256);
-    bwd_delta_kernel<<<blocks, 256, 0, s>>>(static_cast<const bf16*>(dO), static_cast<const bf16*>(dS_loc),
-                                            static_cast<const bf16*>(S_save),
-                                            static_cast<const bf16*>(A_c), d_mask, prefix, delta_loc, delta_glb, dgate,
-                                            p->B, p->Lq, p->Hq, p->D, force_all ? 1 : 0);
+    // one resident wave of 8-warp CTAs, each warp with an equal contiguous share of the tokens
+    int device = 0, sms = 148, per_sm = 0;
+    if (cudaGetDevice(&device) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    auto kern = p->D == 128 ? bwd_delta_kernel<128> : bwd_delta_kernel<64>;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 256, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+    int64_t blocks = (int64_t)sms * per_sm;
+    const int64_t max_blocks = ((int64_t)p->B * p->Lq + 7) / 8;
+    if (blocks > max_blocks) blocks = max_blocks;
+    kern<<<(unsigned)blocks, 256, 0, s>>>(static_cast<const bf16*>(dO), static_cast<const bf16*>(dS_loc),
+                                          static_cast<const bf16*>(S_save), static_cast<const bf16*>(A_c), d_mask,
+                                          prefix, delta_loc, delta_glb, dgate, p->B, p->Lq, p->Hq,
+                                          force_all ? 1 : 0);
     if (cudaGetLastError() != cudaSuccess) return L2A_ERR_CUDA;
     if (force_all) {
       dim3 grid((p->Lq + 255) / 256, p->Hq, p->B);
