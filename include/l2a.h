@@ -46,9 +46,11 @@ typedef enum {
 
 /* l2a_params.flags */
 #define L2A_FLAG_SAVE_FOR_BWD 1u  /* forward also writes S_save and A_c (needed by l2a_backward)  */
-#define L2A_FLAG_SKIP_LOCAL 2u    /* forward: no local module; O = d * A (the "SWA-0" ablation)   */
+#define L2A_FLAG_SKIP_LOCAL 2u    /* forward: no local module; O = d * A (the "SWA-0" ablation).   */
+                                  /* backward: gradients of the Global Attention module only       */
 #define L2A_FLAG_SKIP_GLOBAL 4u   /* forward: local module only; O = S (first phase of the layer, */
-                                  /* before the router has seen S)                                */
+                                  /* before the router has seen S).  backward: gradients of the   */
+                                  /* Local Attention module only                                  */
 #define L2A_FLAG_GLOBAL_PHASE 16u  /* forward: second phase of the layer.  O (and S_save) already hold   */
                                   /* the local output from an earlier L2A_FLAG_SKIP_GLOBAL call; only  */
                                   /* the routed rows' global attention runs and is added into O.       */
@@ -168,6 +170,13 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
  * the local part is a sliding-window attention backward).  With one Q/K/V set feeding both
  * modules, dQ_t = dQ_loc,t + d_t * dQ_glb,t and dK, dV sum both modules' contributions and the
  * query heads of each KV group.
+ *
+ * When the Global Attention module has its own Q/K/V (its own projections of s_t, Section 3.1), the layer is two
+ * calls each way: forward L2A_FLAG_SKIP_GLOBAL with the local set, then L2A_FLAG_GLOBAL_PHASE with the global
+ * set; backward L2A_FLAG_SKIP_GLOBAL with the local set (gradients of Q, K, V; d_mask, q_idx, n_routed, prefix,
+ * A_c, lse_glb may be NULL) and L2A_FLAG_SKIP_LOCAL with the global set (dQ is zero outside the routed rows;
+ * S_save, lse_loc may be NULL).  Both skip flags at once, or either with L2A_FLAG_FORCE_ALL_GLOBAL, is
+ * L2A_ERR_INVALID_ARG.
  *
  *   Q, K, V, d_mask, q_idx, n_routed, prefix : as given to l2a_forward.
  *   dO          in : bf16 [B, Lq, Hq, D], gradient of the loss w.r.t. O.

@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const bf16* __restrict__
   const int n_pass = (Hq + kHeadsPerPass - 1) / kHeadsPerPass;
   for (int64_t token = t_begin; token < t_end; ++token) {
     const int b = (int)(token / L), t = (int)(token % L);
-    const bool routed = d_mask[token] != 0;
+    const bool routed = d_mask != nullptr && d_mask[token] != 0;     // NULL: the global part is skipped
     const int c = routed ? prefix[(int64_t)b * (L + 1) + t] : 0;
     // a_by_row: the global output was computed for every token and A is indexed by row (forced-global iterations)
     const bool with_a = routed || a_by_row;
@@ -90,8 +90,7 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const bf16* __restrict__
       float dl = 0.f, dg = 0.f;
       if (h < Hq) {
         const uint4 o = __ldg(po + p * 32);
-        const uint4 sv = __ldg(ps + p * 32);
-        dl = dot8(split ? __ldg(pl + p * 32) : o, sv);
+        if (S != nullptr) dl = dot8(split ? __ldg(pl + p * 32) : o, __ldg(ps + p * 32));   // NULL: local part skipped
         if (with_a) dg = dot8(o, __ldg(pa + p * 32));
       }
 #pragma unroll
@@ -100,7 +99,7 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const bf16* __restrict__
         dg += __shfl_xor_sync(0xffffffffu, dg, off);
       }
       if (h < Hq && (lane % kLanesPerHead) == 0) {
-        delta_loc[((int64_t)b * Hq + h) * L + t] = dl;
+        if (S != nullptr) delta_loc[((int64_t)b * Hq + h) * L + t] = dl;
         if (routed) delta_glb[((int64_t)b * Hq + h) * L + c] = dg;
         gate += dg;
       }
@@ -131,6 +130,7 @@ struct BwdArgs {
   int window, q_pos_offset;
   float scale, scale_log2;
   int global_mode;  // dq kernel only
+  int skip_local, skip_global;   // gradients of one module only (the other module has its own Q/K/V)
   const int32_t* q_idx;
   const int32_t* n_routed;
   const int32_t* prefix;
@@ -483,10 +483,10 @@ __device__ __forceinline__ ItemPlan make_plan(const BwdArgs& a, int b, int k0) {
   const long long tmax_ll = (long long)k0 + kTileN - 1 + a.window - a.q_pos_offset;
   int tmax = tmax_ll > a.Lq - 1 ? a.Lq - 1 : (int)tmax_ll;
   if (tmin < 0) tmin = 0;
-  if (tmax < tmin) { p.loc_t0 = 0; p.loc_nt = 0; }
+  if (tmax < tmin || a.skip_local) { p.loc_t0 = 0; p.loc_nt = 0; }
   else { p.loc_t0 = tmin / kTileM; p.loc_nt = tmax / kTileM - p.loc_t0 + 1; }
   // global: compact rows whose position is >= k0
-  const int n_c = a.n_routed[b];
+  const int n_c = a.skip_global ? 0 : a.n_routed[b];
   if (tmin > a.Lq - 1 || n_c == 0) { p.glb_t0 = 0; p.glb_nt = 0; }
   else {
     const int c_min = a.prefix[(int64_t)b * (a.Lq + 1) + tmin];
@@ -525,7 +525,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   const int G = a.Hq / a.Hkv;
   const int k0 = j * kTileN;
   const ItemPlan plan = make_plan(a, b, k0);
-  const int n_c = a.n_routed[b];
+  const int n_c = a.skip_global ? 0 : a.n_routed[b];   // the routing arrays may be NULL when the global part is skipped
 
   extern __shared__ __align__(1024) uint8_t smem[];
   uint8_t* sK = smem + SM::kKOff;
@@ -901,10 +901,17 @@ cudaError_t launch_bwd_kernels(const BwdArgs& base, const CUtensorMap& mapQ, con
   const unsigned n_tiles = (base.Lq + kTileM - 1) / kTileM;
   BwdArgs a = base;
   a.global_mode = 0;
-  bwd_dq_kernel<D><<<n_tiles * base.B * base.Hq, kDqThreads, DqSmem<D>::kTotal, s>>>(mapQ, mapDO, mapK, mapV, a);
+  if (!base.skip_local) {
+    bwd_dq_kernel<D><<<n_tiles * base.B * base.Hq, kDqThreads, DqSmem<D>::kTotal, s>>>(mapQ, mapDO, mapK, mapV, a);
+  } else {
+    // the global launch adds into dQ at the routed positions: every other row of dQ is zero
+    e = cudaMemsetAsync(base.dQ, 0, (size_t)base.B * base.Lq * base.Hq * D * sizeof(bf16), s);
+    if (e != cudaSuccess) return e;
+  }
   phase_events().mark(s);
   a.global_mode = 1;
-  bwd_dq_kernel<D><<<n_tiles * base.B * base.Hq, kDqThreads, DqSmem<D>::kTotal, s>>>(mapQc, mapDOc, mapK, mapV, a);
+  if (!base.skip_global)
+    bwd_dq_kernel<D><<<n_tiles * base.B * base.Hq, kDqThreads, DqSmem<D>::kTotal, s>>>(mapQc, mapDOc, mapK, mapV, a);
   phase_events().mark(s);
   return cudaGetLastError();
 }
@@ -943,11 +950,13 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   size_t need = 0;
   l2a_status st = l2a_workspace_bytes(p, nullptr, nullptr, &need);
   if (st != L2A_OK) return st;
-  if (p->flags & (L2A_FLAG_SKIP_LOCAL | L2A_FLAG_SKIP_GLOBAL)) return L2A_ERR_UNSUPPORTED;
+  const bool skip_local = p->flags & L2A_FLAG_SKIP_LOCAL, skip_global = p->flags & L2A_FLAG_SKIP_GLOBAL;
+  if (skip_local && skip_global) return L2A_ERR_INVALID_ARG;
   const bool force_all = p->flags & L2A_FLAG_FORCE_ALL_GLOBAL;
-  if (!Q || !K || !V || !d_mask || !q_idx || !n_routed || !prefix || !dO || !S_save || !A_c || !lse_loc || !lse_glb ||
-      !dQ || !dK || !dV)
-    return L2A_ERR_INVALID_ARG;
+  if (!Q || !K || !V || !dO || !dQ || !dK || !dV) return L2A_ERR_INVALID_ARG;
+  if (!skip_global && (!d_mask || !q_idx || !n_routed || !prefix || !A_c || !lse_glb)) return L2A_ERR_INVALID_ARG;
+  if (!skip_local && (!S_save || !lse_loc)) return L2A_ERR_INVALID_ARG;
+  if (force_all && (skip_local || skip_global)) return L2A_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(dO) || !aligned16(S_save) || !aligned16(A_c) ||
       !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
     return L2A_ERR_INVALID_ARG;
@@ -973,11 +982,14 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   PhaseEvents& pe = phase_events();
   struct ClearOnExit { PhaseEvents& p; ~ClearOnExit() { p.clear(); } } clear_on_exit{pe};
   pe.mark(s);
-  if (launch_gather_rows(static_cast<const bf16*>(Q), Qc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s) != cudaSuccess)
-    return L2A_ERR_CUDA;
-  if (launch_gather_rows(static_cast<const bf16*>(dO), dOc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s) !=
-      cudaSuccess)
-    return L2A_ERR_CUDA;
+  if (!skip_global) {
+    if (launch_gather_rows(static_cast<const bf16*>(Q), Qc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s) !=
+        cudaSuccess)
+      return L2A_ERR_CUDA;
+    if (launch_gather_rows(static_cast<const bf16*>(dO), dOc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s) !=
+        cudaSuccess)
+      return L2A_ERR_CUDA;
+  }
   pe.mark(s);
   {
     // one resident wave of 8-warp CTAs, each warp with an equal contiguous share of the tokens
@@ -989,8 +1001,9 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
     const int64_t max_blocks = ((int64_t)p->B * p->Lq + 7) / 8;
     if (blocks > max_blocks) blocks = max_blocks;
     kern<<<(unsigned)blocks, 256, 0, s>>>(static_cast<const bf16*>(dO), static_cast<const bf16*>(dS_loc),
-                                          static_cast<const bf16*>(S_save), static_cast<const bf16*>(A_c), d_mask,
-                                          prefix, delta_loc, delta_glb, dgate, p->B, p->Lq, p->Hq,
+                                          static_cast<const bf16*>(skip_local ? nullptr : S_save),
+                                          static_cast<const bf16*>(A_c), skip_global ? nullptr : d_mask, prefix,
+                                          delta_loc, delta_glb, dgate, p->B, p->Lq, p->Hq,
                                           force_all ? 1 : 0);
     if (cudaGetLastError() != cudaSuccess) return L2A_ERR_CUDA;
     if (force_all) {
@@ -1007,6 +1020,8 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   a.scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->D);
   a.scale_log2 = a.scale * kLog2e;
   a.global_mode = 0;
+  a.skip_local = skip_local ? 1 : 0;
+  a.skip_global = skip_global ? 1 : 0;
   a.q_idx = q_idx; a.n_routed = n_routed; a.prefix = prefix;
   a.lse_loc = lse_loc; a.lse_glb = force_all ? lse_c : lse_glb; a.delta_loc = delta_loc; a.delta_glb = delta_glb;
   a.dQ = static_cast<bf16*>(dQ); a.dK = static_cast<bf16*>(dK); a.dV = static_cast<bf16*>(dV);
