@@ -81,3 +81,21 @@ def test_decode_pruned_layer_ring_cache():
     l2a.l2a_decode(p, t["Q"].cuda(), Kr, Vr, None, O, ws)
     torch.cuda.synchronize()
     check_close(to_f64(O), ref["s"], "decode over a ring-buffer local cache")
+
+
+def test_decode_full_size_cache():
+    """The benchmark's decode configuration (128K-token cache, 32/8 heads, 2048-key chunks): a decode step is a
+    single query row per sequence, so the oracle computes every output element."""
+    cfg = synth.CONFIGS["qwen3_8b_128k"]
+    B, Lk = 2, cfg.L
+    t = synth.qkv(B, 1, cfg.Hq, cfg.Hkv, cfg.D, seed=2024, Lk=Lk)
+    d = np.array([[1], [0]], dtype=np.uint8)
+    p = l2a.params(B, 1, Lk, cfg.Hq, cfg.Hkv, cfg.D, cfg.W)
+    ws = torch.empty(l2a.l2a_decode_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    O = torch.full((B, 1, cfg.Hq, cfg.D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    l2a.l2a_decode(p, t["Q"].cuda(), t["K"].cuda(), t["V"].cuda(), torch.from_numpy(d[:, 0].copy()).cuda(), O, ws)
+    torch.cuda.synchronize()
+    assert l2a.l2a_workspace_status(ws) == 0
+    sh = oracle.Shape(B, 1, Lk, cfg.Hq, cfg.Hkv, cfg.D, cfg.W)
+    ref = oracle.forward_full(sh, synth.as_u16(t["Q"]), synth.as_u16(t["K"]), synth.as_u16(t["V"]), d)
+    check_close(to_f64(O), ref["o"], "decode O at 128K")
