@@ -29,6 +29,9 @@ constexpr int kBoxBytes = 128 * 128;
 constexpr float kLog2e = 1.4426950408889634f;
 
 // Optional per-role clock tracing of one CTA of the dK/dV kernel (development builds only: -DL2A_TRACE=<block>).
+#ifndef L2A_TRACE_WARP
+#define L2A_TRACE_WARP 0   // the compute warp whose phases are recorded
+#endif
 #ifdef L2A_TRACE
 __device__ long long g_trace[4][8192];
 #define L2A_TRACE_POINT(role, idx)                                                              \
@@ -305,28 +308,28 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
                  (kk > 0 || it > 0) ? 1u : 0u, leader);
         tc_commit(&bar->k_empty[it % 3], leader);
       };
-      bool ok = mbar_wait_warp(&bar->q_full, 0, abort_flag) && mbar_wait_warp(&bar->k_full[0], 0, abort_flag) &&
-                mbar_wait_warp(&bar->v_full[0], 0, abort_flag);
+      bool ok = mbar_spin_warp(&bar->q_full, 0, abort_flag) && mbar_spin_warp(&bar->k_full[0], 0, abort_flag) &&
+                mbar_spin_warp(&bar->v_full[0], 0, abort_flag);
       if (ok) {
         tc_fence_after();
         issue_S(0);
         issue_dP(0);
         if (n_blocks > 1) {
-          ok = mbar_wait_warp(&bar->k_full[1], 0, abort_flag);
+          ok = mbar_spin_warp(&bar->k_full[1], 0, abort_flag);
           if (ok) { tc_fence_after(); issue_S(1); }
         }
       }
       for (int it = 0; ok && it < n_blocks; ++it) {
-        if (!mbar_wait_warp(&bar->ds_full, it & 1, abort_flag)) { ok = false; break; }
+        if (!mbar_spin_warp(&bar->ds_full, it & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         issue_dQ(it);
         if (it + 1 < n_blocks) {
-          if (!mbar_wait_warp(&bar->v_full[(it + 1) & 1], ((it + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+          if (!mbar_spin_warp(&bar->v_full[(it + 1) & 1], ((it + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
           issue_dP(it + 1);
         }
         if (it + 2 < n_blocks) {
-          if (!mbar_wait_warp(&bar->k_full[(it + 2) % 3], ((it + 2) / 3) & 1, abort_flag)) { ok = false; break; }
+          if (!mbar_spin_warp(&bar->k_full[(it + 2) % 3], ((it + 2) / 3) & 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
           issue_S(it + 2);
         }
@@ -703,8 +706,8 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
                  (kk > 0 || !first) ? 1u : 0u, leader);
         tc_commit(&bar->q_empty[qs], leader);
       };
-      bool ok = mbar_wait_warp(&bar->kv_full, 0, abort_flag) && mbar_wait_warp(&bar->q_full[0], 0, abort_flag) &&
-                mbar_wait_warp(&bar->do_full[0], 0, abort_flag);
+      bool ok = mbar_spin_warp(&bar->kv_full, 0, abort_flag) && mbar_spin_warp(&bar->q_full[0], 0, abort_flag) &&
+                mbar_spin_warp(&bar->do_full[0], 0, abort_flag);
       if (ok) {
         tc_fence_after();
         issue_S(0);
@@ -717,23 +720,23 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         int qn = qs + 1;
         uint32_t qphn = qph;
         if (qn == 3) { qn = 0; qphn ^= 1; }
-        if (!mbar_wait_warp(&bar->p_full, i & 1, abort_flag)) { ok = false; break; }
+        if (!mbar_spin_warp(&bar->p_full, i & 1, abort_flag)) { ok = false; break; }
         if (lane == 0) L2A_TRACE_POINT(0, 4 * i);
         tc_fence_after();
         issue_dV(i & 1, i == 0);
         if (lane == 0) L2A_TRACE_POINT(2, 4 * i + 3);
         if (more) {
-          if (!mbar_wait_warp(&bar->q_full[qn], qphn, abort_flag)) { ok = false; break; }
+          if (!mbar_spin_warp(&bar->q_full[qn], qphn, abort_flag)) { ok = false; break; }
           if (lane == 0) L2A_TRACE_POINT(0, 4 * i + 1);
           tc_fence_after();
           issue_S(qn);
         }
-        if (!mbar_wait_warp(&bar->ds_full, i & 1, abort_flag)) { ok = false; break; }
+        if (!mbar_spin_warp(&bar->ds_full, i & 1, abort_flag)) { ok = false; break; }
         if (lane == 0) L2A_TRACE_POINT(0, 4 * i + 2);
         tc_fence_after();
         issue_dK(qs, i == 0);
         if (more) {
-          if (!mbar_wait_warp(&bar->do_full[(i + 1) & 1], ((i + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+          if (!mbar_spin_warp(&bar->do_full[(i + 1) & 1], ((i + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
           issue_dP((i + 1) & 1);
         }
@@ -767,14 +770,14 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       }
       const bool masked = st_flags[q] != 0;
       if (!__all_sync(0xffffffffu, mbar_wait(&bar->s_full, i & 1, abort_flag))) { ok = false; break; }
-      if (warp == 0 && lane == 0) L2A_TRACE_POINT(1, 4 * i);
+      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_POINT(1, 4 * i);
       tc_fence_after();
       uint32_t pp[16];
       {
         uint32_t sv[32];
         tmem_ld32(s_addr, sv);
         tmem_ld_wait();
-        if (warp == 0 && lane == 0) L2A_TRACE_POINT(2, 4 * i);
+        if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_POINT(2, 4 * i);
         // the element mask is needed only for the few tiles that straddle the causal diagonal or a window edge:
         // two loop versions, so that the common one has no branches
         if (!masked) {
@@ -805,13 +808,13 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           }
         }
       }
-      if (warp == 0 && lane == 0) L2A_TRACE_POINT(2, 4 * i + 1);
+      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_POINT(2, 4 * i + 1);
       tmem_st16(s_addr, pp);     // P^T over the first half of this quarter's own S^T columns
       tmem_st_wait();
-      if (warp == 0 && lane == 0) L2A_TRACE_POINT(2, 4 * i + 2);
+      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_POINT(2, 4 * i + 2);
       tc_fence_before();
       mbar_arrive(&bar->p_full);
-      if (warp == 0 && lane == 0) L2A_TRACE_POINT(1, 4 * i + 1);
+      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_POINT(1, 4 * i + 1);
       // Delta of the same rows, again ahead of the wait; after this the statistics slot may be refilled
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
@@ -820,7 +823,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       }
       mbar_arrive(&bar->st_empty[s]);
       if (!__all_sync(0xffffffffu, mbar_wait(&bar->dp_full, i & 1, abort_flag))) { ok = false; break; }
-      if (warp == 0 && lane == 0) L2A_TRACE_POINT(1, 4 * i + 2);
+      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_POINT(1, 4 * i + 2);
       tc_fence_after();
       uint32_t pd[16];
       {
@@ -840,7 +843,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(&bar->ds_full);
-      if (warp == 0 && lane == 0) L2A_TRACE_POINT(1, 4 * i + 3);
+      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_POINT(1, 4 * i + 3);
     }
     // epilogue: quarters 0,1 store the two column halves of dV, quarters 2,3 those of dK
     if (ok && __all_sync(0xffffffffu, mbar_wait(&bar->final_bar, 0, abort_flag))) {

@@ -218,11 +218,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       auto in_range = [&](int t, int j) { return t ? (j >= lo1 && j <= hi1) : (j >= lo0 && j <= hi0); };
 
       // first key block: Q*K^T for both tiles
-      if (!mbar_wait_warp(&bar->k_full[0], 0, abort_flag)) ok = false;
+      if (!mbar_spin_warp(&bar->k_full[0], 0, abort_flag)) ok = false;
 #pragma unroll
       for (int t = 0; t < kNumTiles; ++t) {
         if (ok && in_range(t, jlo)) {
-          if (!mbar_wait_warp(&bar->q_full[t], 0, abort_flag)) { ok = false; }
+          if (!mbar_spin_warp(&bar->q_full[t], 0, abort_flag)) { ok = false; }
           else { tc_fence_after(); issue_qk(t, 0); }
         }
       }
@@ -237,11 +237,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         for (int t = 0; t < kNumTiles; ++t) {
           if (ok && in_range(t, j)) {
             uint32_t& pc = t ? p_cnt1 : p_cnt0;
-            if (!mbar_wait_warp(&bar->p_full[t], pc & 1, abort_flag)) { ok = false; }
+            if (!mbar_spin_warp(&bar->p_full[t], pc & 1, abort_flag)) { ok = false; }
             else {
               ++pc;
               if (!v_ready) {
-                if (!mbar_wait_warp(&bar->v_full[s], ph, abort_flag)) ok = false;
+                if (!mbar_spin_warp(&bar->v_full[s], ph, abort_flag)) ok = false;
                 v_ready = true;
               }
               if (ok) {
@@ -252,10 +252,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
           }
           if (ok && j + 1 <= jhi && in_range(t, j + 1)) {
             if (!k_ready) {
-              if (!mbar_wait_warp(&bar->k_full[sn], phn, abort_flag)) ok = false;
+              if (!mbar_spin_warp(&bar->k_full[sn], phn, abort_flag)) ok = false;
               k_ready = true;
             }
-            if (ok && j + 1 == (t ? lo1 : lo0) && !mbar_wait_warp(&bar->q_full[t], 0, abort_flag)) ok = false;
+            if (ok && j + 1 == (t ? lo1 : lo0) && !mbar_spin_warp(&bar->q_full[t], 0, abort_flag)) ok = false;
             if (ok) {
               tc_fence_after();
               issue_qk(t, sn);
@@ -264,10 +264,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         }
         if (!ok) break;
         // V block j is released once both tiles' P*V have drained; K block j+1 once both Q*K^T have
-        if (!v_ready && !mbar_wait_warp(&bar->v_full[s], ph, abort_flag)) break;
+        if (!v_ready && !mbar_spin_warp(&bar->v_full[s], ph, abort_flag)) break;
         tc_commit(&bar->v_empty[s], leader);
         if (j + 1 <= jhi) {
-          if (!k_ready && !mbar_wait_warp(&bar->k_full[sn], phn, abort_flag)) break;
+          if (!k_ready && !mbar_spin_warp(&bar->k_full[sn], phn, abort_flag)) break;
           tc_commit(&bar->k_empty[sn], leader);
         }
       }

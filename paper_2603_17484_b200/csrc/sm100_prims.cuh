@@ -107,6 +107,35 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return true;
 }
 
+// Polling wait (mbarrier.test_wait never suspends the thread): lowest wake-up latency, for a single warp whose
+// reaction time is on the critical path.  Bounded like mbar_wait.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_spin_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  bool done = mbar_test_wait(bar, parity);
+  if (!__all_sync(0xffffffffu, done)) {
+    const uint64_t t0 = globaltimer_ns();
+    uint32_t spins = 0;
+    while (!__all_sync(0xffffffffu, done = mbar_test_wait(bar, parity))) {
+      if ((++spins & 0x3ffu) == 0) {
+        if (*abort_flag) return false;
+        if (globaltimer_ns() - t0 > kWaitLimitNs) {
+          *abort_flag = 1;
+          return false;
+        }
+      }
+    }
+  }
+  return true;
+}
+
 // whole-warp wait with a warp-uniform outcome (all 32 lanes must call it)
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
