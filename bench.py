@@ -30,7 +30,7 @@ from paper_2603_17484_b200 import replicas, synth  # noqa: E402
 METRIC = "L2A fwd+bwd useful TFLOP/s at 128K (one layer, one GPU)"
 KERNELS_PER_STEP = 11  # route: count, scan | fwd: gather, local, global | bwd: gather x2, delta, dkv, dq x2
 FWD_PHASES = ("gather_q", "attn_fwd_local", "attn_fwd_global")
-BWD_PHASES = ("gather_q_dO", "bwd_delta", "bwd_dkv", "bwd_dq_local", "bwd_dq_global")
+BWD_PHASES = ("gather_q_dO", "bwd_delta", "bwd_dq_local", "bwd_dq_global", "bwd_dkv")
 
 
 def measured_peaks():

@@ -342,8 +342,8 @@ l2a_status l2a_route_compact_static(const l2a_params* p, const void* router, int
  * k-th phase boundary and then clears the registration.  Phase boundaries:
  *   l2a_forward : 0 start | 1 after the query gather | 2 after the local kernel | 3 after the
  *                 global kernel
- *   l2a_backward: 0 start | 1 after the gathers | 2 after the Delta kernel | 3 after the dK/dV
- *                 kernel | 4 after the local dQ kernel | 5 after the global dQ kernel
+ *   l2a_backward: 0 start | 1 after the gathers | 2 after the Delta kernel | 3 after the local dQ
+ *                 kernel | 4 after the global dQ kernel (dQ is final) | 5 after the dK/dV kernel
  * This is the only per-thread state the library keeps.
  */
 l2a_status l2a_profile_next_call(void* const* events, int n_events);

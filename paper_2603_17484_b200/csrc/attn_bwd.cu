@@ -897,10 +897,8 @@ cudaError_t launch_bwd_kernels(const BwdArgs& base, const CUtensorMap& mapQ, con
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(bwd_dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<D>::kTotal);
   if (e != cudaSuccess) return e;
-  const unsigned n_kblocks = (base.Lk + kTileN - 1) / kTileN;
-  bwd_dkv_kernel<D><<<n_kblocks * base.B * base.Hkv, kDkvThreads, DkvSmem<D>::kTotal, s>>>(mapQ, mapDO, mapQc, mapDOc, mapK,
-                                                                                  mapV, base);
-  phase_events().mark(s);
+  // dQ first: it is the largest result (Hq / Hkv times dK or dV), so a caller that ships results to the host as
+  // they complete can move it while the dK/dV kernel, the longest of the three, is still running
   const unsigned n_tiles = (base.Lq + kTileM - 1) / kTileM;
   BwdArgs a = base;
   a.global_mode = 0;
@@ -915,6 +913,10 @@ cudaError_t launch_bwd_kernels(const BwdArgs& base, const CUtensorMap& mapQ, con
   a.global_mode = 1;
   if (!base.skip_global)
     bwd_dq_kernel<D><<<n_tiles * base.B * base.Hq, kDqThreads, DqSmem<D>::kTotal, s>>>(mapQc, mapDOc, mapK, mapV, a);
+  phase_events().mark(s);
+  const unsigned n_kblocks = (base.Lk + kTileN - 1) / kTileN;
+  bwd_dkv_kernel<D><<<n_kblocks * base.B * base.Hkv, kDkvThreads, DkvSmem<D>::kTotal, s>>>(mapQ, mapDO, mapQc, mapDOc, mapK,
+                                                                                  mapV, base);
   phase_events().mark(s);
   return cudaGetLastError();
 }

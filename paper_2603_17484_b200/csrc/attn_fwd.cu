@@ -87,11 +87,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
   constexpr int kOCol0 = 2 * kTileN;   // first TMEM column of the O accumulators
 
   // ---- work item: heaviest first (largest row index first), heads fastest for K/V reuse in L2
-  const int n_pairs = (a.Lq + kRowsPerCta - 1) / kRowsPerCta;
   const int h = blockIdx.x % a.Hq;
   const int rest = blockIdx.x / a.Hq;
   const int b = rest % a.B;
-  const int pi = n_pairs - 1 - rest / a.B;
+  const int pi = a.pair_end - 1 - rest / a.B;
   const int g = h / (a.Hq / a.Hkv);
   const bool compact = a.global_mode && !a.all_rows;           // rows are compact indices into q_idx
   const int n_rows = compact ? a.n_routed[b] : a.Lq;           // valid (compact) rows of this batch entry
@@ -493,8 +492,8 @@ namespace l2a {
 
 cudaError_t launch_attn_fwd(const FwdArgs& a, const CUtensorMap& mapQ, const CUtensorMap& mapK,
                             const CUtensorMap& mapV, cudaStream_t stream) {
-  const int n_pairs = (a.Lq + kRowsPerCta - 1) / kRowsPerCta;
-  const unsigned grid = (unsigned)n_pairs * a.Hq * a.B;
+  const unsigned grid = (unsigned)(a.pair_end - a.pair_begin) * a.Hq * a.B;
+  if (a.pair_end <= a.pair_begin) return cudaSuccess;
   cudaError_t e;
   if (a.D == 128) {
     e = cudaFuncSetAttribute(attn_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<128>::kTotal);

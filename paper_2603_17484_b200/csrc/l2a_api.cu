@@ -140,9 +140,27 @@ l2a_status l2a_route_compact(const l2a_params* p, const void* router, int router
   return launch_route_compact(a, s) == cudaSuccess ? L2A_OK : L2A_ERR_CUDA;
 }
 
+// l2a_forward over the 256-row query groups [pair_begin, pair_end) (pair_end < 0: all of them).  A proper sub-range
+// is used by l2a_step_host to start Local Attention on the rows whose queries have already arrived; it is only
+// meaningful for the local module (L2A_FLAG_SKIP_GLOBAL), and only the first call of a step clears the status word.
+static l2a_status forward_range(const l2a_params* p, const void* Q, const void* K, const void* V,
+                                const uint8_t* d_mask, const int32_t* q_idx, const int32_t* n_routed,
+                                const int32_t* prefix, void* O, void* S_save, void* A_c, float* lse_loc,
+                                float* lse_glb, void* fwd_ws, size_t fwd_ws_bytes, void* stream, int pair_begin,
+                                int pair_end, bool clear_status);
+
 l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const void* V, const uint8_t* d_mask,
                        const int32_t* q_idx, const int32_t* n_routed, const int32_t* prefix, void* O, void* S_save,
                        void* A_c, float* lse_loc, float* lse_glb, void* fwd_ws, size_t fwd_ws_bytes, void* stream) {
+  return forward_range(p, Q, K, V, d_mask, q_idx, n_routed, prefix, O, S_save, A_c, lse_loc, lse_glb, fwd_ws,
+                       fwd_ws_bytes, stream, 0, -1, true);
+}
+
+static l2a_status forward_range(const l2a_params* p, const void* Q, const void* K, const void* V,
+                                const uint8_t* d_mask, const int32_t* q_idx, const int32_t* n_routed,
+                                const int32_t* prefix, void* O, void* S_save, void* A_c, float* lse_loc,
+                                float* lse_glb, void* fwd_ws, size_t fwd_ws_bytes, void* stream, int pair_begin,
+                                int pair_end, bool clear_status) {
   l2a_status st = check_params(p);
   if (st != L2A_OK) return st;
   const bool save = p->flags & L2A_FLAG_SAVE_FOR_BWD;
@@ -165,7 +183,12 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
   uint8_t* ws = static_cast<uint8_t*>(fwd_ws);
   int* status = reinterpret_cast<int*>(ws);
   bf16* Qc = reinterpret_cast<bf16*>(ws + kWsHeaderBytes);
-  if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, s) != cudaSuccess) return L2A_ERR_CUDA;
+  const int n_pairs = ceil_div(p->Lq, kRowsPerCta);
+  const bool whole = pair_end < 0 || (pair_begin == 0 && pair_end == n_pairs);
+  if (pair_end < 0) pair_end = n_pairs;
+  if (pair_begin < 0 || pair_end > n_pairs || pair_begin > pair_end) return L2A_ERR_INVALID_ARG;
+  if (!whole && !skip_global) return L2A_ERR_INVALID_ARG;
+  if (clear_status && cudaMemsetAsync(ws, 0, kWsHeaderBytes, s) != cudaSuccess) return L2A_ERR_CUDA;
 
   CUtensorMap mapQ, mapK, mapV, mapQc;
   if (!encode_rows_map(&mapQ, Q, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||
@@ -184,6 +207,8 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
   a.status = status;
   a.all_rows = 0;
   a.combine_mask = nullptr;
+  a.pair_begin = 0;
+  a.pair_end = n_pairs;
 
   PhaseEvents& pe = phase_events();
   struct ClearOnExit { PhaseEvents& p; ~ClearOnExit() { p.clear(); } } clear_on_exit{pe};
@@ -201,7 +226,11 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
     a.out = static_cast<bf16*>(save ? S_save : O);
     a.out2 = save ? static_cast<bf16*>(O) : nullptr;
     a.lse = lse_loc;
+    a.pair_begin = pair_begin;
+    a.pair_end = pair_end;
     if (launch_attn_fwd(a, mapQ, mapK, mapV, s) != cudaSuccess) return L2A_ERR_CUDA;
+    a.pair_begin = 0;
+    a.pair_end = n_pairs;
   } else if (skip_local) {
     const size_t bytes = (size_t)p->B * p->Lq * p->Hq * p->D * sizeof(bf16);
     if (cudaMemsetAsync(O, 0, bytes, s) != cudaSuccess) return L2A_ERR_CUDA;  // Algorithm 1: O starts at zero
@@ -318,12 +347,13 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
   const size_t kb = (size_t)p->B * p->Lk * p->Hkv * p->D * sizeof(bf16);
   const size_t rb = (size_t)p->B * p->Lq * (router_kind == L2A_ROUTER_MASK_U8 ? 1 : 4);
   // Two helper streams (created once per host thread and device) overlap the transfers with the kernels:
-  // dO is uploaded while the forward runs, O is downloaded while the backward runs, dK / dV while the dQ
-  // kernels run.  With pageable host memory the copies simply serialise.
+  // dO is uploaded while the forward runs, O is downloaded while the backward runs, dQ while the dK/dV kernel
+  // runs (the backward computes dQ first for this reason); only dK and dV, the small results, leave after the
+  // last kernel.  With pageable host memory the copies simply serialise.
   struct Aux {
     int device = -1;
     cudaStream_t in = nullptr, out = nullptr;
-    cudaEvent_t start = nullptr, up = nullptr, fwd = nullptr, phase[6] = {}, down = nullptr;
+    cudaEvent_t start = nullptr, up = nullptr, fwd = nullptr, phase[6] = {}, down = nullptr, chunk[4] = {};
   };
   static thread_local Aux aux;
   int dev_id = 0;
@@ -333,7 +363,8 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
         cudaStreamCreateWithFlags(&aux.out, cudaStreamNonBlocking) != cudaSuccess)
       return L2A_ERR_CUDA;
     cudaEvent_t* evs[] = {&aux.start, &aux.up, &aux.fwd, &aux.down, &aux.phase[0], &aux.phase[1], &aux.phase[2],
-                          &aux.phase[3], &aux.phase[4], &aux.phase[5]};
+                          &aux.phase[3], &aux.phase[4], &aux.phase[5], &aux.chunk[0], &aux.chunk[1], &aux.chunk[2],
+                          &aux.chunk[3]};
     for (cudaEvent_t* e : evs)
       if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return L2A_ERR_CUDA;
     aux.device = dev_id;
@@ -341,29 +372,77 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
 #define L2A_TRY(x) do { if ((x) != cudaSuccess) return L2A_ERR_CUDA; } while (0)
   L2A_TRY(cudaEventRecord(aux.start, s));
   L2A_TRY(cudaMemcpyAsync(dev->router, host->router, rb, cudaMemcpyHostToDevice, s));
-  L2A_TRY(cudaMemcpyAsync(dev->Q, host->Q, qb, cudaMemcpyHostToDevice, s));
-  L2A_TRY(cudaMemcpyAsync(dev->K, host->K, kb, cudaMemcpyHostToDevice, s));
-  L2A_TRY(cudaMemcpyAsync(dev->V, host->V, kb, cudaMemcpyHostToDevice, s));
-  if (bwd) {   // dO rides the second stream, behind whatever the caller had queued before this call
-    L2A_TRY(cudaStreamWaitEvent(aux.in, aux.start, 0));
-    L2A_TRY(cudaMemcpyAsync(dev->dO, host->dO, qb, cudaMemcpyHostToDevice, aux.in));
-    L2A_TRY(cudaEventRecord(aux.up, aux.in));
-  }
-  st = l2a_route_compact(p, dev->router, router_kind, logit_threshold, dev->d_mask, dev->q_idx, dev->n_routed,
-                         dev->prefix, dev->route_ws, dev->route_ws_bytes, stream);
-  if (st != L2A_OK) return st;
   l2a_params q = *p;
   if (!bwd) q.flags &= ~L2A_FLAG_SAVE_FOR_BWD;
-  st = l2a_forward(&q, dev->Q, dev->K, dev->V, dev->d_mask, dev->q_idx, dev->n_routed, dev->prefix, dev->O,
-                   bwd ? dev->S_save : nullptr, bwd ? dev->A_c : nullptr, bwd ? dev->lse_loc : nullptr,
-                   bwd ? dev->lse_glb : nullptr, dev->fwd_ws, dev->fwd_ws_bytes, stream);
-  if (st != L2A_OK) return st;
+  const int n_pairs = ceil_div(p->Lq, kRowsPerCta);
+  constexpr int kChunks = 4;
+  const bool chunked = p->B == 1 && n_pairs >= 4 * kChunks &&
+                       !(p->flags & (L2A_FLAG_SKIP_LOCAL | L2A_FLAG_SKIP_GLOBAL | L2A_FLAG_GLOBAL_PHASE));
+  if (chunked) {
+    // One sequence: K and V go first, then Q in four row ranges on the upload stream; Local Attention starts on a
+    // range as soon as its queries have landed, so only the first range's copy is exposed.  The global phase
+    // (which needs every query) follows, adding into O exactly as a single l2a_forward call would.
+    L2A_TRY(cudaStreamWaitEvent(aux.in, aux.start, 0));
+    L2A_TRY(cudaMemcpyAsync(dev->K, host->K, kb, cudaMemcpyHostToDevice, aux.in));
+    L2A_TRY(cudaMemcpyAsync(dev->V, host->V, kb, cudaMemcpyHostToDevice, aux.in));
+    const size_t row_bytes = (size_t)p->Hq * p->D * sizeof(bf16);
+    int pair_edge[kChunks + 1];
+    for (int c = 0; c <= kChunks; ++c) pair_edge[c] = (int)((int64_t)n_pairs * c / kChunks);
+    for (int c = 0; c < kChunks; ++c) {
+      const int64_t r0 = (int64_t)pair_edge[c] * kRowsPerCta;
+      int64_t r1 = (int64_t)pair_edge[c + 1] * kRowsPerCta;
+      if (r1 > p->Lq) r1 = p->Lq;
+      L2A_TRY(cudaMemcpyAsync(static_cast<uint8_t*>(dev->Q) + r0 * row_bytes,
+                              static_cast<const uint8_t*>(host->Q) + r0 * row_bytes, (size_t)(r1 - r0) * row_bytes,
+                              cudaMemcpyHostToDevice, aux.in));
+      L2A_TRY(cudaEventRecord(aux.chunk[c], aux.in));
+    }
+    if (bwd) {
+      L2A_TRY(cudaMemcpyAsync(dev->dO, host->dO, qb, cudaMemcpyHostToDevice, aux.in));
+      L2A_TRY(cudaEventRecord(aux.up, aux.in));
+    }
+    st = l2a_route_compact(p, dev->router, router_kind, logit_threshold, dev->d_mask, dev->q_idx, dev->n_routed,
+                           dev->prefix, dev->route_ws, dev->route_ws_bytes, stream);
+    if (st != L2A_OK) return st;
+    l2a_params ql = q;
+    ql.flags = (q.flags & ~L2A_FLAG_FORCE_ALL_GLOBAL) | L2A_FLAG_SKIP_GLOBAL;
+    for (int c = 0; c < kChunks; ++c) {
+      L2A_TRY(cudaStreamWaitEvent(s, aux.chunk[c], 0));
+      st = forward_range(&ql, dev->Q, dev->K, dev->V, dev->d_mask, dev->q_idx, dev->n_routed, dev->prefix, dev->O,
+                         bwd ? dev->S_save : nullptr, bwd ? dev->A_c : nullptr, bwd ? dev->lse_loc : nullptr,
+                         bwd ? dev->lse_glb : nullptr, dev->fwd_ws, dev->fwd_ws_bytes, stream, pair_edge[c],
+                         pair_edge[c + 1], c == 0);
+      if (st != L2A_OK) return st;
+    }
+    l2a_params qg = q;
+    qg.flags |= L2A_FLAG_GLOBAL_PHASE;
+    st = forward_range(&qg, dev->Q, dev->K, dev->V, dev->d_mask, dev->q_idx, dev->n_routed, dev->prefix, dev->O,
+                       bwd ? dev->S_save : nullptr, bwd ? dev->A_c : nullptr, bwd ? dev->lse_loc : nullptr,
+                       bwd ? dev->lse_glb : nullptr, dev->fwd_ws, dev->fwd_ws_bytes, stream, 0, -1, false);
+    if (st != L2A_OK) return st;
+  } else {
+    L2A_TRY(cudaMemcpyAsync(dev->Q, host->Q, qb, cudaMemcpyHostToDevice, s));
+    L2A_TRY(cudaMemcpyAsync(dev->K, host->K, kb, cudaMemcpyHostToDevice, s));
+    L2A_TRY(cudaMemcpyAsync(dev->V, host->V, kb, cudaMemcpyHostToDevice, s));
+    if (bwd) {   // dO rides the second stream, behind whatever the caller had queued before this call
+      L2A_TRY(cudaStreamWaitEvent(aux.in, aux.start, 0));
+      L2A_TRY(cudaMemcpyAsync(dev->dO, host->dO, qb, cudaMemcpyHostToDevice, aux.in));
+      L2A_TRY(cudaEventRecord(aux.up, aux.in));
+    }
+    st = l2a_route_compact(p, dev->router, router_kind, logit_threshold, dev->d_mask, dev->q_idx, dev->n_routed,
+                           dev->prefix, dev->route_ws, dev->route_ws_bytes, stream);
+    if (st != L2A_OK) return st;
+    st = l2a_forward(&q, dev->Q, dev->K, dev->V, dev->d_mask, dev->q_idx, dev->n_routed, dev->prefix, dev->O,
+                     bwd ? dev->S_save : nullptr, bwd ? dev->A_c : nullptr, bwd ? dev->lse_loc : nullptr,
+                     bwd ? dev->lse_glb : nullptr, dev->fwd_ws, dev->fwd_ws_bytes, stream);
+    if (st != L2A_OK) return st;
+  }
   L2A_TRY(cudaEventRecord(aux.fwd, s));
   L2A_TRY(cudaStreamWaitEvent(aux.out, aux.fwd, 0));
   L2A_TRY(cudaMemcpyAsync(host->O, dev->O, qb, cudaMemcpyDeviceToHost, aux.out));
   if (bwd) {
     L2A_TRY(cudaStreamWaitEvent(s, aux.up, 0));
-    // phase boundary 3 of the backward = the dK/dV kernel has finished: its results can leave while dQ is computed
+    // phase boundary 4 of the backward = both dQ kernels have finished: dQ can leave while dK/dV are computed
     void* phase_events[6];
     for (int i = 0; i < 6; ++i) phase_events[i] = aux.phase[i];
     st = l2a_profile_next_call(phase_events, 6);
@@ -372,10 +451,10 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
                       dev->S_save, dev->A_c, dev->lse_loc, dev->lse_glb, dev->dQ, dev->dK, dev->dV, nullptr,
                       dev->bwd_ws, dev->bwd_ws_bytes, stream);
     if (st != L2A_OK) return st;
-    L2A_TRY(cudaStreamWaitEvent(aux.out, aux.phase[3], 0));
-    L2A_TRY(cudaMemcpyAsync(host->dK, dev->dK, kb, cudaMemcpyDeviceToHost, aux.out));
-    L2A_TRY(cudaMemcpyAsync(host->dV, dev->dV, kb, cudaMemcpyDeviceToHost, aux.out));
-    L2A_TRY(cudaMemcpyAsync(host->dQ, dev->dQ, qb, cudaMemcpyDeviceToHost, s));
+    L2A_TRY(cudaStreamWaitEvent(aux.out, aux.phase[4], 0));
+    L2A_TRY(cudaMemcpyAsync(host->dQ, dev->dQ, qb, cudaMemcpyDeviceToHost, aux.out));
+    L2A_TRY(cudaMemcpyAsync(host->dK, dev->dK, kb, cudaMemcpyDeviceToHost, s));
+    L2A_TRY(cudaMemcpyAsync(host->dV, dev->dV, kb, cudaMemcpyDeviceToHost, s));
   }
   L2A_TRY(cudaEventRecord(aux.down, aux.out));
   L2A_TRY(cudaStreamWaitEvent(s, aux.down, 0));   // the caller's stream ends the step with every result delivered

@@ -70,6 +70,7 @@ struct FwdArgs {
   bf16* out2;   // local: optional second copy of s (NULL to skip);  global: O rows, indexed by position
   float* lse;   // local: [B,Hq,Lq] by row;  global: [B,Hq,Lq] by compact row; may be NULL
   int* status;  // workspace status word
+  int pair_begin, pair_end;  // 256-row query groups [pair_begin, pair_end) this launch covers (all: 0 .. ceil(Lq / 256))
 };
 size_t bwd_ws_size(const l2a_params* p);
 

@@ -10,8 +10,9 @@ pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("backward", [False, True])
-def test_step_host_matches_device_calls(backward):
-    B, L, Hq, Hkv, D, W = 2, 1300, 4, 2, 128, 256
+@pytest.mark.parametrize("B,L", [(2, 1300), (1, 4389)])   # one long sequence takes the path that uploads Q in row ranges
+def test_step_host_matches_device_calls(backward, B, L):
+    Hq, Hkv, D, W = 4, 2, 128, 256
     d = synth.mask_bernoulli(B, L, 0.3, seed=17)
     c = Case(B, L, Hq, Hkv, D, W, d, seed=23, backward=backward)
     c.run_forward()
