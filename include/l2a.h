@@ -343,7 +343,9 @@ l2a_status l2a_route_compact_static(const l2a_params* p, const void* router, int
  *   l2a_forward : 0 start | 1 after the query gather | 2 after the local kernel | 3 after the
  *                 global kernel
  *   l2a_backward: 0 start | 1 after the gathers | 2 after the Delta kernel | 3 after the local dQ
- *                 kernel | 4 after the global dQ kernel (dQ is final) | 5 after the dK/dV kernel
+ *                 kernel | 4 after the global dQ kernel (dQ is final) | 5 after the dK/dV kernel.
+ *                 With 7 events the dK/dV kernel runs as two launches (key rows below and from
+ *                 128 * floor(3 * ceil(Lk / 128) / 4), when Lk >= 1024): 5 after the first, 6 after the second
  * This is the only per-thread state the library keeps.
  */
 l2a_status l2a_profile_next_call(void* const* events, int n_events);

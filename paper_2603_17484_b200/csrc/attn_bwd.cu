@@ -134,6 +134,7 @@ struct BwdArgs {
   float scale, scale_log2;
   int global_mode;  // dq kernel only
   int skip_local, skip_global;   // gradients of one module only (the other module has its own Q/K/V)
+  int kb_begin, kb_count;        // dK/dV kernel: key blocks [kb_begin, kb_begin + kb_count) of every KV head
   const int32_t* q_idx;
   const int32_t* n_routed;
   const int32_t* prefix;
@@ -521,8 +522,8 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   const int n_kblocks = (a.Lk + kTileN - 1) / kTileN;
   // key blocks ascending (most work first) inside one KV head; KV heads outermost so that the CTAs
   // running together share the same query tiles in L2
-  const int j = blockIdx.x % n_kblocks;
-  const int rest = blockIdx.x / n_kblocks;
+  const int j = a.kb_begin + blockIdx.x % a.kb_count;
+  const int rest = blockIdx.x / a.kb_count;
   const int b = rest % a.B;
   const int g = rest / a.B;
   const int G = a.Hq / a.Hkv;
@@ -914,14 +915,25 @@ cudaError_t launch_bwd_kernels(const BwdArgs& base, const CUtensorMap& mapQ, con
   if (!base.skip_global)
     bwd_dq_kernel<D><<<n_tiles * base.B * base.Hq, kDqThreads, DqSmem<D>::kTotal, s>>>(mapQc, mapDOc, mapK, mapV, a);
   phase_events().mark(s);
-  const unsigned n_kblocks = (base.Lk + kTileN - 1) / kTileN;
-  bwd_dkv_kernel<D><<<n_kblocks * base.B * base.Hkv, kDkvThreads, DkvSmem<D>::kTotal, s>>>(mapQ, mapDO, mapQc, mapDOc, mapK,
-                                                                                  mapV, base);
-  phase_events().mark(s);
+  const int n_kblocks = (base.Lk + kTileN - 1) / kTileN;
+  // A caller that registered a seventh phase event wants the first three quarters of dK / dV early (to move them
+  // while the rest is computed): two launches over key-block ranges, a boundary in between.
+  const int split = phase_events().n >= 7 ? dkv_split_block(n_kblocks) : 0;
+  a = base;
+  for (int part = 0; part < 2; ++part) {
+    a.kb_begin = part == 0 ? 0 : split;
+    a.kb_count = part == 0 ? (split > 0 ? split : n_kblocks) : n_kblocks - split;
+    if (part == 1 && split == 0) break;
+    bwd_dkv_kernel<D><<<(unsigned)a.kb_count * base.B * base.Hkv, kDkvThreads, DkvSmem<D>::kTotal, s>>>(
+        mapQ, mapDO, mapQc, mapDOc, mapK, mapV, a);
+    phase_events().mark(s);
+  }
   return cudaGetLastError();
 }
 
 }  // namespace
+
+int dkv_split_block(int n_kblocks) { return n_kblocks >= 8 ? (3 * n_kblocks) / 4 : 0; }
 
 size_t bwd_ws_size(const l2a_params* p) { return kWsHeaderBytes + 2 * rows_bytes(p) + 3 * stat_bytes(p); }
 

@@ -353,7 +353,7 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
   struct Aux {
     int device = -1;
     cudaStream_t in = nullptr, out = nullptr;
-    cudaEvent_t start = nullptr, up = nullptr, fwd = nullptr, phase[6] = {}, down = nullptr, chunk[4] = {};
+    cudaEvent_t start = nullptr, up = nullptr, fwd = nullptr, phase[7] = {}, down = nullptr, chunk[4] = {};
   };
   static thread_local Aux aux;
   int dev_id = 0;
@@ -363,7 +363,7 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
         cudaStreamCreateWithFlags(&aux.out, cudaStreamNonBlocking) != cudaSuccess)
       return L2A_ERR_CUDA;
     cudaEvent_t* evs[] = {&aux.start, &aux.up, &aux.fwd, &aux.down, &aux.phase[0], &aux.phase[1], &aux.phase[2],
-                          &aux.phase[3], &aux.phase[4], &aux.phase[5], &aux.chunk[0], &aux.chunk[1], &aux.chunk[2],
+                          &aux.phase[3], &aux.phase[4], &aux.phase[5], &aux.phase[6], &aux.chunk[0], &aux.chunk[1], &aux.chunk[2],
                           &aux.chunk[3]};
     for (cudaEvent_t* e : evs)
       if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return L2A_ERR_CUDA;
@@ -442,10 +442,12 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
   L2A_TRY(cudaMemcpyAsync(host->O, dev->O, qb, cudaMemcpyDeviceToHost, aux.out));
   if (bwd) {
     L2A_TRY(cudaStreamWaitEvent(s, aux.up, 0));
-    // phase boundary 4 of the backward = both dQ kernels have finished: dQ can leave while dK/dV are computed
-    void* phase_events[6];
-    for (int i = 0; i < 6; ++i) phase_events[i] = aux.phase[i];
-    st = l2a_profile_next_call(phase_events, 6);
+    // phase boundary 4 of the backward = both dQ kernels have finished: dQ can leave while dK/dV are computed;
+    // with seven events the dK/dV kernel runs as two launches and boundary 5 says that the key rows of the first
+    // one are final
+    void* phase_events[7];
+    for (int i = 0; i < 7; ++i) phase_events[i] = aux.phase[i];
+    st = l2a_profile_next_call(phase_events, 7);
     if (st != L2A_OK) return st;
     st = l2a_backward(&q, dev->Q, dev->K, dev->V, dev->d_mask, dev->q_idx, dev->n_routed, dev->prefix, dev->dO,
                       dev->S_save, dev->A_c, dev->lse_loc, dev->lse_glb, dev->dQ, dev->dK, dev->dV, nullptr,
@@ -453,8 +455,20 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
     if (st != L2A_OK) return st;
     L2A_TRY(cudaStreamWaitEvent(aux.out, aux.phase[4], 0));
     L2A_TRY(cudaMemcpyAsync(host->dQ, dev->dQ, qb, cudaMemcpyDeviceToHost, aux.out));
-    L2A_TRY(cudaMemcpyAsync(host->dK, dev->dK, kb, cudaMemcpyDeviceToHost, s));
-    L2A_TRY(cudaMemcpyAsync(host->dV, dev->dV, kb, cudaMemcpyDeviceToHost, s));
+    const int64_t split_rows = (int64_t)dkv_split_block(ceil_div(p->Lk, kTileN)) * kTileN;   // 0: one launch
+    const size_t krow = (size_t)p->Hkv * p->D * sizeof(bf16);
+    if (split_rows > 0) L2A_TRY(cudaStreamWaitEvent(aux.out, aux.phase[5], 0));
+    for (int b = 0; b < p->B; ++b) {
+      const size_t base = (size_t)b * p->Lk * krow, early = (size_t)split_rows * krow, late = (size_t)p->Lk * krow - early;
+      uint8_t *hk = static_cast<uint8_t*>(host->dK) + base, *hv = static_cast<uint8_t*>(host->dV) + base;
+      const uint8_t *gk = static_cast<const uint8_t*>(dev->dK) + base, *gv = static_cast<const uint8_t*>(dev->dV) + base;
+      if (early > 0) {
+        L2A_TRY(cudaMemcpyAsync(hk, gk, early, cudaMemcpyDeviceToHost, aux.out));
+        L2A_TRY(cudaMemcpyAsync(hv, gv, early, cudaMemcpyDeviceToHost, aux.out));
+      }
+      L2A_TRY(cudaMemcpyAsync(hk + early, gk + early, late, cudaMemcpyDeviceToHost, s));
+      L2A_TRY(cudaMemcpyAsync(hv + early, gv + early, late, cudaMemcpyDeviceToHost, s));
+    }
   }
   L2A_TRY(cudaEventRecord(aux.down, aux.out));
   L2A_TRY(cudaStreamWaitEvent(s, aux.down, 0));   // the caller's stream ends the step with every result delivered

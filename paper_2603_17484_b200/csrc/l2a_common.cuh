@@ -73,6 +73,8 @@ struct FwdArgs {
   int pair_begin, pair_end;  // 256-row query groups [pair_begin, pair_end) this launch covers (all: 0 .. ceil(Lq / 256))
 };
 size_t bwd_ws_size(const l2a_params* p);
+// First key block of the second dK/dV launch when the backward is asked for the early boundary (0: not split).
+int dkv_split_block(int n_kblocks);
 
 // One-shot, thread-local registration of phase-boundary events (see l2a_profile_next_call).
 struct PhaseEvents {
