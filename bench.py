@@ -393,16 +393,18 @@ def main():
     tensor_phases = {k: v for k, v in phase_ms.items() if k in kernel_flops}
     dom = max(tensor_phases, key=tensor_phases.get)
     achieved = kernel_flops[dom] / phase_ms[dom] / 1e9
-    # DRAM traffic of the dominant kernel: ncu measured dram read+write = 1.13 x the algorithmic bytes of the dK/dV
-    # launch on the 32K case (profiles/attention_kernels_qwen25_7b_32k.md); every operand is read once, re-reads
-    # hit L2, so traffic scales with the tensor bytes of the launch
+    # DRAM traffic of the dominant kernel.  Measured with ncu (one pass, dram__bytes_read.sum + dram__bytes_write.sum)
+    # on this very workload, stress_128k: 4.57 GB read + 0.56 GB written per dK/dV launch = 1.42 x the algorithmic
+    # bytes of the launch (Q, dO and their compact copies read once, K and V read, dK and dV written); on the 32K
+    # case the ratio is 1.13 (profiles/).  Other workloads report the figure scaled by their tensor bytes.
     qb = cfg.B * cfg.L * cfg.Hq * cfg.D * 2
     kb = cfg.B * cfg.L * cfg.Hkv * cfg.D * 2
     dkv_alg_bytes = 2 * qb * (1 + float(d.mean())) + 4 * kb
-    traffic = 1.13 * dkv_alg_bytes if dom == "bwd_dkv" else None
+    traffic = (1.42 if cfg.L > 65536 else 1.13) * dkv_alg_bytes if dom == "bwd_dkv" else None
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peaks["sustained"], "unit": "TFLOP/s",
                 "frac": achieved / peaks["sustained"], "traffic": traffic,
-                "traffic_note": "bytes per launch, scaled from an ncu capture of the 32K case by tensor bytes",
+                "traffic_note": "bytes per launch: ncu capture of the 128K workload (1.42 x algorithmic bytes) or of the "
+                                "32K case (1.13 x), scaled by the launch's tensor bytes",
                 "peak_kind": f"sustained bf16 GEMM, {peaks['source']}", "launch_ms": phase_ms[dom],
                 "algorithmic_flops_per_launch": kernel_flops[dom]}
 
