@@ -519,7 +519,6 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
                const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, const BwdArgs a) {
   using SM = DkvSmem<D>;
   constexpr int kKSteps = D / 16;
-  const int n_kblocks = (a.Lk + kTileN - 1) / kTileN;
   // key blocks ascending (most work first) inside one KV head; KV heads outermost so that the CTAs
   // running together share the same query tiles in L2
   const int j = a.kb_begin + blockIdx.x % a.kb_count;
