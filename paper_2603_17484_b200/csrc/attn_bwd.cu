@@ -41,6 +41,15 @@ __device__ long long g_trace[4][8192];
 #else
 #define L2A_TRACE_POINT(role, idx)
 #endif
+// same for one CTA of the dQ kernel (-DL2A_TRACE=<any> -DL2A_TRACE_DQ=<block>), roles 0 (MMA warp) and 1 (compute warp)
+#if defined(L2A_TRACE) && defined(L2A_TRACE_DQ)
+#define L2A_TRACE_DQ_POINT(role, idx)                                                           \
+  do {                                                                                          \
+    if (blockIdx.x == (L2A_TRACE_DQ) && (idx) < 8192) g_trace[role][idx] = clock64();           \
+  } while (0)
+#else
+#define L2A_TRACE_DQ_POINT(role, idx)
+#endif
 
 // ------------------------------------------------------------------------------------------------
 // Delta / dgate preprocess.  The grid is one resident wave; every warp owns a contiguous range of tokens.  A token's
@@ -322,18 +331,22 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
       }
       for (int it = 0; ok && it < n_blocks; ++it) {
         if (!mbar_spin_warp(&bar->ds_full, it & 1, abort_flag)) { ok = false; break; }
+        if (lane == 0) L2A_TRACE_DQ_POINT(0, 4 * it);
         tc_fence_after();
         issue_dQ(it);
+        if (lane == 0) L2A_TRACE_DQ_POINT(0, 4 * it + 1);
         if (it + 1 < n_blocks) {
           if (!mbar_spin_warp(&bar->v_full[(it + 1) & 1], ((it + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
           issue_dP(it + 1);
         }
+        if (lane == 0) L2A_TRACE_DQ_POINT(0, 4 * it + 2);
         if (it + 2 < n_blocks) {
           if (!mbar_spin_warp(&bar->k_full[(it + 2) % 3], ((it + 2) / 3) & 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
           issue_S(it + 2);
         }
+        if (lane == 0) L2A_TRACE_DQ_POINT(0, 4 * it + 3);
       }
       if (ok) tc_commit(&bar->final_bar, leader);
     }
@@ -355,6 +368,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     bool ok = true;
     for (int it = 0; it < n_blocks; ++it) {
       if (!__all_sync(0xffffffffu, mbar_wait(&bar->s_full[it & 1], (it >> 1) & 1, abort_flag))) { ok = false; break; }
+      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_DQ_POINT(1, 4 * it);
       tc_fence_after();
       const int k0 = (jlo + it) * kTileN + q * 32;   // first key of this quarter
       const bool partial = (k0 + 31 > min_pos) || (k0 < max_pos - w_eff) || ragged;
@@ -377,7 +391,9 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
           sv[e] = __float_as_uint((kp <= pos && kp >= pos_lo) ? p : 0.f);
         }
       }
+      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_DQ_POINT(1, 4 * it + 1);
       if (!__all_sync(0xffffffffu, mbar_wait(&bar->dp_full, it & 1, abort_flag))) { ok = false; break; }
+      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_DQ_POINT(1, 4 * it + 2);
       tc_fence_after();
       uint32_t dv[32];
       tmem_ld32(tmem + lane_base + 384 + q * 32, dv);
@@ -394,6 +410,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(&bar->ds_full);
+      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_DQ_POINT(1, 4 * it + 3);
     }
     // epilogue: quarter q stores D/4 columns of dQ
     if (ok && __all_sync(0xffffffffu, mbar_wait(&bar->final_bar, 0, abort_flag))) {
