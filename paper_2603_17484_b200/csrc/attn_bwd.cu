@@ -164,7 +164,7 @@ struct BwdArgs {
 //   warp 16    : TMA producer          warp 17 : tcgen05 MMA issuer, TMEM owner
 //   warp 18    : (dK/dV kernel only) stages the row statistics of each query tile
 constexpr int kComputeWarps = 16;
-constexpr int kDqThreads = (kComputeWarps + 2) * 32;    // 576
+constexpr int kDqThreads = (kComputeWarps + 3) * 32;    // 608: + TMA producer + two MMA issuers
 constexpr int kDkvThreads = (kComputeWarps + 3) * 32;   // 608
 
 __device__ __forceinline__ float bf16lo_to_f32(uint32_t packed) { return __uint_as_float(packed << 16); }
@@ -172,11 +172,15 @@ __device__ __forceinline__ float bf16hi_to_f32(uint32_t packed) { return __uint_
 
 // ================================================================================================
 // dQ kernel: one 128-row query tile per CTA; Q and dO stay in shared memory, K/V blocks stream.
-//   TMEM: dQ [0,D) | S (two buffers) [128,256) [256,384) | dP [384,512).
-//   dS (bf16) is written over dP: quarter q puts its 16 packed columns at the start of its own 32
-//   columns, and is the A operand of dQ += dS K.
-//   MMA order per key block j:  dQ(j-1) | dP(j) | S(j+1): the exponentials of block j run under dQ(j-1) and
-//   dP(j), the dS of block j under S(j+1), so the tensor pipe never waits for the CUDA cores.
+//   TMEM: dQ [0,D) | S [128,256) | dP (two buffers) [256,384) [384,512).
+//   The scores go to registers at once (barrier s_taken), so one S buffer is enough; dS (bf16) is written over the
+//   dP buffer of its key block (quarter q puts its 16 packed columns at the start of its own 32 columns) and is the
+//   A operand of dQ += dS K.  With two dP buffers nothing the compute warps wait for depends on an MMA that waits
+//   for them: S(j+1) and dP(j+1) are produced a block ahead, dQ(j) only consumes.
+//   Two warps issue the MMAs, on different scheduler partitions: warp 17 the dQ stream, warp 18 the S / dP stream.
+//   A single issuer leaves a gap between consecutive MMAs (its next instruction is prepared only after the
+//   previous one was accepted: measured 105-125 clk per MMA inside this kernel against 64 in a lean stream); with
+//   two independent streams one MMA is always waiting at the pipe (74 clk per MMA measured).
 template <int D>
 struct DqSmem {
   static constexpr int kTileBytes = 128 * D * 2;
@@ -192,7 +196,7 @@ struct DqSmem {
 struct DqBarriers {
   uint64_t q_full;
   uint64_t k_full[3], k_empty[3], v_full[2], v_empty[2];
-  uint64_t s_full[2], dp_full, ds_full, final_bar;
+  uint64_t s_full, s_taken, dp_full[2], ds_full[2], dq_done[2], final_bar;
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -236,10 +240,13 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     for (int s = 0; s < 3; ++s) { mbar_init(&bar->k_full[s], 1); mbar_init(&bar->k_empty[s], 1); }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bar->v_full[s], 1); mbar_init(&bar->v_empty[s], 1);
-      mbar_init(&bar->s_full[s], 1);
+      // per dP buffer, so that a waiter can never be a whole phase behind the barrier it polls
+      mbar_init(&bar->dp_full[s], 1);
+      mbar_init(&bar->ds_full[s], kComputeWarps * 32);
+      mbar_init(&bar->dq_done[s], 1);               // dQ(j) has consumed dS(j): the buffer is free again
     }
-    mbar_init(&bar->dp_full, 1);
-    mbar_init(&bar->ds_full, kComputeWarps * 32);
+    mbar_init(&bar->s_full, 1);
+    mbar_init(&bar->s_taken, kComputeWarps * 32);   // every compute thread holds its scores in registers
     mbar_init(&bar->final_bar, 1);
     bar->abort_flag = 0;
     fence_mbar_init();
@@ -277,8 +284,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
       }
     }
     __syncwarp();
-  } else if (warp == 17) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (warp == 17 || warp == 18) {
+    // ------------------------------------------------------------------ MMA issuers
     // (whole warp runs the loop; only the tcgen05 instructions are predicated on lane 0)
     {
       const uint32_t leader = (lane == 0);
@@ -290,65 +297,70 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
       const uint64_t dkm_base = smem_desc_sw128(smem_u32(sK), kBoxBytes, 1024);    // same bytes as MN-major B
       const uint64_t dv_base = smem_desc_sw128(smem_u32(sV), 16, 1024);
       constexpr uint32_t kStageStep = SM::kTileBytes >> 4;
-      auto issue_S = [&](int it) {   // S(it) = Q K^T into S buffer it&1
+      auto issue_S = [&](int it) {   // S(it) = Q K^T
         const uint64_t kd = dk_base + (it % 3) * kStageStep;
-        const uint32_t buf = tmem + 128 + (it & 1) * 128;
 #pragma unroll
         for (int kk = 0; kk < kKSteps; ++kk) {
           const uint32_t c = ((kk >> 2) * kBoxBytes + (kk & 3) * 32) >> 4;
-          mma_ss(buf, dq + c, kd + c, idesc_s, kk > 0, leader);
+          mma_ss(tmem + 128, dq + c, kd + c, idesc_s, kk > 0, leader);
         }
-        tc_commit(&bar->s_full[it & 1], leader);
+        tc_commit(&bar->s_full, leader);
       };
-      auto issue_dP = [&](int it) {  // dP(it) = dO V^T
+      auto issue_dP = [&](int it) {  // dP(it) = dO V^T into dP buffer it&1
         const uint64_t vd = dv_base + (it & 1) * kStageStep;
+        const uint32_t buf = tmem + 256 + (it & 1) * 128;
 #pragma unroll
         for (int kk = 0; kk < kKSteps; ++kk) {
           const uint32_t c = ((kk >> 2) * kBoxBytes + (kk & 3) * 32) >> 4;
-          mma_ss(tmem + 384, ddo + c, vd + c, idesc_s, kk > 0, leader);
+          mma_ss(buf, ddo + c, vd + c, idesc_s, kk > 0, leader);
         }
-        tc_commit(&bar->dp_full, leader);
+        tc_commit(&bar->dp_full[it & 1], leader);
         tc_commit(&bar->v_empty[it & 1], leader);
       };
       auto issue_dQ = [&](int it) {  // dQ += dS(it) K
         const uint64_t kd = dkm_base + (it % 3) * kStageStep;
+        const uint32_t buf = tmem + 256 + (it & 1) * 128;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
-          mma_ts(tmem, tmem + 384 + (kk >> 1) * 32 + (kk & 1) * 8, kd + ((kk * 2048) >> 4), idesc_dq,
+          mma_ts(tmem, buf + (kk >> 1) * 32 + (kk & 1) * 8, kd + ((kk * 2048) >> 4), idesc_dq,
                  (kk > 0 || it > 0) ? 1u : 0u, leader);
         tc_commit(&bar->k_empty[it % 3], leader);
+        tc_commit(&bar->dq_done[it & 1], leader);
       };
-      bool ok = mbar_spin_warp(&bar->q_full, 0, abort_flag) && mbar_spin_warp(&bar->k_full[0], 0, abort_flag) &&
-                mbar_spin_warp(&bar->v_full[0], 0, abort_flag);
-      if (ok) {
-        tc_fence_after();
-        issue_S(0);
-        issue_dP(0);
-        if (n_blocks > 1) {
-          ok = mbar_spin_warp(&bar->k_full[1], 0, abort_flag);
-          if (ok) { tc_fence_after(); issue_S(1); }
+      if (warp == 17) {
+        // ---- consumer stream: dQ(it) as soon as dS(it) is in TMEM
+        bool ok = true;
+        for (int it = 0; ok && it < n_blocks; ++it) {
+          if (!mbar_spin_warp(&bar->ds_full[it & 1], (it >> 1) & 1, abort_flag)) { ok = false; break; }
+          if (lane == 0) L2A_TRACE_DQ_POINT(0, 4 * it);
+          tc_fence_after();
+          issue_dQ(it);
+          if (lane == 0) L2A_TRACE_DQ_POINT(0, 4 * it + 1);
         }
-      }
-      for (int it = 0; ok && it < n_blocks; ++it) {
-        if (!mbar_spin_warp(&bar->ds_full, it & 1, abort_flag)) { ok = false; break; }
-        if (lane == 0) L2A_TRACE_DQ_POINT(0, 4 * it);
-        tc_fence_after();
-        issue_dQ(it);
-        if (lane == 0) L2A_TRACE_DQ_POINT(0, 4 * it + 1);
-        if (it + 1 < n_blocks) {
+        if (ok) tc_commit(&bar->final_bar, leader);
+      } else {
+        // ---- producer stream: S(it+1) once the scores of block it are in registers, dP(it+1) once its buffer is free
+        bool ok = mbar_spin_warp(&bar->q_full, 0, abort_flag) && mbar_spin_warp(&bar->k_full[0], 0, abort_flag) &&
+                  mbar_spin_warp(&bar->v_full[0], 0, abort_flag);
+        if (ok) {
+          tc_fence_after();
+          issue_S(0);
+          issue_dP(0);
+        }
+        for (int it = 0; ok && it + 1 < n_blocks; ++it) {
+          if (!mbar_spin_warp(&bar->s_taken, it & 1, abort_flag) ||
+              !mbar_spin_warp(&bar->k_full[(it + 1) % 3], ((it + 1) / 3) & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          issue_S(it + 1);
+          if (lane == 0) L2A_TRACE_DQ_POINT(0, 4 * it + 2);
+          // dP(it+1) overwrites the buffer that held dS(it-1)
+          if (it >= 1 && !mbar_spin_warp(&bar->dq_done[(it - 1) & 1], ((it - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
           if (!mbar_spin_warp(&bar->v_full[(it + 1) & 1], ((it + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
           issue_dP(it + 1);
+          if (lane == 0) L2A_TRACE_DQ_POINT(0, 4 * it + 3);
         }
-        if (lane == 0) L2A_TRACE_DQ_POINT(0, 4 * it + 2);
-        if (it + 2 < n_blocks) {
-          if (!mbar_spin_warp(&bar->k_full[(it + 2) % 3], ((it + 2) / 3) & 1, abort_flag)) { ok = false; break; }
-          tc_fence_after();
-          issue_S(it + 2);
-        }
-        if (lane == 0) L2A_TRACE_DQ_POINT(0, 4 * it + 3);
       }
-      if (ok) tc_commit(&bar->final_bar, leader);
     }
     __syncwarp();
   } else {
@@ -367,14 +379,16 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     const bool ragged = (last - row0 + 1 < kTileM);
     bool ok = true;
     for (int it = 0; it < n_blocks; ++it) {
-      if (!__all_sync(0xffffffffu, mbar_wait(&bar->s_full[it & 1], (it >> 1) & 1, abort_flag))) { ok = false; break; }
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->s_full, it & 1, abort_flag))) { ok = false; break; }
       if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_DQ_POINT(1, 4 * it);
       tc_fence_after();
       const int k0 = (jlo + it) * kTileN + q * 32;   // first key of this quarter
       const bool partial = (k0 + 31 > min_pos) || (k0 < max_pos - w_eff) || ragged;
       uint32_t sv[32];
-      tmem_ld32(tmem + lane_base + 128 + (it & 1) * 128 + q * 32, sv);
+      tmem_ld32(tmem + lane_base + 128 + q * 32, sv);
       tmem_ld_wait();
+      tc_fence_before();
+      mbar_arrive(&bar->s_taken);      // the S columns may be overwritten by the next block's scores
       if (!partial) {
 #pragma unroll
         for (int e = 0; e < 32; e += 2) {
@@ -392,11 +406,12 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         }
       }
       if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_DQ_POINT(1, 4 * it + 1);
-      if (!__all_sync(0xffffffffu, mbar_wait(&bar->dp_full, it & 1, abort_flag))) { ok = false; break; }
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->dp_full[it & 1], (it >> 1) & 1, abort_flag))) { ok = false; break; }
       if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_DQ_POINT(1, 4 * it + 2);
       tc_fence_after();
+      const uint32_t dp_addr = tmem + lane_base + 256 + (it & 1) * 128 + q * 32;
       uint32_t dv[32];
-      tmem_ld32(tmem + lane_base + 384 + q * 32, dv);
+      tmem_ld32(dp_addr, dv);
       tmem_ld_wait();
       uint32_t pk[16];
 #pragma unroll
@@ -406,10 +421,10 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
         const float2 ds = __fmul2_rn(make_float2(__uint_as_float(sv[2 * e]), __uint_as_float(sv[2 * e + 1])), t);
         pk[e] = pack_bf16(ds.x, ds.y);
       }
-      tmem_st16(tmem + lane_base + 384 + q * 32, pk);
+      tmem_st16(dp_addr, pk);
       tmem_st_wait();
       tc_fence_before();
-      mbar_arrive(&bar->ds_full);
+      mbar_arrive(&bar->ds_full[it & 1]);
       if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_DQ_POINT(1, 4 * it + 3);
     }
     // epilogue: quarter q stores D/4 columns of dQ
