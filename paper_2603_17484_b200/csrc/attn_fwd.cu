@@ -99,6 +99,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
 
   const int32_t* q_idx_b = a.q_idx + (int64_t)b * a.Lq;
   const int w_eff = a.global_mode ? 0x3fffffff : a.window;
+  if (a.global_mode) {
+    // launches restricted to a row range take the groups whose last row falls into it: every group exactly once
+    const int c_last = min(row0 + kRowsPerCta, n_rows) - 1;
+    const int t_last = compact ? q_idx_b[c_last] : c_last;
+    if (t_last < a.row_begin || t_last >= a.row_end) return;
+  }
 
   TileRange tr[kNumTiles];
   int jlo = 0x7fffffff, jhi = -1;

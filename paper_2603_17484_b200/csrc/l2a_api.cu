@@ -143,11 +143,13 @@ l2a_status l2a_route_compact(const l2a_params* p, const void* router, int router
 // l2a_forward over the 256-row query groups [pair_begin, pair_end) (pair_end < 0: all of them).  A proper sub-range
 // is used by l2a_step_host to start Local Attention on the rows whose queries have already arrived; it is only
 // meaningful for the local module (L2A_FLAG_SKIP_GLOBAL), and only the first call of a step clears the status word.
+// [row_begin, row_end) restricts the global phase (L2A_FLAG_GLOBAL_PHASE) to the routed rows of that range: the
+// gather takes exactly those rows, the attention launch the compact groups whose last row lies in the range.
 static l2a_status forward_range(const l2a_params* p, const void* Q, const void* K, const void* V,
                                 const uint8_t* d_mask, const int32_t* q_idx, const int32_t* n_routed,
                                 const int32_t* prefix, void* O, void* S_save, void* A_c, float* lse_loc,
                                 float* lse_glb, void* fwd_ws, size_t fwd_ws_bytes, void* stream, int pair_begin,
-                                int pair_end, bool clear_status);
+                                int pair_end, bool clear_status, int row_begin = 0, int row_end = 0x7fffffff);
 
 l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const void* V, const uint8_t* d_mask,
                        const int32_t* q_idx, const int32_t* n_routed, const int32_t* prefix, void* O, void* S_save,
@@ -160,7 +162,7 @@ static l2a_status forward_range(const l2a_params* p, const void* Q, const void* 
                                 const uint8_t* d_mask, const int32_t* q_idx, const int32_t* n_routed,
                                 const int32_t* prefix, void* O, void* S_save, void* A_c, float* lse_loc,
                                 float* lse_glb, void* fwd_ws, size_t fwd_ws_bytes, void* stream, int pair_begin,
-                                int pair_end, bool clear_status) {
+                                int pair_end, bool clear_status, int row_begin, int row_end) {
   l2a_status st = check_params(p);
   if (st != L2A_OK) return st;
   const bool save = p->flags & L2A_FLAG_SAVE_FOR_BWD;
@@ -188,6 +190,9 @@ static l2a_status forward_range(const l2a_params* p, const void* Q, const void* 
   if (pair_end < 0) pair_end = n_pairs;
   if (pair_begin < 0 || pair_end > n_pairs || pair_begin > pair_end) return L2A_ERR_INVALID_ARG;
   if (!whole && !skip_global) return L2A_ERR_INVALID_ARG;
+  const bool row_range = row_begin > 0 || row_end < p->Lq;
+  if (row_range && (!global_phase || row_begin < 0 || row_begin > row_end)) return L2A_ERR_INVALID_ARG;
+  if (row_end > p->Lq) row_end = p->Lq;
   if (clear_status && cudaMemsetAsync(ws, 0, kWsHeaderBytes, s) != cudaSuccess) return L2A_ERR_CUDA;
 
   CUtensorMap mapQ, mapK, mapV, mapQc;
@@ -209,14 +214,16 @@ static l2a_status forward_range(const l2a_params* p, const void* Q, const void* 
   a.combine_mask = nullptr;
   a.pair_begin = 0;
   a.pair_end = n_pairs;
+  a.row_begin = row_range ? row_begin : 0;
+  a.row_end = row_range ? row_end : 0x7fffffff;
 
   PhaseEvents& pe = phase_events();
   struct ClearOnExit { PhaseEvents& p; ~ClearOnExit() { p.clear(); } } clear_on_exit{pe};
   pe.mark(s);
   if (!skip_global && !force_all) {
     // consolidate routed query rows (Algorithm 1, step 1); independent of the local pass
-    if (launch_gather_rows(static_cast<const bf16*>(Q), Qc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s) !=
-        cudaSuccess)
+    if (launch_gather_rows(static_cast<const bf16*>(Q), Qc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s,
+                           row_range ? prefix : nullptr, row_begin, row_end) != cudaSuccess)
       return L2A_ERR_CUDA;
   }
   pe.mark(s);
@@ -353,7 +360,7 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
   struct Aux {
     int device = -1;
     cudaStream_t in = nullptr, out = nullptr;
-    cudaEvent_t start = nullptr, up = nullptr, fwd = nullptr, phase[7] = {}, down = nullptr, chunk[4] = {};
+    cudaEvent_t start = nullptr, up = nullptr, fwd = nullptr, phase[7] = {}, down = nullptr, chunk[8] = {};
   };
   static thread_local Aux aux;
   int dev_id = 0;
@@ -364,7 +371,7 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
       return L2A_ERR_CUDA;
     cudaEvent_t* evs[] = {&aux.start, &aux.up, &aux.fwd, &aux.down, &aux.phase[0], &aux.phase[1], &aux.phase[2],
                           &aux.phase[3], &aux.phase[4], &aux.phase[5], &aux.phase[6], &aux.chunk[0], &aux.chunk[1], &aux.chunk[2],
-                          &aux.chunk[3]};
+                          &aux.chunk[3], &aux.chunk[4], &aux.chunk[5], &aux.chunk[6], &aux.chunk[7]};
     for (cudaEvent_t* e : evs)
       if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return L2A_ERR_CUDA;
     aux.device = dev_id;
@@ -375,23 +382,34 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
   l2a_params q = *p;
   if (!bwd) q.flags &= ~L2A_FLAG_SAVE_FOR_BWD;
   const int n_pairs = ceil_div(p->Lq, kRowsPerCta);
-  constexpr int kChunks = 4;
-  const bool chunked = p->B == 1 && n_pairs >= 4 * kChunks &&
+  constexpr int kChunks = 8;
+  const bool chunked = p->B == 1 && n_pairs >= 2 * kChunks &&
                        !(p->flags & (L2A_FLAG_SKIP_LOCAL | L2A_FLAG_SKIP_GLOBAL | L2A_FLAG_GLOBAL_PHASE));
   if (chunked) {
-    // One sequence: K and V go first, then Q in four row ranges on the upload stream; Local Attention starts on a
-    // range as soon as its queries have landed, so only the first range's copy is exposed.  The global phase
-    // (which needs every query) follows, adding into O exactly as a single l2a_forward call would.
+    // One sequence: K, V and Q go up in eight row ranges on the upload stream (attention is causal: the queries of a
+    // range need no later keys); Local Attention and then the Global Attention of the routed rows of a range start
+    // as soon as it has landed, so only the first range's copy is exposed.  Results equal a single l2a_forward call.
     L2A_TRY(cudaStreamWaitEvent(aux.in, aux.start, 0));
-    L2A_TRY(cudaMemcpyAsync(dev->K, host->K, kb, cudaMemcpyHostToDevice, aux.in));
-    L2A_TRY(cudaMemcpyAsync(dev->V, host->V, kb, cudaMemcpyHostToDevice, aux.in));
-    const size_t row_bytes = (size_t)p->Hq * p->D * sizeof(bf16);
+    const size_t row_bytes = (size_t)p->Hq * p->D * sizeof(bf16), krow_bytes = (size_t)p->Hkv * p->D * sizeof(bf16);
     int pair_edge[kChunks + 1];
     for (int c = 0; c <= kChunks; ++c) pair_edge[c] = (int)((int64_t)n_pairs * c / kChunks);
+    int64_t k_done = 0;   // key rows uploaded so far
     for (int c = 0; c < kChunks; ++c) {
       const int64_t r0 = (int64_t)pair_edge[c] * kRowsPerCta;
       int64_t r1 = (int64_t)pair_edge[c + 1] * kRowsPerCta;
       if (r1 > p->Lq) r1 = p->Lq;
+      // the rows of this range see the keys up to position r1 - 1 + q_pos_offset (everything in the last range)
+      int64_t k1 = c + 1 == kChunks ? p->Lk : r1 + p->q_pos_offset;
+      if (k1 > p->Lk) k1 = p->Lk;
+      if (k1 > k_done) {
+        L2A_TRY(cudaMemcpyAsync(static_cast<uint8_t*>(dev->K) + k_done * krow_bytes,
+                                static_cast<const uint8_t*>(host->K) + k_done * krow_bytes,
+                                (size_t)(k1 - k_done) * krow_bytes, cudaMemcpyHostToDevice, aux.in));
+        L2A_TRY(cudaMemcpyAsync(static_cast<uint8_t*>(dev->V) + k_done * krow_bytes,
+                                static_cast<const uint8_t*>(host->V) + k_done * krow_bytes,
+                                (size_t)(k1 - k_done) * krow_bytes, cudaMemcpyHostToDevice, aux.in));
+        k_done = k1;
+      }
       L2A_TRY(cudaMemcpyAsync(static_cast<uint8_t*>(dev->Q) + r0 * row_bytes,
                               static_cast<const uint8_t*>(host->Q) + r0 * row_bytes, (size_t)(r1 - r0) * row_bytes,
                               cudaMemcpyHostToDevice, aux.in));
@@ -404,8 +422,9 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
     st = l2a_route_compact(p, dev->router, router_kind, logit_threshold, dev->d_mask, dev->q_idx, dev->n_routed,
                            dev->prefix, dev->route_ws, dev->route_ws_bytes, stream);
     if (st != L2A_OK) return st;
-    l2a_params ql = q;
+    l2a_params ql = q, qg = q;
     ql.flags = (q.flags & ~L2A_FLAG_FORCE_ALL_GLOBAL) | L2A_FLAG_SKIP_GLOBAL;
+    qg.flags |= L2A_FLAG_GLOBAL_PHASE;
     for (int c = 0; c < kChunks; ++c) {
       L2A_TRY(cudaStreamWaitEvent(s, aux.chunk[c], 0));
       st = forward_range(&ql, dev->Q, dev->K, dev->V, dev->d_mask, dev->q_idx, dev->n_routed, dev->prefix, dev->O,
@@ -413,13 +432,15 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
                          bwd ? dev->lse_glb : nullptr, dev->fwd_ws, dev->fwd_ws_bytes, stream, pair_edge[c],
                          pair_edge[c + 1], c == 0);
       if (st != L2A_OK) return st;
+      // Global Attention of the routed rows that have arrived so far: the compact groups whose last row lies in
+      // this range (a group that straddles two ranges waits for the later one)
+      const int r0 = pair_edge[c] * kRowsPerCta;
+      const int r1 = c + 1 == kChunks ? p->Lq : pair_edge[c + 1] * kRowsPerCta;
+      st = forward_range(&qg, dev->Q, dev->K, dev->V, dev->d_mask, dev->q_idx, dev->n_routed, dev->prefix, dev->O,
+                         bwd ? dev->S_save : nullptr, bwd ? dev->A_c : nullptr, bwd ? dev->lse_loc : nullptr,
+                         bwd ? dev->lse_glb : nullptr, dev->fwd_ws, dev->fwd_ws_bytes, stream, 0, -1, false, r0, r1);
+      if (st != L2A_OK) return st;
     }
-    l2a_params qg = q;
-    qg.flags |= L2A_FLAG_GLOBAL_PHASE;
-    st = forward_range(&qg, dev->Q, dev->K, dev->V, dev->d_mask, dev->q_idx, dev->n_routed, dev->prefix, dev->O,
-                       bwd ? dev->S_save : nullptr, bwd ? dev->A_c : nullptr, bwd ? dev->lse_loc : nullptr,
-                       bwd ? dev->lse_glb : nullptr, dev->fwd_ws, dev->fwd_ws_bytes, stream, 0, -1, false);
-    if (st != L2A_OK) return st;
   } else {
     L2A_TRY(cudaMemcpyAsync(dev->Q, host->Q, qb, cudaMemcpyHostToDevice, s));
     L2A_TRY(cudaMemcpyAsync(dev->K, host->K, kb, cudaMemcpyHostToDevice, s));

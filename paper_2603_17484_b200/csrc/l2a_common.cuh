@@ -42,9 +42,11 @@ constexpr int kRouteBlockElems = 4096;  // positions per CTA of the route/compac
 cudaError_t launch_route_compact(const RouteArgs& a, cudaStream_t stream);
 
 // Gathers rows src[b, q_idx[b][c], :] -> dst[b, c, :] for c < n_routed[b], and zero-fills rows up to
-// the next multiple of kRowsPerCta (bounded by L) so that padded MMA tiles read zeros.
+// the next multiple of kRowsPerCta (bounded by L) so that padded MMA tiles read zeros.  With `prefix` given, only the
+// routed rows t in [row_begin, row_end) are gathered (the padding with the range that ends at L).
 cudaError_t launch_gather_rows(const bf16* src, bf16* dst, const int32_t* q_idx, const int32_t* n_routed,
-                               int B, int L, int row_elems, cudaStream_t stream);
+                               int B, int L, int row_elems, cudaStream_t stream, const int32_t* prefix = nullptr,
+                               int row_begin = 0, int row_end = 0);
 
 // z[b,t] = w . S[b,t,:] + bias (fp32 accumulation); optional sum over t of sigmoid(z)^2 per batch entry
 cudaError_t launch_router_logits(const bf16* S, const float* w, float bias, float* logits, float* sum_sq, int B,
@@ -71,6 +73,7 @@ struct FwdArgs {
   float* lse;   // local: [B,Hq,Lq] by row;  global: [B,Hq,Lq] by compact row; may be NULL
   int* status;  // workspace status word
   int pair_begin, pair_end;  // 256-row query groups [pair_begin, pair_end) this launch covers (all: 0 .. ceil(Lq / 256))
+  int row_begin, row_end;    // global mode: only the groups whose LAST row t lies in [row_begin, row_end)
 };
 size_t bwd_ws_size(const l2a_params* p);
 // First key block of the second dK/dV launch when the backward is asked for the early boundary (0: not split).

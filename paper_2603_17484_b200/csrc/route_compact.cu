@@ -118,14 +118,23 @@ __global__ void __launch_bounds__(kThreads) route_scan_kernel(RouteArgs a) {
 __global__ void __launch_bounds__(256) gather_rows_kernel(const bf16* __restrict__ src, bf16* __restrict__ dst,
                                                           const int32_t* __restrict__ q_idx,
                                                           const int32_t* __restrict__ n_routed, int L,
-                                                          int row_chunks /* 16-byte chunks per row */) {
+                                                          int row_chunks /* 16-byte chunks per row */,
+                                                          const int32_t* __restrict__ prefix, int row_begin,
+                                                          int row_end) {
   const int b = blockIdx.y;
   const int n_c = n_routed[b];
   int n_pad = (n_c + kRowsPerCta - 1) / kRowsPerCta * kRowsPerCta;
   if (n_pad > L) n_pad = L;
+  // optional restriction to the routed rows t in [row_begin, row_end): they are the compact rows
+  // [prefix[row_begin], prefix[row_end]); the zero padding belongs to the range that ends at L
+  int c_begin = 0;
+  if (prefix != nullptr) {
+    c_begin = prefix[(int64_t)b * (L + 1) + row_begin];
+    if (row_end < L) n_pad = prefix[(int64_t)b * (L + 1) + row_end];
+  }
   const uint4* s = reinterpret_cast<const uint4*>(src) + (int64_t)b * L * row_chunks;
   uint4* d = reinterpret_cast<uint4*>(dst) + (int64_t)b * L * row_chunks;
-  for (int c = blockIdx.x; c < n_pad; c += gridDim.x) {
+  for (int c = c_begin + blockIdx.x; c < n_pad; c += gridDim.x) {
     if (c < n_c) {
       const int t = q_idx[(int64_t)b * L + c];
       for (int i = threadIdx.x; i < row_chunks; i += blockDim.x)
@@ -228,11 +237,12 @@ cudaError_t launch_route_compact(const RouteArgs& a, cudaStream_t stream) {
 }
 
 cudaError_t launch_gather_rows(const bf16* src, bf16* dst, const int32_t* q_idx, const int32_t* n_routed, int B,
-                               int L, int row_elems, cudaStream_t stream) {
+                               int L, int row_elems, cudaStream_t stream, const int32_t* prefix, int row_begin,
+                               int row_end) {
   const int row_chunks = row_elems * 2 / 16;
   int gx = L < 148 * 16 ? L : 148 * 16;
   dim3 grid(gx, B);
-  gather_rows_kernel<<<grid, 256, 0, stream>>>(src, dst, q_idx, n_routed, L, row_chunks);
+  gather_rows_kernel<<<grid, 256, 0, stream>>>(src, dst, q_idx, n_routed, L, row_chunks, prefix, row_begin, row_end);
   return cudaGetLastError();
 }
 

@@ -10,11 +10,13 @@ pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("backward", [False, True])
-@pytest.mark.parametrize("B,L", [(2, 1300), (1, 4389)])   # one long sequence takes the path that uploads Q in row ranges
-def test_step_host_matches_device_calls(backward, B, L):
+# one long sequence takes the path that uploads K, V and Q in row ranges and starts the attention of each range as
+# it lands; the last case has more keys than queries (q_pos_offset = 300)
+@pytest.mark.parametrize("B,L,Lk", [(2, 1300, None), (1, 4389, None), (1, 4200, 4500)])
+def test_step_host_matches_device_calls(backward, B, L, Lk):
     Hq, Hkv, D, W = 4, 2, 128, 256
     d = synth.mask_bernoulli(B, L, 0.3, seed=17)
-    c = Case(B, L, Hq, Hkv, D, W, d, seed=23, backward=backward)
+    c = Case(B, L, Hq, Hkv, D, W, d, seed=23, backward=backward, Lk=Lk)
     c.run_forward()
     want = {"O": c.buf.O.clone()}
     if backward:
