@@ -12,8 +12,12 @@ Gradients additionally inherit the bf16 rounding of the MMA operands P and dS (r
 flash-attention practice): an element of dQ picks up scale * 2^-9 * sum_j |dS_ij| |k_j|.  With N(0,1) inputs dO.v has
 standard deviation sqrt(D) ~ 11, so the very first rows (two or three keys, P ~ 0.5) can carry |dS| ~ 10, where bf16
 is spaced 0.0625 apart, and a dQ element can be off by ~0.03 (reproduced by emulating the kernel's roundings in
-numpy).  Gradient checks therefore let a fraction of at most 1e-5 of the elements exceed the bound, and none by more
-than a factor of two."""
+numpy).  A dK element of an early key sums such terms over every row and every query head of its group: with G = 8,
+D = 64 (scale 1/8) and ~500 terms of |dS| ~ 3 its noise has a standard deviation of ~0.01, so the largest of
+~10^4 elements reaches 0.03-0.04.  Gradient checks therefore let a fraction of at most 1e-5 of the elements (rounded
+up to a whole element) exceed the bound, and none by more than a factor of two."""
+import math
+
 import numpy as np
 import torch
 
@@ -40,7 +44,7 @@ def check_close(got: np.ndarray, want: np.ndarray, what: str, max_abs=MAX_ABS, m
     i = np.unravel_index(np.argmax(excess), err.shape)
     n_over = int((excess > 0).sum())
     msg = f"{what}: abs err {err[i]:.4g} at {i} (got {got[i]}, want {want[i]}), max abs err {err.max():.4g}, {n_over} over"
-    assert n_over <= outlier_frac * err.size, msg
+    assert n_over <= math.ceil(outlier_frac * err.size), msg
     assert (err <= 2.0 * bound).all(), msg
     mean_tol = mean_abs + 2.0 ** -9 * np.abs(want).mean()
     assert err.mean() <= mean_tol, f"{what}: mean abs err {err.mean():.4g} > {mean_tol:.4g}"
