@@ -99,3 +99,33 @@ def test_decode_full_size_cache():
     sh = oracle.Shape(B, 1, Lk, cfg.Hq, cfg.Hkv, cfg.D, cfg.W)
     ref = oracle.forward_full(sh, synth.as_u16(t["Q"]), synth.as_u16(t["K"]), synth.as_u16(t["V"]), d)
     check_close(to_f64(O), ref["o"], "decode O at 128K")
+
+
+def _decode_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        B = int(rng.integers(1, 5))
+        Lk = int(rng.choice([1, 2, 63, 64, 65, 129, 1000, 2049, 4097, 6000]))
+        pos = Lk - 1 - int(rng.choice([0, 0, 0, 1, 17])) if Lk > 20 else Lk - 1
+        Hkv = int(rng.integers(1, 3))
+        G = int(rng.integers(1, 9))
+        D = int(rng.choice([64, 128]))
+        W = int(rng.choice([0, 1, 63, 64, 500, 4096]))
+        out.append((B, Lk, pos, Hkv * G, Hkv, D, W, 500 + i))
+    return out
+
+
+@pytest.mark.parametrize("B,Lk,pos,Hq,Hkv,D,W,seed", _decode_shapes(16, 20260317))
+def test_decode_random_shape(B, Lk, pos, Hq, Hkv, D, W, seed):
+    t = synth.qkv(B, 1, Hq, Hkv, D, seed=seed, Lk=Lk)
+    d = (np.random.default_rng(seed).random((B, 1)) < 0.5).astype(np.uint8)
+    p = l2a.params(B, 1, Lk, Hq, Hkv, D, W, q_pos_offset=pos)
+    ws = torch.empty(l2a.l2a_decode_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    O = torch.full((B, 1, Hq, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    l2a.l2a_decode(p, t["Q"].cuda(), t["K"].cuda(), t["V"].cuda(), torch.from_numpy(d[:, 0].copy()).cuda(), O, ws)
+    torch.cuda.synchronize()
+    assert l2a.l2a_workspace_status(ws) == 0
+    sh = oracle.Shape(B, 1, Lk, Hq, Hkv, D, W, q_pos_offset=pos)
+    ref = oracle.forward_full(sh, synth.as_u16(t["Q"]), synth.as_u16(t["K"]), synth.as_u16(t["V"]), d)
+    check_close(to_f64(O), ref["o"], "decode O")
