@@ -67,6 +67,7 @@ typedef enum {
 /* router_kind of l2a_route_compact */
 #define L2A_ROUTER_MASK_U8 0     /* router = uint8 [B, Lq], non-zero => routed                    */
 #define L2A_ROUTER_LOGITS_F32 1  /* router = fp32 logits [B, Lq]; d = (z >= logit_threshold)      */
+#define L2A_ROUTER_LOGITS_BF16 2 /* router = bf16 logits [B, Lq], compared in fp32 (exact upcast)  */
 
 typedef struct l2a_params {
   int32_t B, Lq, Lk, Hq, Hkv, D;
@@ -103,7 +104,7 @@ l2a_status l2a_workspace_status(const void* ws, void* stream);
  * Routing decision and query compaction (Eq. 3; Section 3.2 "consolidated into a compact,
  * contiguous buffer ... original sequence positions recorded"; Algorithm 1, step 1).
  *
- *   router      in : [B, Lq] uint8 mask or fp32 logits, per router_kind.  For logits the decision
+ *   router      in : [B, Lq] uint8 mask, fp32 logits or bf16 logits, per router_kind.  For logits the decision
  *                    is taken on the logit in fp32, d = (z >= logit_threshold); threshold 0 is
  *                    sigmoid(z) >= 0.5, the tie z == threshold routes, NaN does not.
  *   d_mask      out: [B, Lq] uint8, 0 or 1.
@@ -285,7 +286,7 @@ l2a_status l2a_decode(const l2a_params* p, const void* q, const void* K, const v
  */
 typedef struct l2a_host_io {
   const void *Q, *K, *V;  /* bf16, layouts above                                   */
-  const void* router;     /* [B, Lq] uint8 or fp32, per router_kind                */
+  const void* router;     /* [B, Lq] uint8, fp32 or bf16, per router_kind          */
   const void* dO;         /* bf16 [B, Lq, Hq, D] or NULL for a forward-only step   */
   void* O;                /* out                                                   */
   void *dQ, *dK, *dV;     /* out; may be NULL when dO is NULL                      */

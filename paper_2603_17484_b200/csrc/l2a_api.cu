@@ -119,9 +119,12 @@ l2a_status l2a_route_compact(const l2a_params* p, const void* router, int router
   l2a_status st = check_params(p);
   if (st != L2A_OK) return st;
   if (!router || !d_mask || !q_idx || !n_routed || !prefix) return L2A_ERR_INVALID_ARG;
-  if (router_kind != L2A_ROUTER_MASK_U8 && router_kind != L2A_ROUTER_LOGITS_F32) return L2A_ERR_INVALID_ARG;
+  if (router_kind != L2A_ROUTER_MASK_U8 && router_kind != L2A_ROUTER_LOGITS_F32 &&
+      router_kind != L2A_ROUTER_LOGITS_BF16)
+    return L2A_ERR_INVALID_ARG;
   if (!aligned(q_idx, 4) || !aligned(n_routed, 4) || !aligned(prefix, 4)) return L2A_ERR_INVALID_ARG;
   if (router_kind == L2A_ROUTER_LOGITS_F32 && !aligned(router, 4)) return L2A_ERR_INVALID_ARG;
+  if (router_kind == L2A_ROUTER_LOGITS_BF16 && !aligned(router, 2)) return L2A_ERR_INVALID_ARG;
   if (!ws_ok(route_ws, route_ws_bytes, route_ws_size(p))) return L2A_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(route_ws, 0, kWsHeaderBytes, s) != cudaSuccess) return L2A_ERR_CUDA;
@@ -348,11 +351,14 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
   if (bwd && (!host->dQ || !host->dK || !host->dV || !dev->dO || !dev->dQ || !dev->dK || !dev->dV ||
               !(p->flags & L2A_FLAG_SAVE_FOR_BWD)))
     return L2A_ERR_INVALID_ARG;
-  if (router_kind != L2A_ROUTER_MASK_U8 && router_kind != L2A_ROUTER_LOGITS_F32) return L2A_ERR_INVALID_ARG;
+  if (router_kind != L2A_ROUTER_MASK_U8 && router_kind != L2A_ROUTER_LOGITS_F32 &&
+      router_kind != L2A_ROUTER_LOGITS_BF16)
+    return L2A_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t qb = (size_t)p->B * p->Lq * p->Hq * p->D * sizeof(bf16);
   const size_t kb = (size_t)p->B * p->Lk * p->Hkv * p->D * sizeof(bf16);
-  const size_t rb = (size_t)p->B * p->Lq * (router_kind == L2A_ROUTER_MASK_U8 ? 1 : 4);
+  const size_t rb = (size_t)p->B * p->Lq *
+                    (router_kind == L2A_ROUTER_MASK_U8 ? 1 : router_kind == L2A_ROUTER_LOGITS_BF16 ? 2 : 4);
   // Two helper streams (created once per host thread and device) overlap the transfers with the kernels:
   // dO is uploaded while the forward runs, O is downloaded while the backward runs, dQ while the dK/dV kernel
   // runs (the backward computes dQ first for this reason); only dK and dV, the small results, leave after the

@@ -33,6 +33,10 @@ __device__ __forceinline__ uint32_t load_flags(const void* router, int kind, flo
       for (int i = 0; i < kPerThread; ++i)
         if (t0 + i < L && m[t0 + i]) flags |= 1u << i;
     }
+  } else if (kind == L2A_ROUTER_LOGITS_BF16) {
+    const bf16* z = static_cast<const bf16*>(router) + row_base;
+    for (int i = 0; i < kPerThread; ++i)
+      if (t0 + i < L && __bfloat162float(z[t0 + i]) >= thr) flags |= 1u << i;   // the upcast is exact
   } else {
     const float* z = static_cast<const float*>(router) + row_base;
     for (int i = 0; i < kPerThread; ++i)
@@ -282,11 +286,14 @@ extern "C" l2a_status l2a_route_compact_static(const l2a_params* p, const void* 
   l2a_status st = l2a_workspace_bytes(p, &unused, nullptr, nullptr);
   if (st != L2A_OK) return st;
   if (!router || !d_mask || !q_idx || !n_routed || !prefix) return L2A_ERR_INVALID_ARG;
-  if (router_kind != L2A_ROUTER_MASK_U8 && router_kind != L2A_ROUTER_LOGITS_F32) return L2A_ERR_INVALID_ARG;
+  if (router_kind != L2A_ROUTER_MASK_U8 && router_kind != L2A_ROUTER_LOGITS_F32 &&
+      router_kind != L2A_ROUTER_LOGITS_BF16)
+    return L2A_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(q_idx) | reinterpret_cast<uintptr_t>(n_routed) |
        reinterpret_cast<uintptr_t>(prefix)) & 3)
     return L2A_ERR_INVALID_ARG;
   if (router_kind == L2A_ROUTER_LOGITS_F32 && (reinterpret_cast<uintptr_t>(router) & 3)) return L2A_ERR_INVALID_ARG;
+  if (router_kind == L2A_ROUTER_LOGITS_BF16 && (reinterpret_cast<uintptr_t>(router) & 1)) return L2A_ERR_INVALID_ARG;
   const int nblocks = l2a::ceil_div(p->Lq, l2a::kRouteBlockElems);
   if ((int64_t)p->B * nblocks > L2A_STATIC_ROUTE_SLOTS) return L2A_ERR_UNSUPPORTED;  // beyond the fixed scratch
   int32_t* counts = static_counts_for_current_device();

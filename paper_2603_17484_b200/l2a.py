@@ -23,6 +23,7 @@ FLAG_FORCE_ALL_GLOBAL = 8
 FLAG_GLOBAL_PHASE = 16
 ROUTER_MASK_U8 = 0
 ROUTER_LOGITS_F32 = 1
+ROUTER_LOGITS_BF16 = 2
 
 EXPORTS = (
     "l2a_version", "l2a_status_string", "l2a_workspace_bytes", "l2a_workspace_status",

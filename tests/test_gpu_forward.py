@@ -48,6 +48,33 @@ def test_route_compact_logits_bit_exact():
     assert list(d[0, :8]) == [0, 0, 0, 0, 0, 1, 0, 0]  # thr = 0.25
 
 
+def test_route_compact_bf16_logits_bit_exact():
+    """bf16 logits are compared in fp32 after an exact upcast: the reference is the fp32 route on the upcast values."""
+    B, L = 3, 9001
+    z = torch.from_numpy(synth.router_logits(B, L, -0.8416, seed=5)).to(torch.bfloat16)
+    z[0, :6] = torch.tensor([0.0, -0.0, float("nan"), float("inf"), -float("inf"), 0.25], dtype=torch.bfloat16)
+    z32 = z.float().numpy()
+    for thr in (0.0, 0.25):
+        d = oracle.route(z32, thr)
+        p = l2a.params(B, L, L, 2, 1, 64, 8)
+        buf = l2a.Buffers.allocate(p, router_dtype=torch.bfloat16)
+        buf.router.copy_(z)
+        buf.route(l2a.ROUTER_LOGITS_BF16, thr)
+        torch.cuda.synchronize()
+        q_idx, n, prefix = oracle.compact(d)
+        assert np.array_equal(buf.d_mask.cpu().numpy(), d)
+        assert np.array_equal(buf.q_idx.cpu().numpy(), q_idx)
+        assert np.array_equal(buf.n_routed.cpu().numpy(), n)
+        assert np.array_equal(buf.prefix.cpu().numpy(), prefix)
+    assert 0.1 < d.mean() < 0.3
+    # the allocation-free entry point takes the same kinds
+    buf.d_mask.zero_()
+    l2a.l2a_route_compact_static(p, buf.router, l2a.ROUTER_LOGITS_BF16, 0.25, buf.d_mask, buf.q_idx, buf.n_routed,
+                                 buf.prefix)
+    torch.cuda.synchronize()
+    assert np.array_equal(buf.d_mask.cpu().numpy(), d)
+
+
 # ------------------------------------------------------------------------------- forward, element by element
 
 def test_forward_tiny_config_full():
