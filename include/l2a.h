@@ -75,6 +75,14 @@ typedef struct l2a_params {
   int32_t q_pos_offset; /* p = t + q_pos_offset; pass Lk - Lq for bottom-right aligned causality  */
   float softmax_scale;  /* scores are softmax_scale * q.k ; pass 0 for the default 1/sqrt(D)      */
   uint32_t flags;       /* L2A_FLAG_*                                                             */
+  /* Optional strides, in elements, of the [B, L, H, D] tensors: {batch stride, token stride}; the heads of
+   * a token and the D values of a head stay contiguous (head stride = D).  {0, 0} = dense.  Both must be
+   * multiples of 8 (16 bytes), token stride >= H * D, batch stride >= L * token stride.  This is the layout of
+   * slices of a fused QKV projection output [B, L, (Hq + 2 Hkv) * D].  q_stride applies to Q and dQ, k_stride to
+   * K and dK, v_stride to V and dV, o_stride to O, dO and dS_loc.  S_save, A_c and the workspaces are always
+   * dense.  l2a_step_host, l2a_router_backward and the q / O arguments of l2a_decode take dense tensors only
+   * (L2A_ERR_UNSUPPORTED otherwise). */
+  int64_t q_stride[2], k_stride[2], v_stride[2], o_stride[2];
 } l2a_params;
 
 /* Version / capability string of the loaded library (host pointer, static storage). */

@@ -72,7 +72,7 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const bf16* __restrict__
                                                         const uint8_t* __restrict__ d_mask,
                                                         const int32_t* __restrict__ prefix, float* __restrict__ delta_loc,
                                                         float* __restrict__ delta_glb, float* __restrict__ dgate, int B,
-                                                        int L, int Hq, int a_by_row) {
+                                                        int L, int Hq, int a_by_row, int64_t do_bs, int64_t do_ts) {
   constexpr int kLanesPerHead = D / 8;                 // 16-byte chunks per head row
   constexpr int kHeadsPerPass = 32 / kLanesPerHead;
   const int lane = threadIdx.x & 31;
@@ -89,10 +89,11 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const bf16* __restrict__
     const int c = routed ? prefix[(int64_t)b * (L + 1) + t] : 0;
     // a_by_row: the global output was computed for every token and A is indexed by row (forced-global iterations)
     const bool with_a = routed || a_by_row;
-    const int64_t row = token * Hq * D;
+    const int64_t row = token * Hq * D;                          // S: dense
+    const int64_t orow = b * do_bs + t * do_ts;                  // dO, dO_loc: the strides of O
     const int64_t crow = ((int64_t)b * L + (a_by_row ? t : c)) * Hq * D;
-    const uint4* po = reinterpret_cast<const uint4*>(dO + row) + lane;
-    const uint4* pl = reinterpret_cast<const uint4*>(dO_loc + row) + lane;
+    const uint4* po = reinterpret_cast<const uint4*>(dO + orow) + lane;
+    const uint4* pl = reinterpret_cast<const uint4*>(dO_loc + orow) + lane;
     const uint4* ps = reinterpret_cast<const uint4*>(S + row) + lane;
     const uint4* pa = reinterpret_cast<const uint4*>(A_c + crow) + lane;
     float gate = 0.f;
@@ -144,6 +145,7 @@ struct BwdArgs {
   int global_mode;  // dq kernel only
   int skip_local, skip_global;   // gradients of one module only (the other module has its own Q/K/V)
   int kb_begin, kb_count;        // dK/dV kernel: key blocks [kb_begin, kb_begin + kb_count) of every KV head
+  RowStrides dq_st, dk_st, dv_st;   // strides of the gradient tensors in elements
   const int32_t* q_idx;
   const int32_t* n_routed;
   const int32_t* prefix;
@@ -431,7 +433,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     if (ok && __all_sync(0xffffffffu, mbar_wait(&bar->final_bar, 0, abort_flag))) {
       tc_fence_after();
       constexpr int kCols = D / 4;     // 32 (D = 128) or 16 (D = 64)
-      bf16* dst = valid ? a.dQ + (((int64_t)b * a.Lq + seq_row) * a.Hq + h) * D + q * kCols : nullptr;
+      bf16* dst = valid ? a.dQ + b * a.dq_st.b + seq_row * a.dq_st.t + (int64_t)h * D + q * kCols : nullptr;
       uint32_t v[32];
       tmem_ld32(tmem + lane_base + (q * kCols & ~31), v);   // D = 64: quarters 0,1 / 2,3 share a 32-column load
       tmem_ld_wait();
@@ -580,9 +582,9 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     for (int i = tid; i < kTileN * (D / 8); i += blockDim.x) {
       const int kr = i / (D / 8), c8 = i % (D / 8);
       if (k0 + kr < a.Lk) {
-        const int64_t o = (((int64_t)b * a.Lk + k0 + kr) * a.Hkv + g) * D + c8 * 8;
-        *reinterpret_cast<uint4*>(a.dK + o) = make_uint4(0, 0, 0, 0);
-        *reinterpret_cast<uint4*>(a.dV + o) = make_uint4(0, 0, 0, 0);
+        const int64_t o = (int64_t)g * D + c8 * 8;
+        *reinterpret_cast<uint4*>(a.dK + b * a.dk_st.b + (k0 + kr) * a.dk_st.t + o) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(a.dV + b * a.dv_st.b + (k0 + kr) * a.dv_st.t + o) = make_uint4(0, 0, 0, 0);
       }
     }
     return;
@@ -882,7 +884,8 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       tc_fence_after();
       const bool valid = kp < a.Lk;
       const int which = q >> 1, half = q & 1;
-      const int64_t o = (((int64_t)b * a.Lk + (valid ? kp : 0)) * a.Hkv + g) * D + half * (D / 2);
+      const RowStrides st = which == 0 ? a.dv_st : a.dk_st;
+      const int64_t o = b * st.b + (valid ? kp : 0) * st.t + (int64_t)g * D + half * (D / 2);
       bf16* dst = (which == 0 ? a.dV : a.dK) + o;
       const float mul = which == 0 ? 1.0f : a.scale;
 #pragma unroll
@@ -938,8 +941,11 @@ cudaError_t launch_bwd_kernels(const BwdArgs& base, const CUtensorMap& mapQ, con
     bwd_dq_kernel<D><<<n_tiles * base.B * base.Hq, kDqThreads, DqSmem<D>::kTotal, s>>>(mapQ, mapDO, mapK, mapV, a);
   } else {
     // the global launch adds into dQ at the routed positions: every other row of dQ is zero
-    e = cudaMemsetAsync(base.dQ, 0, (size_t)base.B * base.Lq * base.Hq * D * sizeof(bf16), s);
-    if (e != cudaSuccess) return e;
+    for (int b = 0; b < base.B; ++b) {
+      e = cudaMemset2DAsync(base.dQ + b * base.dq_st.b, (size_t)base.dq_st.t * sizeof(bf16), 0,
+                            (size_t)base.Hq * D * sizeof(bf16), base.Lq, s);
+      if (e != cudaSuccess) return e;
+    }
   }
   phase_events().mark(s);
   a.global_mode = 1;
@@ -1019,23 +1025,27 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   float* lse_c = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + 2 * stat_bytes(p));
 
   CUtensorMap mapQ, mapDO, mapQc, mapDOc, mapK, mapV;
-  if (!encode_rows_map(&mapQ, Q, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||
-      !encode_rows_map(&mapDO, dS_loc, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||   // local items: dL/ds_t
+  const RowStrides qs = resolve_strides(p->q_stride, p->Lq, p->Hq * p->D);
+  const RowStrides ks = resolve_strides(p->k_stride, p->Lk, p->Hkv * p->D);
+  const RowStrides vs = resolve_strides(p->v_stride, p->Lk, p->Hkv * p->D);
+  const RowStrides os = resolve_strides(p->o_stride, p->Lq, p->Hq * p->D);
+  if (!encode_rows_map(&mapQ, Q, p->B, p->Lq, p->Hq * p->D, kTileM, p->D, qs.b, qs.t) ||
+      !encode_rows_map(&mapDO, dS_loc, p->B, p->Lq, p->Hq * p->D, kTileM, p->D, os.b, os.t) ||   // local items: dL/ds_t
       !encode_rows_map(&mapQc, Qc, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||
       !encode_rows_map(&mapDOc, dOc, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||
-      !encode_rows_map(&mapK, K, p->B, p->Lk, p->Hkv * p->D, kTileN, p->D) ||
-      !encode_rows_map(&mapV, V, p->B, p->Lk, p->Hkv * p->D, kTileN, p->D))
+      !encode_rows_map(&mapK, K, p->B, p->Lk, p->Hkv * p->D, kTileN, p->D, ks.b, ks.t) ||
+      !encode_rows_map(&mapV, V, p->B, p->Lk, p->Hkv * p->D, kTileN, p->D, vs.b, vs.t))
     return L2A_ERR_CUDA;
 
   PhaseEvents& pe = phase_events();
   struct ClearOnExit { PhaseEvents& p; ~ClearOnExit() { p.clear(); } } clear_on_exit{pe};
   pe.mark(s);
   if (!skip_global) {
-    if (launch_gather_rows(static_cast<const bf16*>(Q), Qc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s) !=
-        cudaSuccess)
+    if (launch_gather_rows(static_cast<const bf16*>(Q), Qc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s, nullptr, 0,
+                           0, qs) != cudaSuccess)
       return L2A_ERR_CUDA;
-    if (launch_gather_rows(static_cast<const bf16*>(dO), dOc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s) !=
-        cudaSuccess)
+    if (launch_gather_rows(static_cast<const bf16*>(dO), dOc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s, nullptr,
+                           0, 0, os) != cudaSuccess)
       return L2A_ERR_CUDA;
   }
   pe.mark(s);
@@ -1052,7 +1062,7 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
                                           static_cast<const bf16*>(skip_local ? nullptr : S_save),
                                           static_cast<const bf16*>(A_c), skip_global ? nullptr : d_mask, prefix,
                                           delta_loc, delta_glb, dgate, p->B, p->Lq, p->Hq,
-                                          force_all ? 1 : 0);
+                                          force_all ? 1 : 0, os.b, os.t);
     if (cudaGetLastError() != cudaSuccess) return L2A_ERR_CUDA;
     if (force_all) {
       dim3 grid((p->Lq + 255) / 256, p->Hq, p->B);
@@ -1073,6 +1083,7 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   a.q_idx = q_idx; a.n_routed = n_routed; a.prefix = prefix;
   a.lse_loc = lse_loc; a.lse_glb = force_all ? lse_c : lse_glb; a.delta_loc = delta_loc; a.delta_glb = delta_glb;
   a.dQ = static_cast<bf16*>(dQ); a.dK = static_cast<bf16*>(dK); a.dV = static_cast<bf16*>(dV);
+  a.dq_st = qs; a.dk_st = ks; a.dv_st = vs;
   a.status = reinterpret_cast<int*>(ws);
   cudaError_t e = p->D == 128 ? launch_bwd_kernels<128>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, s)
                               : launch_bwd_kernels<64>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, s);

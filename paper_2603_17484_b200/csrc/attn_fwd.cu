@@ -426,13 +426,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             const float lse = (m_use + log2f(l)) * 0.6931471805599453f;
             a.lse[((int64_t)b * a.Hq + h) * a.Lq + row] = lse;
           }
-          const int64_t row_stride = (int64_t)a.Hq * D;
           bf16* dst1 = nullptr;   // row-indexed destination (s rows, or compact a rows)
           bf16* dst2 = nullptr;   // position-indexed destination
           if (valid) {
-            if (a.out) dst1 = a.out + ((int64_t)b * a.Lq + row) * row_stride + (int64_t)h * D + hf * (D / 2);
+            if (a.out) dst1 = a.out + b * a.out_st.b + row * a.out_st.t + (int64_t)h * D + hf * (D / 2);
             if (a.out2 && (a.combine_mask == nullptr || a.combine_mask[(int64_t)b * a.Lq + seq_row]))
-              dst2 = a.out2 + ((int64_t)b * a.Lq + seq_row) * row_stride + (int64_t)h * D + hf * (D / 2);
+              dst2 = a.out2 + b * a.out2_st.b + seq_row * a.out2_st.t + (int64_t)h * D + hf * (D / 2);
           }
           const bool accumulate = a.global_mode && a.accumulate_into_out2;
 #pragma unroll

@@ -346,8 +346,11 @@ extern "C" l2a_status l2a_decode(const l2a_params* p, const void* q, const void*
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, s) != cudaSuccess) return L2A_ERR_CUDA;
   CUtensorMap mapK, mapV;
-  if (!encode_rows_map(&mapK, K, p->B, p->Lk, p->Hkv * p->D, kDecKeys, p->D) ||
-      !encode_rows_map(&mapV, V, p->B, p->Lk, p->Hkv * p->D, kDecKeys, p->D))
+  if (!is_dense(p->q_stride, p->Lq, p->Hq * p->D) || !is_dense(p->o_stride, p->Lq, p->Hq * p->D)) return L2A_ERR_UNSUPPORTED;
+  const RowStrides ks = resolve_strides(p->k_stride, p->Lk, p->Hkv * p->D);
+  const RowStrides vs = resolve_strides(p->v_stride, p->Lk, p->Hkv * p->D);
+  if (!encode_rows_map(&mapK, K, p->B, p->Lk, p->Hkv * p->D, kDecKeys, p->D, ks.b, ks.t) ||
+      !encode_rows_map(&mapV, V, p->B, p->Lk, p->Hkv * p->D, kDecKeys, p->D, vs.b, vs.t))
     return L2A_ERR_CUDA;
   DecodeArgs a;
   a.B = p->B; a.Lk = p->Lk; a.Hq = p->Hq; a.Hkv = p->Hkv; a.G = p->Hq / p->Hkv;

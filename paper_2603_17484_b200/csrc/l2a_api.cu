@@ -36,6 +36,9 @@ l2a_status check_params(const l2a_params* p) {
   if (!(p->softmax_scale >= 0.f) || isinf(p->softmax_scale)) return L2A_ERR_INVALID_ARG;
   if ((int64_t)p->B * p->Lq >= (1ll << 31) || (int64_t)p->B * p->Lk >= (1ll << 31)) return L2A_ERR_INVALID_ARG;
   if (p->D != 64 && p->D != 128) return L2A_ERR_UNSUPPORTED;
+  if (!strides_ok(p->q_stride, p->Lq, p->Hq * p->D) || !strides_ok(p->k_stride, p->Lk, p->Hkv * p->D) ||
+      !strides_ok(p->v_stride, p->Lk, p->Hkv * p->D) || !strides_ok(p->o_stride, p->Lq, p->Hq * p->D))
+    return L2A_ERR_INVALID_ARG;
   return L2A_OK;
 }
 
@@ -58,14 +61,16 @@ PhaseEvents& phase_events() {
 }
 
 bool encode_rows_map(CUtensorMap* map, const void* base, int batch, int rows, int row_elems, int box_rows,
-                     int head_dim) {
+                     int head_dim, int64_t batch_stride, int64_t token_stride) {
   encode_tiled_fn enc = get_encode();
   if (!enc) return false;
   // [batch, rows, row_elems] seen as {64 elements, rows, row_elems / 64 column chunks, batch}: one copy of a
   // {64, box_rows, head_dim / 64, 1} box lands in shared memory as head_dim / 64 consecutive 128-byte-swizzled
   // sub-tiles of box_rows x 64 elements -- the layout the MMA operand descriptors address.
   cuuint64_t dims[4] = {64, (cuuint64_t)rows, (cuuint64_t)(row_elems / 64), (cuuint64_t)batch};
-  cuuint64_t strides[3] = {(cuuint64_t)row_elems * 2, 128, (cuuint64_t)rows * row_elems * 2};
+  const int64_t ts = token_stride > 0 ? token_stride : row_elems;
+  const int64_t bs = batch_stride > 0 ? batch_stride : (int64_t)rows * ts;
+  cuuint64_t strides[3] = {(cuuint64_t)ts * 2, 128, (cuuint64_t)bs * 2};
   cuuint32_t box[4] = {64, (cuuint32_t)box_rows, (cuuint32_t)(head_dim / 64), 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
@@ -199,9 +204,14 @@ static l2a_status forward_range(const l2a_params* p, const void* Q, const void* 
   if (clear_status && cudaMemsetAsync(ws, 0, kWsHeaderBytes, s) != cudaSuccess) return L2A_ERR_CUDA;
 
   CUtensorMap mapQ, mapK, mapV, mapQc;
-  if (!encode_rows_map(&mapQ, Q, p->B, p->Lq, p->Hq * p->D, kTileM, p->D) ||
-      !encode_rows_map(&mapK, K, p->B, p->Lk, p->Hkv * p->D, kTileN, p->D) ||
-      !encode_rows_map(&mapV, V, p->B, p->Lk, p->Hkv * p->D, kTileN, p->D) ||
+  const RowStrides qs = resolve_strides(p->q_stride, p->Lq, p->Hq * p->D);
+  const RowStrides ks = resolve_strides(p->k_stride, p->Lk, p->Hkv * p->D);
+  const RowStrides vs = resolve_strides(p->v_stride, p->Lk, p->Hkv * p->D);
+  const RowStrides os = resolve_strides(p->o_stride, p->Lq, p->Hq * p->D);
+  const RowStrides dense_q = {(int64_t)p->Lq * p->Hq * p->D, (int64_t)p->Hq * p->D};
+  if (!encode_rows_map(&mapQ, Q, p->B, p->Lq, p->Hq * p->D, kTileM, p->D, qs.b, qs.t) ||
+      !encode_rows_map(&mapK, K, p->B, p->Lk, p->Hkv * p->D, kTileN, p->D, ks.b, ks.t) ||
+      !encode_rows_map(&mapV, V, p->B, p->Lk, p->Hkv * p->D, kTileN, p->D, vs.b, vs.t) ||
       !encode_rows_map(&mapQc, Qc, p->B, p->Lq, p->Hq * p->D, kTileM, p->D))
     return L2A_ERR_CUDA;
 
@@ -226,7 +236,7 @@ static l2a_status forward_range(const l2a_params* p, const void* Q, const void* 
   if (!skip_global && !force_all) {
     // consolidate routed query rows (Algorithm 1, step 1); independent of the local pass
     if (launch_gather_rows(static_cast<const bf16*>(Q), Qc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s,
-                           row_range ? prefix : nullptr, row_begin, row_end) != cudaSuccess)
+                           row_range ? prefix : nullptr, row_begin, row_end, qs) != cudaSuccess)
       return L2A_ERR_CUDA;
   }
   pe.mark(s);
@@ -235,6 +245,8 @@ static l2a_status forward_range(const l2a_params* p, const void* Q, const void* 
     a.accumulate_into_out2 = 0;
     a.out = static_cast<bf16*>(save ? S_save : O);
     a.out2 = save ? static_cast<bf16*>(O) : nullptr;
+    a.out_st = save ? dense_q : os;
+    a.out2_st = os;
     a.lse = lse_loc;
     a.pair_begin = pair_begin;
     a.pair_end = pair_end;
@@ -242,8 +254,11 @@ static l2a_status forward_range(const l2a_params* p, const void* Q, const void* 
     a.pair_begin = 0;
     a.pair_end = n_pairs;
   } else if (skip_local) {
-    const size_t bytes = (size_t)p->B * p->Lq * p->Hq * p->D * sizeof(bf16);
-    if (cudaMemsetAsync(O, 0, bytes, s) != cudaSuccess) return L2A_ERR_CUDA;  // Algorithm 1: O starts at zero
+    // Algorithm 1: O starts at zero (row by row when O is strided)
+    for (int b = 0; b < p->B; ++b)
+      if (cudaMemset2DAsync(static_cast<bf16*>(O) + b * os.b, (size_t)os.t * sizeof(bf16), 0,
+                            (size_t)p->Hq * p->D * sizeof(bf16), p->Lq, s) != cudaSuccess)
+        return L2A_ERR_CUDA;
   }
   pe.mark(s);
   if (!skip_global) {
@@ -251,6 +266,8 @@ static l2a_status forward_range(const l2a_params* p, const void* Q, const void* 
     a.accumulate_into_out2 = skip_local ? 0 : 1;
     a.out = static_cast<bf16*>(A_c);
     a.out2 = static_cast<bf16*>(O);
+    a.out_st = dense_q;
+    a.out2_st = os;
     a.lse = lse_glb;
     if (force_all) {
       // Global Attention for every token (Section 3.3): same kernel over all rows in place; a_t is stored for
@@ -285,6 +302,7 @@ l2a_status l2a_router_backward(const l2a_params* p, const void* S, const float* 
   if (st != L2A_OK) return st;
   if (!S || !w || !logits) return L2A_ERR_INVALID_ARG;
   if ((dO == nullptr) != (dS_loc == nullptr)) return L2A_ERR_INVALID_ARG;   // the combined gradient needs both
+  if (dO != nullptr && !is_dense(p->o_stride, p->Lq, p->Hq * p->D)) return L2A_ERR_UNSUPPORTED;
   if (!aligned(S, 16) || !aligned(w, 16) || !aligned(dO, 16) || !aligned(dS_loc, 16) || !aligned(logits, 4) ||
       !aligned(dgate, 4) || !aligned(dz, 4) || !aligned(dw, 4) || !aligned(dbias, 4))
     return L2A_ERR_INVALID_ARG;
@@ -354,6 +372,9 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
   if (router_kind != L2A_ROUTER_MASK_U8 && router_kind != L2A_ROUTER_LOGITS_F32 &&
       router_kind != L2A_ROUTER_LOGITS_BF16)
     return L2A_ERR_INVALID_ARG;
+  if (!is_dense(p->q_stride, p->Lq, p->Hq * p->D) || !is_dense(p->k_stride, p->Lk, p->Hkv * p->D) ||
+      !is_dense(p->v_stride, p->Lk, p->Hkv * p->D) || !is_dense(p->o_stride, p->Lq, p->Hq * p->D))
+    return L2A_ERR_UNSUPPORTED;     // host buffers and their device mirrors are dense
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t qb = (size_t)p->B * p->Lq * p->Hq * p->D * sizeof(bf16);
   const size_t kb = (size_t)p->B * p->Lk * p->Hkv * p->D * sizeof(bf16);

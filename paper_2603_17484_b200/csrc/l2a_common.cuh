@@ -23,7 +23,27 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // [batch, rows, heads*D] bf16 tensor so that ONE copy brings a box_rows x head_dim tile into shared memory in
 // the 128-byte-swizzled layout the MMA operand descriptors expect.  Returns false on failure.
 bool encode_rows_map(CUtensorMap* map, const void* base, int batch, int rows, int row_elems, int box_rows,
-                     int head_dim);
+                     int head_dim, int64_t batch_stride = 0, int64_t token_stride = 0);   // strides in elements; 0 = dense
+
+// Strides of a [B, L, H, D] tensor in elements ({batch, token}); heads and head values are contiguous.
+struct RowStrides {
+  int64_t b, t;
+};
+inline RowStrides resolve_strides(const int64_t (&s)[2], int L, int row_elems) {
+  RowStrides r;
+  r.t = s[1] > 0 ? s[1] : row_elems;
+  r.b = s[0] > 0 ? s[0] : (int64_t)L * r.t;
+  return r;
+}
+inline bool strides_ok(const int64_t (&s)[2], int L, int row_elems) {
+  if (s[0] < 0 || s[1] < 0) return false;
+  const RowStrides r = resolve_strides(s, L, row_elems);
+  return r.t % 8 == 0 && r.b % 8 == 0 && r.t >= row_elems && r.b >= (int64_t)L * r.t;
+}
+inline bool is_dense(const int64_t (&s)[2], int L, int row_elems) {
+  const RowStrides r = resolve_strides(s, L, row_elems);
+  return r.t == row_elems && r.b == (int64_t)L * row_elems;
+}
 
 // Launchers (each returns the CUDA error of its launch).  Defined in the kernel files.
 struct RouteArgs {
@@ -46,7 +66,7 @@ cudaError_t launch_route_compact(const RouteArgs& a, cudaStream_t stream);
 // routed rows t in [row_begin, row_end) are gathered (the padding with the range that ends at L).
 cudaError_t launch_gather_rows(const bf16* src, bf16* dst, const int32_t* q_idx, const int32_t* n_routed,
                                int B, int L, int row_elems, cudaStream_t stream, const int32_t* prefix = nullptr,
-                               int row_begin = 0, int row_end = 0);
+                               int row_begin = 0, int row_end = 0, RowStrides src_strides = RowStrides{0, 0});
 
 // z[b,t] = w . S[b,t,:] + bias (fp32 accumulation); optional sum over t of sigmoid(z)^2 per batch entry
 cudaError_t launch_router_logits(const bf16* S, const float* w, float bias, float* logits, float* sum_sq, int B,
@@ -72,6 +92,7 @@ struct FwdArgs {
   bf16* out2;   // local: optional second copy of s (NULL to skip);  global: O rows, indexed by position
   float* lse;   // local: [B,Hq,Lq] by row;  global: [B,Hq,Lq] by compact row; may be NULL
   int* status;  // workspace status word
+  RowStrides out_st, out2_st;   // strides of out / out2 in elements
   int pair_begin, pair_end;  // 256-row query groups [pair_begin, pair_end) this launch covers (all: 0 .. ceil(Lq / 256))
   int row_begin, row_end;    // global mode: only the groups whose LAST row t lies in [row_begin, row_end)
 };

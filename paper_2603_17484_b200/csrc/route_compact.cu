@@ -124,7 +124,8 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const bf16* __restrict
                                                           const int32_t* __restrict__ n_routed, int L,
                                                           int row_chunks /* 16-byte chunks per row */,
                                                           const int32_t* __restrict__ prefix, int row_begin,
-                                                          int row_end) {
+                                                          int row_end, int64_t src_batch_chunks,
+                                                          int64_t src_row_chunks) {
   const int b = blockIdx.y;
   const int n_c = n_routed[b];
   int n_pad = (n_c + kRowsPerCta - 1) / kRowsPerCta * kRowsPerCta;
@@ -136,13 +137,13 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const bf16* __restrict
     c_begin = prefix[(int64_t)b * (L + 1) + row_begin];
     if (row_end < L) n_pad = prefix[(int64_t)b * (L + 1) + row_end];
   }
-  const uint4* s = reinterpret_cast<const uint4*>(src) + (int64_t)b * L * row_chunks;
+  const uint4* s = reinterpret_cast<const uint4*>(src) + b * src_batch_chunks;   // source strides in 16-byte chunks
   uint4* d = reinterpret_cast<uint4*>(dst) + (int64_t)b * L * row_chunks;
   for (int c = c_begin + blockIdx.x; c < n_pad; c += gridDim.x) {
     if (c < n_c) {
       const int t = q_idx[(int64_t)b * L + c];
       for (int i = threadIdx.x; i < row_chunks; i += blockDim.x)
-        d[(int64_t)c * row_chunks + i] = __ldg(&s[(int64_t)t * row_chunks + i]);
+        d[(int64_t)c * row_chunks + i] = __ldg(&s[t * src_row_chunks + i]);
     } else {
       for (int i = threadIdx.x; i < row_chunks; i += blockDim.x)
         d[(int64_t)c * row_chunks + i] = make_uint4(0, 0, 0, 0);
@@ -242,11 +243,14 @@ cudaError_t launch_route_compact(const RouteArgs& a, cudaStream_t stream) {
 
 cudaError_t launch_gather_rows(const bf16* src, bf16* dst, const int32_t* q_idx, const int32_t* n_routed, int B,
                                int L, int row_elems, cudaStream_t stream, const int32_t* prefix, int row_begin,
-                               int row_end) {
+                               int row_end, RowStrides src_strides) {
   const int row_chunks = row_elems * 2 / 16;
+  const int64_t ts = src_strides.t > 0 ? src_strides.t : row_elems;
+  const int64_t bs = src_strides.b > 0 ? src_strides.b : (int64_t)L * ts;
   int gx = L < 148 * 16 ? L : 148 * 16;
   dim3 grid(gx, B);
-  gather_rows_kernel<<<grid, 256, 0, stream>>>(src, dst, q_idx, n_routed, L, row_chunks, prefix, row_begin, row_end);
+  gather_rows_kernel<<<grid, 256, 0, stream>>>(src, dst, q_idx, n_routed, L, row_chunks, prefix, row_begin, row_end,
+                                               bs / 8, ts / 8);
   return cudaGetLastError();
 }
 

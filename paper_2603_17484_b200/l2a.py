@@ -39,6 +39,8 @@ class L2AParams(ctypes.Structure):
         ("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32), ("D", ctypes.c_int32),
         ("window", ctypes.c_int32), ("q_pos_offset", ctypes.c_int32),
         ("softmax_scale", ctypes.c_float), ("flags", ctypes.c_uint32),
+        ("q_stride", ctypes.c_int64 * 2), ("k_stride", ctypes.c_int64 * 2),
+        ("v_stride", ctypes.c_int64 * 2), ("o_stride", ctypes.c_int64 * 2),
     ]
 
 
@@ -75,16 +77,21 @@ def status_string(code: int) -> str:
     return lib().l2a_status_string(code).decode()
 
 
-def params(B, Lq, Lk, Hq, Hkv, D, window, q_pos_offset=None, softmax_scale=0.0, flags=0) -> L2AParams:
+def params(B, Lq, Lk, Hq, Hkv, D, window, q_pos_offset=None, softmax_scale=0.0, flags=0, q_stride=None,
+           k_stride=None, v_stride=None, o_stride=None) -> L2AParams:
+    """Strides: optional (batch stride, token stride) in elements; None = dense (see include/l2a.h)."""
+    two = ctypes.c_int64 * 2
+    st = [two(*(s if s is not None else (0, 0))) for s in (q_stride, k_stride, v_stride, o_stride)]
     return L2AParams(B, Lq, Lk, Hq, Hkv, D, window, Lk - Lq if q_pos_offset is None else q_pos_offset,
-                     softmax_scale, flags)
+                     softmax_scale, flags, *st)
 
 
 def _ptr(t):
     if t is None:
         return ctypes.c_void_p(0)
     if isinstance(t, torch.Tensor):
-        assert t.is_contiguous(), "tensors passed to the C ABI must be contiguous"
+        # strided views (slices of a fused buffer) are described by the strides in L2AParams; only the base
+        # address is passed
         return ctypes.c_void_p(t.data_ptr())
     return ctypes.c_void_p(int(t))
 

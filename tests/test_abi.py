@@ -57,4 +57,19 @@ def test_workspace_sizes_and_validation(lib):
 
 
 def test_params_struct_layout_matches_header():
-    assert ctypes.sizeof(l2a.L2AParams) == 40
+    # ten 32-bit fields, then four {batch, token} stride pairs of 64-bit integers
+    assert ctypes.sizeof(l2a.L2AParams) == 40 + 4 * 2 * 8
+    assert l2a.L2AParams.q_stride.offset == 40 and l2a.L2AParams.o_stride.offset == 88
+
+
+def test_stride_arguments_are_validated_on_the_host():
+    ok = dict(B=2, Lq=256, Lk=256, Hq=4, Hkv=2, D=128, window=16)
+    row = 4 * 128
+    l2a.l2a_workspace_bytes(l2a.params(**ok, q_stride=(256 * 2 * row, 2 * row)))          # a slice of a wider buffer
+    for bad in ((0, row + 4),            # not a multiple of 8 elements
+                (0, row - 8),            # rows overlap
+                (255 * row, row),        # batches overlap
+                (-8, row)):
+        with pytest.raises(l2a.L2AError) as e:
+            l2a.l2a_workspace_bytes(l2a.params(**ok, q_stride=bad))
+        assert e.value.code == -1
