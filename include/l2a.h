@@ -56,6 +56,15 @@ typedef enum {
                                   /* the routed rows' global attention runs and is added into O.       */
                                   /* Lets the caller compute the router decision from S in between     */
                                   /* (Eq. 2 -> 3 -> 4 -> 5 in the order the layer defines them).       */
+#define L2A_FLAG_FUSED_DQ 32u      /* backward, experimental: five GEMMs per tile pair instead of seven -- dQ is  */
+                                  /* produced inside the dK/dV kernel and summed in an fp32 buffer with atomic   */
+                                  /* reductions, then rounded to bf16.  Same tolerance as the default path; dK   */
+                                  /* and dV are bit-identical to it, dQ is not bit-reproducible from run to run. */
+                                  /* The backward workspace grows by B * Lq * Hq * D * 4 bytes (pass the same    */
+                                  /* flags to l2a_workspace_bytes).  Not combined with L2A_FLAG_SKIP_LOCAL,        */
+                                  /* L2A_FLAG_SKIP_GLOBAL or L2A_FLAG_FORCE_ALL_GLOBAL (invalid argument).  On   */
+                                  /* B200 the reductions' L2 traffic makes it slower than the default at long    */
+                                  /* sequences, so it is off by default.                                         */
 #define L2A_FLAG_FORCE_ALL_GLOBAL 8u /* training iterations that invoke Global Attention for every    */
                                   /* token regardless of d_t (Section 3.3: done with a small       */
                                   /* probability so that masked tokens' routers get a gradient).   */

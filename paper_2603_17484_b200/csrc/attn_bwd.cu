@@ -146,6 +146,7 @@ struct BwdArgs {
   int skip_local, skip_global;   // gradients of one module only (the other module has its own Q/K/V)
   int kb_begin, kb_count;        // dK/dV kernel: key blocks [kb_begin, kb_begin + kb_count) of every KV head
   RowStrides dq_st, dk_st, dv_st;   // strides of the gradient tensors in elements
+  float* dq_acc;                 // fused mode: fp32 [B, Lq, Hq, D] accumulator of dQ
   const int32_t* q_idx;
   const int32_t* n_routed;
   const int32_t* prefix;
@@ -918,6 +919,472 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   if (warp == 17) tmem_dealloc(tmem, 512);
 }
 
+// ================================================================================================
+// Fused backward kernel (L2A_FLAG_FUSED_DQ): the dK/dV kernel above plus the fifth GEMM, dQ(i) = dS(i) K, so that S and
+// dP are computed once (five GEMMs per tile pair instead of seven).  dQ(i) is a fresh 128 x D accumulator per item:
+// it borrows the S^T columns (S^T(i) is in registers by then), is read out by the compute warps (lane = query row)
+// and added to an fp32 dQ buffer in global memory with red.global.add.v4.f32 -- local and global contributions
+// and all key blocks meet there, in no fixed order, so dQ is not bit-reproducible from run to run in this mode.
+// dS is needed twice: transposed in TMEM (A operand of dK, as above) and in shared memory, [key][query], read
+// MN-major as the A operand of dQ; it takes the place of the third Q stage.
+//   TMEM: dV [0,D) | dK [D,2D) | T [256,384): S^T(i), then dQ(i) | U [384,512): dP^T(i), then P^T(i) | dS^T(i).
+//   MMA order per item i:  dQ(i) | dV(i) | dK(i) | S^T(i+1) (after dQ(i) was read out) | dP^T(i+1).
+template <int D>
+struct FusedSmem {
+  static constexpr int kTileBytes = 128 * D * 2;
+  static constexpr int kKOff = 0;
+  static constexpr int kVOff = kTileBytes;
+  static constexpr int kQOff = 2 * kTileBytes;                 // 2 stages
+  static constexpr int kDoOff = kQOff + 2 * kTileBytes;        // 2 stages
+  static constexpr int kDsOff = kDoOff + 2 * kTileBytes;       // dS: 128 keys x 128 queries bf16
+  static constexpr int kStatOff = kDsOff + 128 * 128 * 2;
+  static constexpr int kStatSlot = (2 * 128 + 8) * 4;
+  static constexpr int kBarOff = kStatOff + 2 * kStatSlot;
+  static constexpr int kTotal = kBarOff + 256;
+};
+struct FusedBarriers {
+  uint64_t kv_full;
+  uint64_t q_full[2], q_empty[2];
+  uint64_t do_full[2], do_empty[2];
+  uint64_t st_full[2], st_empty[2];
+  uint64_t s_full, dp_full, pds_full, dq_full, t_free, final_bar;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kDkvThreads, 1)
+bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapDO,
+               const __grid_constant__ CUtensorMap mapQc, const __grid_constant__ CUtensorMap mapDOc,
+               const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, const BwdArgs a) {
+  using SM = FusedSmem<D>;
+  constexpr int kKSteps = D / 16;
+  // key blocks ascending (most work first) inside one KV head; KV heads outermost so that the CTAs
+  // running together share the same query tiles in L2
+  const int j = a.kb_begin + blockIdx.x % a.kb_count;
+  const int rest = blockIdx.x / a.kb_count;
+  const int b = rest % a.B;
+  const int g = rest / a.B;
+  const int G = a.Hq / a.Hkv;
+  const int k0 = j * kTileN;
+  const ItemPlan plan = make_plan(a, b, k0);
+  const int n_c = a.skip_global ? 0 : a.n_routed[b];   // the routing arrays may be NULL when the global part is skipped
+
+  extern __shared__ __align__(1024) uint8_t smem[];
+  uint8_t* sK = smem + SM::kKOff;
+  uint8_t* sV = smem + SM::kVOff;
+  uint8_t* sQ = smem + SM::kQOff;
+  uint8_t* sDO = smem + SM::kDoOff;
+  FusedBarriers* bar = reinterpret_cast<FusedBarriers*>(smem + SM::kBarOff);
+  uint8_t* sDS = smem + SM::kDsOff;          // dS (bf16, [key][query]) for dQ = dS K
+  volatile int* abort_flag = &bar->abort_flag;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  if ((smem_u32(smem) & 1023u) != 0) {   // the swizzled tiles need a 1024-byte aligned base: refuse to run otherwise
+    if (tid == 0) atomicExch(a.status, 2);
+    return;
+  }
+  if (plan.total == 0) {
+    // no query can see these keys: their gradients are zero
+    for (int i = tid; i < kTileN * (D / 8); i += blockDim.x) {
+      const int kr = i / (D / 8), c8 = i % (D / 8);
+      if (k0 + kr < a.Lk) {
+        const int64_t o = (int64_t)g * D + c8 * 8;
+        *reinterpret_cast<uint4*>(a.dK + b * a.dk_st.b + (k0 + kr) * a.dk_st.t + o) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(a.dV + b * a.dv_st.b + (k0 + kr) * a.dv_st.t + o) = make_uint4(0, 0, 0, 0);
+      }
+    }
+    return;
+  }
+
+  if (tid == 0) {
+    mbar_init(&bar->kv_full, 1);
+    for (int s = 0; s < 2; ++s) { mbar_init(&bar->q_full[s], 1); mbar_init(&bar->q_empty[s], 1); }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&bar->do_full[s], 1); mbar_init(&bar->do_empty[s], 1);
+      mbar_init(&bar->st_full[s], 32); mbar_init(&bar->st_empty[s], kComputeWarps * 32);
+    }
+    mbar_init(&bar->s_full, 1);
+    mbar_init(&bar->dp_full, 1);
+    mbar_init(&bar->pds_full, kComputeWarps * 32);   // P^T, dS^T in TMEM and dS in shared memory
+    mbar_init(&bar->dq_full, 1);                     // dQ(i) is in TMEM
+    mbar_init(&bar->t_free, kComputeWarps * 32);     // dQ(i) has been read out: the columns may take S^T(i+1)
+    mbar_init(&bar->final_bar, 1);
+    bar->abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 17) { tmem_alloc(&bar->tmem_base, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bar->tmem_base;
+  if (tmem != 0) {
+    // all 512 columns were requested, so the allocation must start at column 0; the MMA warp relies on it to
+    // keep its TMEM operand addresses compile-time constants
+    __syncthreads();
+    if (warp == 17) tmem_dealloc(tmem, 512);
+    if (tid == 0) atomicExch(a.status, 3);
+    return;
+  }
+
+  if (warp == 16) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&mapQ); tma_prefetch_desc(&mapDO); tma_prefetch_desc(&mapQc); tma_prefetch_desc(&mapDOc);
+      mbar_expect_tx(&bar->kv_full, 2 * SM::kTileBytes);
+      tma_load_4d(sK, &mapK, &bar->kv_full, 0, k0, g * (D / 64), b);
+      tma_load_4d(sV, &mapV, &bar->kv_full, 0, k0, g * (D / 64), b);
+      ItemCursor cur(plan, g * G);
+      int qs = 0;
+      uint32_t qph = 0;
+      for (int i = 0; i < plan.total; ++i) {
+        const int glb = cur.glb(), row0 = cur.tile() * kTileM, hc = cur.h * (D / 64);
+        cur.next();
+        if (!mbar_wait(&bar->q_empty[qs], qph ^ 1, abort_flag)) break;
+        mbar_expect_tx(&bar->q_full[qs], SM::kTileBytes);
+        tma_load_4d(sQ + qs * SM::kTileBytes, glb ? &mapQc : &mapQ, &bar->q_full[qs], 0, row0, hc, b);
+        if (!mbar_wait(&bar->do_empty[i & 1], ((i >> 1) & 1) ^ 1, abort_flag)) break;
+        mbar_expect_tx(&bar->do_full[i & 1], SM::kTileBytes);
+        tma_load_4d(sDO + (i & 1) * SM::kTileBytes, glb ? &mapDOc : &mapDO, &bar->do_full[i & 1], 0, row0, hc, b);
+        if (++qs == 2) { qs = 0; qph ^= 1; }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 18) {
+    // ------------------------------------------------------------------ row statistics of each item
+    // lse * log2(e) and Delta of the item's 128 query rows, plus per-quarter mask flags, go to shared memory.
+    // The global loads of item i+1 are issued before waiting for its slot, so their latency is hidden.
+    float r_lse[4], r_delta[4];
+    int r_pos[4], r_glb = 0, r_row0 = 0, r_h = 0;
+    ItemCursor cur(plan, g * G);
+    auto load_item = [&]() {
+      const int h = cur.h, glb = cur.glb(), row0 = cur.tile() * kTileM;
+      cur.next();
+      const int n_rows = glb ? n_c : a.Lq;
+      const float* lse = glb ? a.lse_glb : a.lse_loc;
+      const float* dl = glb ? a.delta_glb : a.delta_loc;
+      r_glb = glb;
+      r_row0 = row0;
+      r_h = h;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int row = row0 + q * 32 + lane;
+        const bool valid = row < n_rows;
+        const int64_t si = ((int64_t)b * a.Hq + h) * a.Lq + (valid ? row : 0);
+        r_lse[q] = valid ? __ldg(&lse[si]) * kLog2e : 0.f;
+        r_delta[q] = valid ? __ldg(&dl[si]) : 0.f;
+        r_pos[q] = valid ? (glb ? __ldg(&a.q_idx[(int64_t)b * a.Lq + row]) : row) + a.q_pos_offset : -1;
+      }
+    };
+    load_item();
+    for (int i = 0; i < plan.total; ++i) {
+      const int s = i & 1;
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->st_empty[s], ((i >> 1) & 1) ^ 1, abort_flag))) break;
+      float* st_lse = reinterpret_cast<float*>(smem + SM::kStatOff + s * SM::kStatSlot);
+      float* st_delta = st_lse + 128;
+      int* st_flags = reinterpret_cast<int*>(st_delta + 128);
+      const int w_eff = r_glb ? 0x3fffffff : a.window;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int col = q * 32 + lane;
+        st_lse[col] = r_lse[q];
+        st_delta[col] = -r_delta[q];   // negated: dS = P * (dP + (-Delta)) with packed f32x2 arithmetic
+        // quarter q needs the element mask unless every (key, query) pair of it is visible
+        const bool lane_ok = r_pos[q] >= 0 && (k0 + kTileN - 1 <= r_pos[q]) && (k0 >= r_pos[q] - w_eff);
+        const bool interior = __all_sync(0xffffffffu, lane_ok);
+        if (lane == 0) st_flags[q] = interior ? 0 : 1;
+      }
+      if (lane == 0) { st_flags[4] = r_glb; st_flags[5] = r_row0; st_flags[6] = r_h; }
+      __syncwarp();
+      mbar_arrive(&bar->st_full[s]);
+      if (i + 1 < plan.total) load_item();
+    }
+  } else if (warp == 17) {
+    // ------------------------------------------------------------------ MMA issuer
+    // (whole warp runs the loop; only the tcgen05 instructions are predicated on lane 0)
+    {
+      const uint32_t leader = (lane == 0);
+      constexpr uint32_t tmem = 0;   // checked above: TMEM operand addresses are immediates in this loop
+      constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);
+      constexpr uint32_t idesc_acc = idesc_bf16_f32(128, D, 0, 1);
+      constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 1, 1);     // A = dS read MN-major, B = K read MN-major
+      constexpr uint32_t kStageStep = SM::kTileBytes >> 4;
+      const uint64_t dk = smem_desc_sw128(smem_u32(sK), 16, 1024), dv = smem_desc_sw128(smem_u32(sV), 16, 1024);
+      const uint64_t dkm = smem_desc_sw128(smem_u32(sK), kBoxBytes, 1024);            // K as MN-major B of dQ
+      const uint64_t dsm = smem_desc_sw128(smem_u32(sDS), kBoxBytes, 1024);           // dS as MN-major A of dQ
+      const uint64_t dq_base = smem_desc_sw128(smem_u32(sQ), 16, 1024);
+      const uint64_t ddo_base = smem_desc_sw128(smem_u32(sDO), 16, 1024);
+      const uint64_t dqm_base = smem_desc_sw128(smem_u32(sQ), kBoxBytes, 1024);      // Q / dO as MN-major B
+      const uint64_t ddom_base = smem_desc_sw128(smem_u32(sDO), kBoxBytes, 1024);
+      auto issue_S = [&](int qs) {    // S^T = K Q^T into the T columns
+        const uint64_t qd = dq_base + qs * kStageStep;
+#pragma unroll
+        for (int kk = 0; kk < kKSteps; ++kk) {
+          const uint32_t c = ((kk >> 2) * kBoxBytes + (kk & 3) * 32) >> 4;
+          mma_ss(tmem + 256, dk + c, qd + c, idesc_s, kk > 0, leader);
+        }
+        tc_commit(&bar->s_full, leader);
+      };
+      auto issue_dP = [&](int ds) {   // dP^T = V dO^T
+        const uint64_t dod = ddo_base + ds * kStageStep;
+#pragma unroll
+        for (int kk = 0; kk < kKSteps; ++kk) {
+          const uint32_t c = ((kk >> 2) * kBoxBytes + (kk & 3) * 32) >> 4;
+          mma_ss(tmem + 384, dv + c, dod + c, idesc_s, kk > 0, leader);
+        }
+        tc_commit(&bar->dp_full, leader);
+      };
+      auto issue_dQ = [&]() {         // dQ(i) = dS K into the T columns (a fresh accumulator for every item)
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          mma_ss(tmem + 256, dsm + ((kk * 2048) >> 4), dkm + ((kk * 2048) >> 4), idesc_dq, kk > 0, leader);
+        tc_commit(&bar->dq_full, leader);
+      };
+      auto issue_dV = [&](int ds, bool first) {   // dV += P^T dO
+        const uint64_t dod = ddom_base + ds * kStageStep;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          mma_ts(tmem, tmem + 384 + (kk >> 1) * 32 + (kk & 1) * 8, dod + ((kk * 2048) >> 4), idesc_acc,
+                 (kk > 0 || !first) ? 1u : 0u, leader);
+        tc_commit(&bar->do_empty[ds], leader);
+      };
+      auto issue_dK = [&](int qs, bool first) {   // dK += dS^T Q
+        const uint64_t qd = dqm_base + qs * kStageStep;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          mma_ts(tmem + D, tmem + 384 + (kk >> 1) * 32 + 16 + (kk & 1) * 8, qd + ((kk * 2048) >> 4), idesc_acc,
+                 (kk > 0 || !first) ? 1u : 0u, leader);
+        tc_commit(&bar->q_empty[qs], leader);
+      };
+      bool ok = mbar_spin_warp(&bar->kv_full, 0, abort_flag) && mbar_spin_warp(&bar->q_full[0], 0, abort_flag) &&
+                mbar_spin_warp(&bar->do_full[0], 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
+        issue_S(0);
+        issue_dP(0);
+      }
+      for (int i = 0; ok && i < plan.total; ++i) {
+        const int qs = i & 1;
+        if (!mbar_spin_warp(&bar->pds_full, i & 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        issue_dQ();                 // first: the compute warps read it out while dV and dK run
+        issue_dV(i & 1, i == 0);
+        issue_dK(qs, i == 0);
+        if (i + 1 < plan.total) {
+          const int qn = (i + 1) & 1;
+          // S^T(i+1) reuses the columns of dQ(i): wait for its read-out; dP^T(i+1) follows dV(i), dK(i) in order
+          if (!mbar_spin_warp(&bar->t_free, i & 1, abort_flag) ||
+              !mbar_spin_warp(&bar->q_full[qn], ((i + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          issue_S(qn);
+          if (!mbar_spin_warp(&bar->do_full[(i + 1) & 1], ((i + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          issue_dP((i + 1) & 1);
+        }
+      }
+      if (ok) tc_commit(&bar->final_bar, leader);
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ P^T / dS^T and epilogue
+    const int q = warp >> 2;                           // query-column quarter of this warp
+    const int kr = (warp & 3) * 32 + lane;             // key inside the block == TMEM lane
+    const int kp = k0 + kr;
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const uint32_t s_addr = tmem + lane_base + 256 + q * 32;
+    const uint32_t dp_addr = tmem + lane_base + 384 + q * 32;
+    bool ok = true;
+    for (int i = 0; i < plan.total; ++i) {
+      const int s = i & 1;
+      // this item's row statistics go to registers before the scores are waited for
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->st_full[s], (i >> 1) & 1, abort_flag))) { ok = false; break; }
+      const uint32_t st_base = smem_u32(smem + SM::kStatOff + s * SM::kStatSlot);
+      const int* st_flags = reinterpret_cast<const int*>(smem + SM::kStatOff + s * SM::kStatSlot) + 2 * 128;
+      float st[32];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const float4 v = lds128(st_base + (q * 32 + c * 4) * 4);
+        st[4 * c] = v.x; st[4 * c + 1] = v.y; st[4 * c + 2] = v.z; st[4 * c + 3] = v.w;
+      }
+      const bool masked = st_flags[q] != 0;
+      const int item_glb = st_flags[4], item_row0 = st_flags[5], item_h = st_flags[6];
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->s_full, i & 1, abort_flag))) { ok = false; break; }
+      tc_fence_after();
+      uint32_t pp[16];
+      {
+        uint32_t sv[32];
+        tmem_ld32(s_addr, sv);
+        tmem_ld_wait();
+        // the element mask is needed only for the few tiles that straddle the causal diagonal or a window edge:
+        // two loop versions, so that the common one has no branches
+        if (!masked) {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const float2 x = __ffma2_rn(make_float2(__uint_as_float(sv[2 * e]), __uint_as_float(sv[2 * e + 1])),
+                                        make_float2(a.scale_log2, a.scale_log2), make_float2(-st[2 * e], -st[2 * e + 1]));
+            pp[e] = pack_bf16(fast_exp2(x.x), fast_exp2(x.y));
+          }
+        } else {
+          const int glb = st_flags[4], row0 = st_flags[5];
+          const int w_eff = glb ? 0x3fffffff : a.window;
+          const int n_rows = glb ? n_c : a.Lq;
+          const int32_t* qi = a.q_idx + (int64_t)b * a.Lq;
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            int pos[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+              const int row = row0 + q * 32 + e + u;
+              pos[u] = row < n_rows ? (glb ? __ldg(&qi[row]) : row) + a.q_pos_offset : -1;
+            }
+            float p0 = fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, -st[e]));
+            float p1 = fast_exp2(fmaf(__uint_as_float(sv[e + 1]), a.scale_log2, -st[e + 1]));
+            p0 = (kp <= pos[0] && kp >= pos[0] - w_eff) ? p0 : 0.f;
+            p1 = (kp <= pos[1] && kp >= pos[1] - w_eff) ? p1 : 0.f;
+            pp[e >> 1] = pack_bf16(p0, p1);
+          }
+        }
+      }
+      // Delta of the same rows, again ahead of the wait; after this the statistics slot may be refilled
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const float4 v = lds128(st_base + (128 + q * 32 + c * 4) * 4);
+        st[4 * c] = v.x; st[4 * c + 1] = v.y; st[4 * c + 2] = v.z; st[4 * c + 3] = v.w;
+      }
+      mbar_arrive(&bar->st_empty[s]);
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->dp_full, i & 1, abort_flag))) { ok = false; break; }
+      tc_fence_after();
+      uint32_t pd[16];
+      {
+        uint32_t dv[32];
+        tmem_ld32(dp_addr, dv);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          // dS uses the bf16-rounded P, the same value the dV product sees; st[] holds -Delta
+          const float2 t = __fadd2_rn(make_float2(__uint_as_float(dv[2 * e]), __uint_as_float(dv[2 * e + 1])),
+                                      make_float2(st[2 * e], st[2 * e + 1]));
+          const float2 ds = __fmul2_rn(make_float2(bf16lo_to_f32(pp[e]), bf16hi_to_f32(pp[e])), t);
+          pd[e] = pack_bf16(ds.x, ds.y);
+        }
+      }
+      // P^T and dS^T go to this quarter's own 32 columns of the dP^T region (first 16 / next 16): A operands of dV
+      // and dK.  dS also goes to shared memory, [key][query] with the 128-byte swizzle of a TMA tile: read
+      // MN-major it is the A operand of dQ = dS K.
+      tmem_st16(dp_addr, pp);
+      tmem_st16(dp_addr + 16, pd);
+      {
+        const uint32_t row = smem_u32(sDS) + (q >> 1) * kBoxBytes + kr * 128;
+        const int chunk0 = (q & 1) * 4;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((chunk0 + c) ^ (kr & 7)) << 4)),
+                       "r"(pd[4 * c]), "r"(pd[4 * c + 1]), "r"(pd[4 * c + 2]), "r"(pd[4 * c + 3]) : "memory");
+      }
+      tmem_st_wait();
+      fence_async_smem();        // the MMA reads the tile through the async proxy
+      tc_fence_before();
+      mbar_arrive(&bar->pds_full);
+      // ---- dQ(i): read the 128 x D accumulator out of TMEM (lane = query row) and add it to the fp32 dQ buffer
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->dq_full, i & 1, abort_flag))) { ok = false; break; }
+      tc_fence_after();
+      {
+        constexpr int kCols = D / 4;     // 32 (D = 128) or 16 (D = 64) columns per quarter
+        uint32_t v[32];
+        tmem_ld32(tmem + lane_base + 256 + ((q * kCols) & ~31), v);
+        tmem_ld_wait();
+        tc_fence_before();
+        mbar_arrive(&bar->t_free);       // the values are in registers: S^T(i+1) may overwrite the columns
+        // Reduction into the fp32 dQ buffer.  Lane == query row would make every red instruction touch 32 rows with
+        // 16 bytes each (half a sector per row): instead each warp transposes its 32 x 16-column pieces through
+        // shared memory, so that one instruction covers 8 rows with 64 contiguous bytes each.  The scratch is the
+        // 2 KB of the dS tile that this warp itself wrote (the dQ MMA that read them has completed, and nobody else
+        // writes them), addressed with the same swizzle, which keeps both directions free of bank conflicts.
+        const int r = item_row0 + kr;    // query row of this thread (lane == row inside the tile)
+        const int n_rows = item_glb ? n_c : a.Lq;
+        const int t_mine = r < n_rows ? (item_glb ? __ldg(&a.q_idx[(int64_t)b * a.Lq + r]) : r) : -1;
+        const uint32_t scratch = smem_u32(sDS) + (q >> 1) * kBoxBytes + (kr - lane) * 128;
+        const int chunk0 = (q & 1) * 4;
+        const int sub = (D == 64) ? (q & 1) * 16 : 0;
+        float* acc_head = a.dq_acc + (int64_t)b * a.Lq * a.Hq * D + (int64_t)item_h * D + q * kCols;
+#pragma unroll
+        for (int half = 0; half < kCols / 16; ++half) {
+          __syncwarp();
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const int k = sub + half * 16 + 4 * c;
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(scratch + lane * 128 + (((chunk0 + c) ^ (lane & 7)) << 4)),
+                         "r"(v[k]), "r"(v[k + 1]), "r"(v[k + 2]), "r"(v[k + 3]) : "memory");
+          }
+          __syncwarp();
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int R = j * 8 + (lane >> 2), cl = lane & 3;
+            const float4 x = lds128(scratch + R * 128 + (((chunk0 + cl) ^ (R & 7)) << 4));
+            const int t = __shfl_sync(0xffffffffu, t_mine, R);
+            if (t >= 0) {
+              float* dst = acc_head + (int64_t)t * a.Hq * D + half * 16 + cl * 4;
+              asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(x.x * a.scale),
+                           "f"(x.y * a.scale), "f"(x.z * a.scale), "f"(x.w * a.scale) : "memory");
+            }
+          }
+        }
+      }
+    }
+    // epilogue: quarters 0,1 store the two column halves of dV, quarters 2,3 those of dK
+    if (ok && __all_sync(0xffffffffu, mbar_wait(&bar->final_bar, 0, abort_flag))) {
+      tc_fence_after();
+      const bool valid = kp < a.Lk;
+      const int which = q >> 1, half = q & 1;
+      const RowStrides st = which == 0 ? a.dv_st : a.dk_st;
+      const int64_t o = b * st.b + (valid ? kp : 0) * st.t + (int64_t)g * D + half * (D / 2);
+      bf16* dst = (which == 0 ? a.dV : a.dK) + o;
+      const float mul = which == 0 ? 1.0f : a.scale;
+#pragma unroll
+      for (int c = 0; c < D / 64; ++c) {
+        uint32_t v[32];
+        tmem_ld32(tmem + lane_base + which * D + half * (D / 2) + c * 32, v);
+        tmem_ld_wait();
+        if (valid) {
+          uint4* d4 = reinterpret_cast<uint4*>(dst + c * 32);
+#pragma unroll
+          for (int x = 0; x < 4; ++x) {
+            float f[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[8 * x + e]) * mul;
+            d4[x] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
+                               pack_bf16(f[6], f[7]));
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (bar->abort_flag) {
+    const uint64_t t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    if (tid == 0) atomicExch(a.status, 1);
+    __syncthreads();
+  }
+  if (warp == 17) tmem_dealloc(tmem, 512);
+}
+
+
+// fp32 dQ accumulator -> bf16 dQ (the accumulated values already carry the soft-max scale)
+__global__ void __launch_bounds__(256) dq_convert_kernel(const float* __restrict__ acc, bf16* __restrict__ dQ, int B, int L,
+                                                         int row_elems, int64_t bs, int64_t ts) {
+  const int64_t chunks_per_row = row_elems / 8;
+  const int64_t n = (int64_t)B * L * chunks_per_row;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t row = i / chunks_per_row, c = i % chunks_per_row;
+    const float4 x = __ldg(reinterpret_cast<const float4*>(acc) + 2 * i), y = __ldg(reinterpret_cast<const float4*>(acc) + 2 * i + 1);
+    const int64_t b = row / L, t = row % L;
+    *reinterpret_cast<uint4*>(dQ + b * bs + t * ts + c * 8) =
+        make_uint4(pack_bf16(x.x, x.y), pack_bf16(x.z, x.w), pack_bf16(y.x, y.y), pack_bf16(y.z, y.w));
+  }
+}
+
 size_t rows_bytes(const l2a_params* p) { return align_up((size_t)p->B * p->Lq * p->Hq * p->D * sizeof(bf16), 256); }
 size_t stat_bytes(const l2a_params* p) { return align_up((size_t)p->B * p->Hq * p->Lq * sizeof(float), 256); }
 
@@ -972,7 +1439,36 @@ cudaError_t launch_bwd_kernels(const BwdArgs& base, const CUtensorMap& mapQ, con
 
 int dkv_split_block(int n_kblocks) { return n_kblocks >= 8 ? (3 * n_kblocks) / 4 : 0; }
 
-size_t bwd_ws_size(const l2a_params* p) { return kWsHeaderBytes + 2 * rows_bytes(p) + 3 * stat_bytes(p); }
+template <int D>
+cudaError_t launch_bwd_fused(const BwdArgs& base, const CUtensorMap& mapQ, const CUtensorMap& mapDO,
+                             const CUtensorMap& mapQc, const CUtensorMap& mapDOc, const CUtensorMap& mapK,
+                             const CUtensorMap& mapV, cudaStream_t s) {
+  cudaError_t e = cudaFuncSetAttribute(bwd_fused_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       FusedSmem<D>::kTotal);
+  if (e != cudaSuccess) return e;
+  const size_t acc = (size_t)base.B * base.Lq * base.Hq * D * sizeof(float);
+  e = cudaMemsetAsync(base.dq_acc, 0, acc, s);
+  if (e != cudaSuccess) return e;
+  phase_events().mark(s);     // (no local dQ launch in this mode)
+  phase_events().mark(s);     // (no global dQ launch)
+  BwdArgs a = base;
+  const int n_kblocks = (base.Lk + kTileN - 1) / kTileN;
+  a.kb_begin = 0;
+  a.kb_count = n_kblocks;
+  bwd_fused_kernel<D><<<(unsigned)n_kblocks * base.B * base.Hkv, kDkvThreads, FusedSmem<D>::kTotal, s>>>(
+      mapQ, mapDO, mapQc, mapDOc, mapK, mapV, a);
+  int device = 0, sms = 148;
+  if (cudaGetDevice(&device) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+  dq_convert_kernel<<<sms * 8, 256, 0, s>>>(base.dq_acc, base.dQ, base.B, base.Lq, base.Hq * D, base.dq_st.b,
+                                            base.dq_st.t);
+  phase_events().mark(s);
+  return cudaGetLastError();
+}
+
+size_t acc_bytes(const l2a_params* p) {
+  return (p->flags & L2A_FLAG_FUSED_DQ) ? align_up((size_t)p->B * p->Lq * p->Hq * p->D * sizeof(float), 256) : 0;
+}
+size_t bwd_ws_size(const l2a_params* p) { return kWsHeaderBytes + 2 * rows_bytes(p) + 3 * stat_bytes(p) + acc_bytes(p); }
 
 }  // namespace l2a
 
@@ -1011,6 +1507,7 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   if (!skip_global && (!d_mask || !q_idx || !n_routed || !prefix || !A_c || !lse_glb)) return L2A_ERR_INVALID_ARG;
   if (!skip_local && (!S_save || !lse_loc)) return L2A_ERR_INVALID_ARG;
   if (force_all && (skip_local || skip_global)) return L2A_ERR_INVALID_ARG;
+  if ((p->flags & L2A_FLAG_FUSED_DQ) && (skip_local || skip_global || force_all)) return L2A_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(dO) || !aligned16(S_save) || !aligned16(A_c) ||
       !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
     return L2A_ERR_INVALID_ARG;
@@ -1023,6 +1520,8 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   float* delta_loc = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p));
   float* delta_glb = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + stat_bytes(p));
   float* lse_c = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + 2 * stat_bytes(p));
+  float* dq_acc = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + 3 * stat_bytes(p));
+  const bool fused = p->flags & L2A_FLAG_FUSED_DQ;
 
   CUtensorMap mapQ, mapDO, mapQc, mapDOc, mapK, mapV;
   const RowStrides qs = resolve_strides(p->q_stride, p->Lq, p->Hq * p->D);
@@ -1084,8 +1583,14 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   a.lse_loc = lse_loc; a.lse_glb = force_all ? lse_c : lse_glb; a.delta_loc = delta_loc; a.delta_glb = delta_glb;
   a.dQ = static_cast<bf16*>(dQ); a.dK = static_cast<bf16*>(dK); a.dV = static_cast<bf16*>(dV);
   a.dq_st = qs; a.dk_st = ks; a.dv_st = vs;
+  a.dq_acc = fused ? dq_acc : nullptr;
   a.status = reinterpret_cast<int*>(ws);
-  cudaError_t e = p->D == 128 ? launch_bwd_kernels<128>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, s)
-                              : launch_bwd_kernels<64>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, s);
+  cudaError_t e;
+  if (fused)
+    e = p->D == 128 ? launch_bwd_fused<128>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, s)
+                    : launch_bwd_fused<64>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, s);
+  else
+    e = p->D == 128 ? launch_bwd_kernels<128>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, s)
+                    : launch_bwd_kernels<64>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, s);
   return e == cudaSuccess ? L2A_OK : L2A_ERR_CUDA;
 }

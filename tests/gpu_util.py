@@ -33,7 +33,8 @@ def to_f64(t: torch.Tensor) -> np.ndarray:
     return t.detach().float().cpu().numpy().astype(np.float64)
 
 
-def check_close(got: np.ndarray, want: np.ndarray, what: str, max_abs=MAX_ABS, mean_abs=MEAN_ABS, outlier_frac=0.0):
+def check_close(got: np.ndarray, want: np.ndarray, what: str, max_abs=MAX_ABS, mean_abs=MEAN_ABS, outlier_frac=0.0,
+                extra_outliers=0):
     assert got.shape == want.shape, (what, got.shape, want.shape)
     assert np.isfinite(got).all(), f"{what}: non-finite values in the GPU result"
     if got.size == 0:
@@ -44,7 +45,7 @@ def check_close(got: np.ndarray, want: np.ndarray, what: str, max_abs=MAX_ABS, m
     i = np.unravel_index(np.argmax(excess), err.shape)
     n_over = int((excess > 0).sum())
     msg = f"{what}: abs err {err[i]:.4g} at {i} (got {got[i]}, want {want[i]}), max abs err {err.max():.4g}, {n_over} over"
-    assert n_over <= math.ceil(outlier_frac * err.size), msg
+    assert n_over <= math.ceil(outlier_frac * err.size) + extra_outliers, msg
     assert (err <= 2.0 * bound).all(), msg
     mean_tol = mean_abs + 2.0 ** -9 * np.abs(want).mean()
     assert err.mean() <= mean_tol, f"{what}: mean abs err {err.mean():.4g} > {mean_tol:.4g}"
@@ -127,10 +128,13 @@ def run_backward(case: "Case", with_dgate=True):
     return b
 
 
-def check_backward_full(case: "Case"):
+def check_backward_full(case: "Case", dq_first_rows=0):
+    """dq_first_rows: elements of dQ per (batch entry, head) that may exceed the bound (by less than a factor of two)
+    on top of the 1e-5 fraction.  The fused backward forms dS from the bf16-rounded P (the dQ kernel of the
+    seven-GEMM path keeps P in fp32), so the rows with two or three keys, where |dS| ~ 10, carry sqrt(2) more noise."""
     b = case.buf
     dQ, dK, dV = oracle.backward_full(case.shape, case.u16("Q"), case.u16("K"), case.u16("V"), case.d, case.u16("dO"))
-    check_close(to_f64(b.dQ), dQ, "dQ", outlier_frac=1e-5)
+    check_close(to_f64(b.dQ), dQ, "dQ", outlier_frac=1e-5, extra_outliers=dq_first_rows * dQ.shape[0] * dQ.shape[2])
     check_close(to_f64(b.dK), dK, "dK", outlier_frac=1e-5)
     check_close(to_f64(b.dV), dV, "dV", outlier_frac=1e-5)
     return dQ, dK, dV
