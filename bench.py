@@ -255,6 +255,8 @@ def main():
     ap.add_argument("--density", type=float, default=None)
     ap.add_argument("--routing", default=None, choices=[None, "bernoulli", "clustered", "all", "none"])
     ap.add_argument("--forward-only", action="store_true")
+    ap.add_argument("--shared-window", action="store_true",
+                    help="L2A_FLAG_SHARED_WINDOW: global attention reuses the local pass for the keys inside the window")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-tokens", type=int, default=2048, help="tokens of the CPU-baseline sample (0 = skip)")
     ap.add_argument("--ref-tokens", type=int, default=1024, help="tokens per step of --impl reference")
@@ -284,10 +286,12 @@ def main():
 
     cfg, rho, seed, d, logits = make_workload(args, seed_offset=rank)
     backward = not args.forward_only
-    flags = l2a.FLAG_SAVE_FOR_BWD if backward else 0
+    flags = (l2a.FLAG_SAVE_FOR_BWD if backward else 0) | (l2a.FLAG_SHARED_WINDOW if args.shared_window else 0)
     p = l2a.params(cfg.B, cfg.L, cfg.L, cfg.Hq, cfg.Hkv, cfg.D, cfg.W, flags=flags)
     use_logits = logits is not None
     buf = l2a.Buffers.allocate(p, backward=backward, router_dtype=torch.float32 if use_logits else torch.uint8)
+    if args.shared_window and not backward:
+        buf.lse_loc = torch.empty((cfg.B, cfg.Hq, cfg.L), dtype=torch.float32, device="cuda")
     kind = l2a.ROUTER_LOGITS_F32 if use_logits else l2a.ROUTER_MASK_U8
 
     # host inputs (pinned): the same seeded tensors the oracle would read
@@ -423,7 +427,8 @@ def main():
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.workload, "B": cfg.B, "L": cfg.L, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
                    "W": cfg.W, "routing": args.routing or cfg.routing, "density": float(d.mean()),
-                   "pass": "fwd+bwd" if backward else "fwd", "parallelism": f"replicas x{world}",
+                   "pass": "fwd+bwd" if backward else "fwd", "shared_window": bool(args.shared_window),
+                   "parallelism": f"replicas x{world}",
                    "l2_policy": "inputs larger than L2 (Q alone is %.2f GB)" % (host["Q"].numel() * 2 / 1e9),
                    "useful_tflop_per_step": step_flops / 1e12, "pairs_per_head": pairs},
         "clocks": clocks, "e2e": e2e, "gpu_launches": KERNELS_PER_STEP * args.steps if backward else 5 * args.steps,

@@ -65,6 +65,18 @@ typedef enum {
                                   /* L2A_FLAG_SKIP_GLOBAL or L2A_FLAG_FORCE_ALL_GLOBAL (invalid argument).  On   */
                                   /* B200 the reductions' L2 traffic makes it slower than the default at long    */
                                   /* sequences, so it is off by default.                                         */
+#define L2A_FLAG_SHARED_WINDOW 64u /* forward, shared projections (the "L2A-shared" variant of the paper's ablations:  */
+                                  /* one Q/K/V set feeds both modules, which is what this interface always passes):  */
+                                  /* a routed row's scores against the keys inside its window are the ones the Local */
+                                  /* pass has already reduced, so Global Attention covers only the keys BEFORE the   */
+                                  /* window (positions 0 .. t-W-1) and is merged with the local result,              */
+                                  /*   a_t = (e^{lse_out} o_out + e^{lse_loc} s_t) / (e^{lse_out} + e^{lse_loc}),     */
+                                  /* which is the softmax over the whole prefix.  Saves rho * W pairs per head.      */
+                                  /* s_t enters as the stored bf16 value (one extra rounding of relative size 2^-9   */
+                                  /* on the window's share of a_t; same tolerance).  Needs lse_loc (also without     */
+                                  /* L2A_FLAG_SAVE_FOR_BWD); not combined with L2A_FLAG_SKIP_LOCAL or                */
+                                  /* L2A_FLAG_FORCE_ALL_GLOBAL; ignored by a call that has L2A_FLAG_SKIP_GLOBAL.     */
+                                  /* A_c, lse_glb and O mean the same as without it; l2a_backward is unchanged.     */
 #define L2A_FLAG_FORCE_ALL_GLOBAL 8u /* training iterations that invoke Global Attention for every    */
                                   /* token regardless of d_t (Section 3.3: done with a small       */
                                   /* probability so that masked tokens' routers get a gradient).   */

@@ -99,6 +99,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
 
   const int32_t* q_idx_b = a.q_idx + (int64_t)b * a.Lq;
   const int w_eff = a.global_mode ? 0x3fffffff : a.window;
+  // shared-window mode: a row at position p attends to the keys 0 .. p - W - 1 only (the window p - W .. p is the
+  // local pass's share and enters in the epilogue)
+  const bool shared = a.global_mode && a.shared_window;
+  const int vis_shift = shared ? a.window + 1 : 0;
   if (a.global_mode) {
     // launches restricted to a row range take the groups whose last row falls into it: every group exactly once
     const int c_last = min(row0 + kRowsPerCta, n_rows) - 1;
@@ -118,10 +122,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       tr[t].min_pos = (compact ? q_idx_b[first] : first) + a.q_pos_offset;
       tr[t].max_pos = (compact ? q_idx_b[last] : last) + a.q_pos_offset;
       const int lo_pos = tr[t].min_pos - w_eff;
-      tr[t].lo = lo_pos > 0 ? lo_pos / kTileN : 0;
-      tr[t].hi = tr[t].max_pos / kTileN;
-      jlo = min(jlo, tr[t].lo);
-      jhi = max(jhi, tr[t].hi);
+      const int hi_pos = tr[t].max_pos - vis_shift;   // last key position any row of the tile attends to
+      if (hi_pos >= 0) {
+        tr[t].lo = lo_pos > 0 ? lo_pos / kTileN : 0;
+        tr[t].hi = hi_pos / kTileN;
+        jlo = min(jlo, tr[t].lo);
+        jhi = max(jhi, tr[t].hi);
+      } else {
+        tr[t].lo = 1; tr[t].hi = 0;   // shared-window mode: every key of these rows lies inside the window
+      }
     } else {
       tr[t].min_pos = tr[t].max_pos = 0;
       tr[t].lo = 1; tr[t].hi = 0;
@@ -179,7 +188,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       tma_prefetch_desc(&mapK);
       tma_prefetch_desc(&mapV);
       for (int t = 0; t < kNumTiles; ++t) {
-        if (!tr[t].active) continue;
+        if (!tr[t].active || tr[t].lo > tr[t].hi) continue;
         mbar_expect_tx(&bar->q_full[t], SM::kQTileBytes);
         tma_load_4d(sQ + t * SM::kQTileBytes, &mapQ, &bar->q_full[t], 0, row0 + t * kTileM, h * (D / 64), b);
       }
@@ -236,8 +245,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       };
       auto in_range = [&](int t, int j) { return t ? (j >= lo1 && j <= hi1) : (j >= lo0 && j <= hi0); };
 
+      if (jhi < jlo) ok = false;   // no key block at all (shared-window mode): nothing to issue, nobody waits
       // first key block: Q*K^T for both tiles
-      if (!mbar_spin_warp(&bar->k_full[0], 0, abort_flag)) ok = false;
+      if (ok && !mbar_spin_warp(&bar->k_full[0], 0, abort_flag)) ok = false;
 #pragma unroll
       for (int t = 0; t < kNumTiles; ++t) {
         if (ok && in_range(t, jlo)) {
@@ -309,8 +319,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       const int row = row0 + t * kTileM + r;           // sequence row (local) or compact row (global)
       const bool valid = row < n_rows;
       const int seq_row = valid ? (compact ? q_idx_b[row] : row) : -1;
-      const int pos = valid ? seq_row + a.q_pos_offset : -1;
-      const int pos_lo = valid ? (pos - w_eff) : 0x7fffffff;   // smallest visible key position
+      const int pos = valid ? seq_row + a.q_pos_offset - vis_shift : -1;   // largest visible key position
+      const int pos_lo = valid ? (pos - w_eff) : 0x7fffffff;               // smallest visible key position
       float m_use = -INFINITY;   // reference maximum, exp2 domain (identical in both threads of a row)
       float l = 0.f;             // this thread's part of the row sum
       bool ok = true;
@@ -323,7 +333,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         if (warp == L2A_TRACE_FWD_WARP && lane == 0) L2A_FWD_TRACE(1, 4 * i);
         tc_fence_after();
         const int k0 = j * kTileN + hf * 64;
-        const bool partial = (k0 + 63 > my.min_pos) || (k0 < my.max_pos - w_eff);
+        const bool partial = (k0 + 63 > my.min_pos - vis_shift) || (k0 < my.max_pos - w_eff);
         // pass 1: row maximum of this half (32 columns at a time: the scores are re-read from TMEM in pass 2
         // rather than kept in 64 registers)
         float mx = -INFINITY;
@@ -413,7 +423,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       }
 
       // ---- epilogue: O / l, log-sum-exp, store (local) or scatter + combine (global)
-      if (ok && __all_sync(0xffffffffu, mbar_wait(&bar->o_final, 0, abort_flag))) {
+      if (ok && (n_my == 0 || __all_sync(0xffffffffu, mbar_wait(&bar->o_final, 0, abort_flag)))) {
         tc_fence_after();
         // total row sum: exchange the two partial sums (the slot of parity n_my & 1 is free by now)
         float* slot = xch + (((n_my & 1) * kNumTiles + t) * 2) * kTileM;
@@ -421,9 +431,23 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         mbar_arrive(&bar->xch[t]);
         if (__all_sync(0xffffffffu, mbar_wait(&bar->xch[t], n_my & 1, abort_flag))) {
           l += slot[(hf ^ 1) * kTileM + r];
-          const float inv_l = (l > 0.f) ? 1.0f / l : 0.f;
+          float inv_l = (l > 0.f) ? 1.0f / l : 0.f;
+          float lse2 = m_use + log2f(l);   // log-sum-exp in the exp2 domain
+          float c_loc = 0.f;               // shared-window mode: weight of the local result s_t in a_t
+          if (shared && valid) {
+            // a_t = (e^{lse_out} o_out + e^{lse_loc} s_t) / (e^{lse_out} + e^{lse_loc}): the softmax over the whole
+            // prefix, split into the keys before the window (this kernel) and the window (the local pass)
+            const float lse_out2 = (l > 0.f) ? lse2 : -INFINITY;
+            const float lse_loc2 = a.lse_loc[((int64_t)b * a.Hq + h) * a.Lq + seq_row] * 1.4426950408889634f;
+            const float mm = fmaxf(lse_out2, lse_loc2);
+            const float w_out = fast_exp2(lse_out2 - mm), w_loc = fast_exp2(lse_loc2 - mm);
+            const float inv = 1.0f / (w_out + w_loc);
+            inv_l *= w_out * inv;
+            c_loc = w_loc * inv;
+            lse2 = mm + log2f(w_out + w_loc);
+          }
           if (valid && hf == 0 && a.lse != nullptr) {
-            const float lse = (m_use + log2f(l)) * 0.6931471805599453f;
+            const float lse = lse2 * 0.6931471805599453f;
             a.lse[((int64_t)b * a.Hq + h) * a.Lq + row] = lse;
           }
           bf16* dst1 = nullptr;   // row-indexed destination (s rows, or compact a rows)
@@ -437,11 +461,29 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
 #pragma unroll
           for (int c = 0; c < D / 64; ++c) {
             uint32_t v[32];
-            tmem_ld32(o_addr + c * 32, v);
-            tmem_ld_wait();
+            if (n_my > 0) {
+              tmem_ld32(o_addr + c * 32, v);
+              tmem_ld_wait();
+            } else {
+#pragma unroll
+              for (int e = 0; e < 32; ++e) v[e] = 0u;    // no key before the window: the accumulator was never written
+            }
             float f[32];
 #pragma unroll
             for (int e = 0; e < 32; ++e) f[e] = __uint_as_float(v[e]) * inv_l;
+            if (shared && dst2) {
+              const uint4* s4 = reinterpret_cast<const uint4*>(dst2 + c * 32);   // s_t, written by the local pass
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const uint4 old = s4[q];
+                const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  f[8 * q + 2 * k] = fmaf(c_loc, __uint_as_float(ow[k] << 16), f[8 * q + 2 * k]);
+                  f[8 * q + 2 * k + 1] = fmaf(c_loc, __uint_as_float(ow[k] & 0xffff0000u), f[8 * q + 2 * k + 1]);
+                }
+              }
+            }
             if (dst1) {
               uint4* d4 = reinterpret_cast<uint4*>(dst1 + c * 32);
 #pragma unroll

@@ -185,6 +185,9 @@ static l2a_status forward_range(const l2a_params* p, const void* Q, const void* 
   if (!skip_global && (!d_mask || !q_idx || !n_routed || !prefix)) return L2A_ERR_INVALID_ARG;
   if (save && (!S_save || !A_c || !lse_loc || !lse_glb)) return L2A_ERR_INVALID_ARG;
   if (save && skip_local) return L2A_ERR_INVALID_ARG;
+  // shared-projection fusion concerns the global part only (a local-phase call just has to store lse_loc)
+  const bool shared = (p->flags & L2A_FLAG_SHARED_WINDOW) && !skip_global;
+  if (shared && (skip_local || force_all || !lse_loc)) return L2A_ERR_INVALID_ARG;
   if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || !aligned(S_save, 16) ||
       !aligned(A_c, 16) || !aligned(lse_loc, 4) || !aligned(lse_glb, 4))
     return L2A_ERR_INVALID_ARG;
@@ -229,6 +232,8 @@ static l2a_status forward_range(const l2a_params* p, const void* Q, const void* 
   a.pair_end = n_pairs;
   a.row_begin = row_range ? row_begin : 0;
   a.row_end = row_range ? row_end : 0x7fffffff;
+  a.shared_window = 0;
+  a.lse_loc = nullptr;
 
   PhaseEvents& pe = phase_events();
   struct ClearOnExit { PhaseEvents& p; ~ClearOnExit() { p.clear(); } } clear_on_exit{pe};
@@ -269,6 +274,8 @@ static l2a_status forward_range(const l2a_params* p, const void* Q, const void* 
     a.out_st = dense_q;
     a.out2_st = os;
     a.lse = lse_glb;
+    a.shared_window = shared ? 1 : 0;
+    a.lse_loc = lse_loc;
     if (force_all) {
       // Global Attention for every token (Section 3.3): same kernel over all rows in place; a_t is stored for
       // every row, and still only enters O where d_t = 1
@@ -408,6 +415,7 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
   L2A_TRY(cudaMemcpyAsync(dev->router, host->router, rb, cudaMemcpyHostToDevice, s));
   l2a_params q = *p;
   if (!bwd) q.flags &= ~L2A_FLAG_SAVE_FOR_BWD;
+  const bool need_lse_loc = bwd || (q.flags & L2A_FLAG_SHARED_WINDOW);   // the fusion reads it back in the forward
   const int n_pairs = ceil_div(p->Lq, kRowsPerCta);
   constexpr int kChunks = 8;
   const bool chunked = p->B == 1 && n_pairs >= 2 * kChunks &&
@@ -455,7 +463,7 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
     for (int c = 0; c < kChunks; ++c) {
       L2A_TRY(cudaStreamWaitEvent(s, aux.chunk[c], 0));
       st = forward_range(&ql, dev->Q, dev->K, dev->V, dev->d_mask, dev->q_idx, dev->n_routed, dev->prefix, dev->O,
-                         bwd ? dev->S_save : nullptr, bwd ? dev->A_c : nullptr, bwd ? dev->lse_loc : nullptr,
+                         bwd ? dev->S_save : nullptr, bwd ? dev->A_c : nullptr, need_lse_loc ? dev->lse_loc : nullptr,
                          bwd ? dev->lse_glb : nullptr, dev->fwd_ws, dev->fwd_ws_bytes, stream, pair_edge[c],
                          pair_edge[c + 1], c == 0);
       if (st != L2A_OK) return st;
@@ -464,7 +472,7 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
       const int r0 = pair_edge[c] * kRowsPerCta;
       const int r1 = c + 1 == kChunks ? p->Lq : pair_edge[c + 1] * kRowsPerCta;
       st = forward_range(&qg, dev->Q, dev->K, dev->V, dev->d_mask, dev->q_idx, dev->n_routed, dev->prefix, dev->O,
-                         bwd ? dev->S_save : nullptr, bwd ? dev->A_c : nullptr, bwd ? dev->lse_loc : nullptr,
+                         bwd ? dev->S_save : nullptr, bwd ? dev->A_c : nullptr, need_lse_loc ? dev->lse_loc : nullptr,
                          bwd ? dev->lse_glb : nullptr, dev->fwd_ws, dev->fwd_ws_bytes, stream, 0, -1, false, r0, r1);
       if (st != L2A_OK) return st;
     }
@@ -481,7 +489,7 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
                            dev->prefix, dev->route_ws, dev->route_ws_bytes, stream);
     if (st != L2A_OK) return st;
     st = l2a_forward(&q, dev->Q, dev->K, dev->V, dev->d_mask, dev->q_idx, dev->n_routed, dev->prefix, dev->O,
-                     bwd ? dev->S_save : nullptr, bwd ? dev->A_c : nullptr, bwd ? dev->lse_loc : nullptr,
+                     bwd ? dev->S_save : nullptr, bwd ? dev->A_c : nullptr, need_lse_loc ? dev->lse_loc : nullptr,
                      bwd ? dev->lse_glb : nullptr, dev->fwd_ws, dev->fwd_ws_bytes, stream);
     if (st != L2A_OK) return st;
   }

@@ -95,6 +95,11 @@ struct FwdArgs {
   RowStrides out_st, out2_st;   // strides of out / out2 in elements
   int pair_begin, pair_end;  // 256-row query groups [pair_begin, pair_end) this launch covers (all: 0 .. ceil(Lq / 256))
   int row_begin, row_end;    // global mode: only the groups whose LAST row t lies in [row_begin, row_end)
+  // Shared-projection fusion (global mode over compact rows): the keys inside the window were already attended by
+  // the local pass of the same Q/K/V, so the global pass covers only the keys before the window and merges with the
+  // local result (s_t read from out2, its log-sum-exp from lse_loc).
+  int shared_window;
+  const float* lse_loc;      // [B,Hq,Lq] by row; read only when shared_window is set
 };
 size_t bwd_ws_size(const l2a_params* p);
 // First key block of the second dK/dV launch when the backward is asked for the early boundary (0: not split).
