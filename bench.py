@@ -255,8 +255,10 @@ def main():
     ap.add_argument("--density", type=float, default=None)
     ap.add_argument("--routing", default=None, choices=[None, "bernoulli", "clustered", "all", "none"])
     ap.add_argument("--forward-only", action="store_true")
-    ap.add_argument("--shared-window", action="store_true",
-                    help="L2A_FLAG_SHARED_WINDOW: global attention reuses the local pass for the keys inside the window")
+    ap.add_argument("--shared-window", action=argparse.BooleanOptionalAction, default=True,
+                    help="L2A_FLAG_SHARED_WINDOW (default on: every workload here feeds one Q/K/V set to both "
+                         "modules): global attention reuses the local pass for the keys inside the window; "
+                         "--no-shared-window runs the two modules independently")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-tokens", type=int, default=2048, help="tokens of the CPU-baseline sample (0 = skip)")
     ap.add_argument("--ref-tokens", type=int, default=1024, help="tokens per step of --impl reference")

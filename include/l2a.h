@@ -76,7 +76,15 @@ typedef enum {
                                   /* on the window's share of a_t; same tolerance).  Needs lse_loc (also without     */
                                   /* L2A_FLAG_SAVE_FOR_BWD); not combined with L2A_FLAG_SKIP_LOCAL or                */
                                   /* L2A_FLAG_FORCE_ALL_GLOBAL; ignored by a call that has L2A_FLAG_SKIP_GLOBAL.     */
-                                  /* A_c, lse_glb and O mean the same as without it; l2a_backward is unchanged.     */
+                                  /* A_c, lse_glb and O mean the same as without it, so the backward does not depend */
+                                  /* on how the forward was run.  Passed to l2a_backward, the flag allows the same    */
+                                  /* sharing there: inside the window P_glb = beta_t P_loc with                       */
+                                  /* beta_t = exp(lse_loc - lse_glb) and dP = dO V^T is common to both modules, so    */
+                                  /* the local tile pairs carry both gradients (row statistics                        */
+                                  /* lse' = lse_loc - log(1 + beta), Delta' = (Delta_loc + beta Delta_glb)/(1 + beta)) */
+                                  /* and the global ones stop before the window.  Used only when both outputs get the */
+                                  /* same gradient (not l2a_backward_split with its own dS_loc) and without           */
+                                  /* L2A_FLAG_FUSED_DQ / FORCE_ALL_GLOBAL / SKIP_*; otherwise ignored.                */
 #define L2A_FLAG_FORCE_ALL_GLOBAL 8u /* training iterations that invoke Global Attention for every    */
                                   /* token regardless of d_t (Section 3.3: done with a small       */
                                   /* probability so that masked tokens' routers get a gradient).   */

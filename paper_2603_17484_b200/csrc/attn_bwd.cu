@@ -72,7 +72,9 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const bf16* __restrict__
                                                         const uint8_t* __restrict__ d_mask,
                                                         const int32_t* __restrict__ prefix, float* __restrict__ delta_loc,
                                                         float* __restrict__ delta_glb, float* __restrict__ dgate, int B,
-                                                        int L, int Hq, int a_by_row, int64_t do_bs, int64_t do_ts) {
+                                                        int L, int Hq, int a_by_row, int64_t do_bs, int64_t do_ts,
+                                                        const float* __restrict__ lse_loc,
+                                                        const float* __restrict__ lse_glb, float* __restrict__ lse_eff) {
   constexpr int kLanesPerHead = D / 8;                 // 16-byte chunks per head row
   constexpr int kHeadsPerPass = 32 / kLanesPerHead;
   const int lane = threadIdx.x & 31;
@@ -112,8 +114,23 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const bf16* __restrict__
         dg += __shfl_xor_sync(0xffffffffu, dg, off);
       }
       if (h < Hq && (lane % kLanesPerHead) == 0) {
-        if (S != nullptr) delta_loc[((int64_t)b * Hq + h) * L + t] = dl;
-        if (routed) delta_glb[((int64_t)b * Hq + h) * L + c] = dg;
+        const int64_t it = ((int64_t)b * Hq + h) * L + t, ic = ((int64_t)b * Hq + h) * L + c;
+        float dl_out = dl;
+        if (lse_eff != nullptr) {
+          // Shared-window backward.  Inside the window of a routed row P_glb = beta * P_loc with
+          // beta = exp(lse_loc - lse_glb), and dP is the same product dO V^T for both modules, so the two
+          // contributions add up to P' (dP - Delta') with P' = (1 + beta) P_loc and
+          // Delta' = (Delta_loc + beta * Delta_glb) / (1 + beta): the local items carry them with these statistics.
+          float le = lse_loc[it];
+          if (routed) {
+            const float beta = __expf(le - lse_glb[ic]);
+            dl_out = (dl + beta * dg) / (1.0f + beta);
+            le -= log1pf(beta);
+          }
+          lse_eff[it] = le;
+        }
+        if (S != nullptr) delta_loc[it] = dl_out;
+        if (routed) delta_glb[ic] = dg;
         gate += dg;
       }
     }
@@ -147,6 +164,8 @@ struct BwdArgs {
   int kb_begin, kb_count;        // dK/dV kernel: key blocks [kb_begin, kb_begin + kb_count) of every KV head
   RowStrides dq_st, dk_st, dv_st;   // strides of the gradient tensors in elements
   float* dq_acc;                 // fused mode: fp32 [B, Lq, Hq, D] accumulator of dQ
+  int vis_shift;                 // global items see the keys 0 .. pos - vis_shift: 0, or W + 1 when the window's share of
+                                 // the global gradient is carried by the local items (shared-window backward)
   const int32_t* q_idx;
   const int32_t* n_routed;
   const int32_t* prefix;
@@ -222,8 +241,10 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
   const int32_t* q_idx_b = a.q_idx + (int64_t)b * a.Lq;
   const int w_eff = a.global_mode ? 0x3fffffff : a.window;
   const int last = min(row0 + kTileM - 1, n_rows - 1);
-  const int min_pos = (a.global_mode ? q_idx_b[row0] : row0) + a.q_pos_offset;
-  const int max_pos = (a.global_mode ? q_idx_b[last] : last) + a.q_pos_offset;
+  const int vis_shift = a.global_mode ? a.vis_shift : 0;
+  const int min_pos = (a.global_mode ? q_idx_b[row0] : row0) + a.q_pos_offset - vis_shift;   // last visible key
+  const int max_pos = (a.global_mode ? q_idx_b[last] : last) + a.q_pos_offset - vis_shift;
+  if (max_pos < 0) return;    // (shared-window backward) no row of the tile has a key before its window
   const int jlo = (min_pos - w_eff > 0) ? (min_pos - w_eff) / kTileN : 0;
   const int jhi = max_pos / kTileN;
   const int n_blocks = jhi - jlo + 1;
@@ -374,7 +395,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ 
     const int row = row0 + r;
     const bool valid = row < n_rows;
     const int seq_row = valid ? (a.global_mode ? q_idx_b[row] : row) : -1;
-    const int pos = valid ? seq_row + a.q_pos_offset : -1;
+    const int pos = valid ? seq_row + a.q_pos_offset - vis_shift : -1;
     const int pos_lo = valid ? pos - w_eff : 0x7fffffff;
     const int64_t stat_idx = ((int64_t)b * a.Hq + h) * a.Lq + (valid ? row : 0);
     const float lse2 = valid ? (a.global_mode ? a.lse_glb : a.lse_loc)[stat_idx] * kLog2e : 0.f;
@@ -524,11 +545,13 @@ __device__ __forceinline__ ItemPlan make_plan(const BwdArgs& a, int b, int k0) {
   if (tmin < 0) tmin = 0;
   if (tmax < tmin || a.skip_local) { p.loc_t0 = 0; p.loc_nt = 0; }
   else { p.loc_t0 = tmin / kTileM; p.loc_nt = tmax / kTileM - p.loc_t0 + 1; }
-  // global: compact rows whose position is >= k0
+  // global: compact rows whose last visible key (position - vis_shift) is >= k0
   const int n_c = a.skip_global ? 0 : a.n_routed[b];
-  if (tmin > a.Lq - 1 || n_c == 0) { p.glb_t0 = 0; p.glb_nt = 0; }
+  long long tmin_g = (long long)k0 - a.q_pos_offset + a.vis_shift;
+  if (tmin_g < 0) tmin_g = 0;
+  if (tmin_g > a.Lq - 1 || n_c == 0) { p.glb_t0 = 0; p.glb_nt = 0; }
   else {
-    const int c_min = a.prefix[(int64_t)b * (a.Lq + 1) + tmin];
+    const int c_min = a.prefix[(int64_t)b * (a.Lq + 1) + (int)tmin_g];
     if (c_min >= n_c) { p.glb_t0 = 0; p.glb_nt = 0; }
     else { p.glb_t0 = c_min / kTileM; p.glb_nt = (n_c - 1) / kTileM - p.glb_t0 + 1; }
   }
@@ -667,7 +690,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         const int64_t si = ((int64_t)b * a.Hq + h) * a.Lq + (valid ? row : 0);
         r_lse[q] = valid ? __ldg(&lse[si]) * kLog2e : 0.f;
         r_delta[q] = valid ? __ldg(&dl[si]) : 0.f;
-        r_pos[q] = valid ? (glb ? __ldg(&a.q_idx[(int64_t)b * a.Lq + row]) : row) + a.q_pos_offset : -1;
+        r_pos[q] = valid ? (glb ? __ldg(&a.q_idx[(int64_t)b * a.Lq + row]) - a.vis_shift : row) + a.q_pos_offset : -1;
       }
     };
     load_item();
@@ -833,7 +856,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
               const int row = row0 + q * 32 + e + u;
-              pos[u] = row < n_rows ? (glb ? __ldg(&qi[row]) : row) + a.q_pos_offset : -1;
+              pos[u] = row < n_rows ? (glb ? __ldg(&qi[row]) - a.vis_shift : row) + a.q_pos_offset : -1;
             }
             float p0 = fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, -st[e]));
             float p1 = fast_exp2(fmaf(__uint_as_float(sv[e + 1]), a.scale_log2, -st[e + 1]));
@@ -1073,7 +1096,7 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         const int64_t si = ((int64_t)b * a.Hq + h) * a.Lq + (valid ? row : 0);
         r_lse[q] = valid ? __ldg(&lse[si]) * kLog2e : 0.f;
         r_delta[q] = valid ? __ldg(&dl[si]) : 0.f;
-        r_pos[q] = valid ? (glb ? __ldg(&a.q_idx[(int64_t)b * a.Lq + row]) : row) + a.q_pos_offset : -1;
+        r_pos[q] = valid ? (glb ? __ldg(&a.q_idx[(int64_t)b * a.Lq + row]) - a.vis_shift : row) + a.q_pos_offset : -1;
       }
     };
     load_item();
@@ -1235,7 +1258,7 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
               const int row = row0 + q * 32 + e + u;
-              pos[u] = row < n_rows ? (glb ? __ldg(&qi[row]) : row) + a.q_pos_offset : -1;
+              pos[u] = row < n_rows ? (glb ? __ldg(&qi[row]) - a.vis_shift : row) + a.q_pos_offset : -1;
             }
             float p0 = fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, -st[e]));
             float p1 = fast_exp2(fmaf(__uint_as_float(sv[e + 1]), a.scale_log2, -st[e + 1]));
@@ -1522,6 +1545,10 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   float* lse_c = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + 2 * stat_bytes(p));
   float* dq_acc = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + 3 * stat_bytes(p));
   const bool fused = p->flags & L2A_FLAG_FUSED_DQ;
+  // Shared-window backward: the window's share of a routed row's global gradient rides on the local items (see
+  // bwd_delta_kernel).  Needs the same gradient for both outputs; the flag permits it, other modes just ignore it.
+  const bool share = (p->flags & L2A_FLAG_SHARED_WINDOW) && dS_loc == dO && !skip_local && !skip_global &&
+                     !force_all && !fused;
 
   CUtensorMap mapQ, mapDO, mapQc, mapDOc, mapK, mapV;
   const RowStrides qs = resolve_strides(p->q_stride, p->Lq, p->Hq * p->D);
@@ -1561,7 +1588,7 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
                                           static_cast<const bf16*>(skip_local ? nullptr : S_save),
                                           static_cast<const bf16*>(A_c), skip_global ? nullptr : d_mask, prefix,
                                           delta_loc, delta_glb, dgate, p->B, p->Lq, p->Hq,
-                                          force_all ? 1 : 0, os.b, os.t);
+                                          force_all ? 1 : 0, os.b, os.t, lse_loc, lse_glb, share ? lse_c : nullptr);
     if (cudaGetLastError() != cudaSuccess) return L2A_ERR_CUDA;
     if (force_all) {
       dim3 grid((p->Lq + 255) / 256, p->Hq, p->B);
@@ -1580,7 +1607,8 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   a.skip_local = skip_local ? 1 : 0;
   a.skip_global = skip_global ? 1 : 0;
   a.q_idx = q_idx; a.n_routed = n_routed; a.prefix = prefix;
-  a.lse_loc = lse_loc; a.lse_glb = force_all ? lse_c : lse_glb; a.delta_loc = delta_loc; a.delta_glb = delta_glb;
+  a.lse_loc = share ? lse_c : lse_loc; a.lse_glb = force_all ? lse_c : lse_glb;
+  a.vis_shift = share ? (p->window < (1 << 30) ? p->window : (1 << 30)) + 1 : 0; a.delta_loc = delta_loc; a.delta_glb = delta_glb;
   a.dQ = static_cast<bf16*>(dQ); a.dK = static_cast<bf16*>(dK); a.dV = static_cast<bf16*>(dV);
   a.dq_st = qs; a.dk_st = ks; a.dv_st = vs;
   a.dq_acc = fused ? dq_acc : nullptr;

@@ -27,14 +27,20 @@ def sample_rows(d_row: np.ndarray, n: int, seed: int) -> np.ndarray:
     return np.sort(np.concatenate([fixed, pick_r, pick])).astype(np.int32)
 
 
-def setup(name, rho=None, backward=False, sweep=0):
+# both launch configurations bench.py can time: plain, and with the shared-projection fusion
+SHARED = pytest.mark.parametrize("shared", [False, True], ids=["plain", "shared_window"])
+
+
+def setup(name, rho=None, backward=False, sweep=0, shared=False):
     cfg = synth.CONFIGS[name]
     seed = synth.seed_for(synth.CONFIG_INDEX[name], sweep)
     d, logits = synth.routing(cfg, seed, density=rho)
     host = synth.qkv(cfg.B, cfg.L, cfg.Hq, cfg.Hkv, cfg.D, seed, with_dO=backward)
     p = l2a.params(cfg.B, cfg.L, cfg.L, cfg.Hq, cfg.Hkv, cfg.D, cfg.W,
-                   flags=l2a.FLAG_SAVE_FOR_BWD if backward else 0)
+                   flags=(l2a.FLAG_SAVE_FOR_BWD if backward else 0) | (l2a.FLAG_SHARED_WINDOW if shared else 0))
     buf = l2a.Buffers.allocate(p, backward=backward, router_dtype=torch.float32 if logits is not None else torch.uint8)
+    if shared and not backward:
+        buf.lse_loc = torch.empty((cfg.B, cfg.Hq, cfg.L), dtype=torch.float32, device="cuda")
     for k in ("Q", "K", "V") + (("dO",) if backward else ()):
         getattr(buf, k).copy_(host[k])
     buf.router.copy_(torch.from_numpy(logits if logits is not None else d))
@@ -76,9 +82,10 @@ def test_forward_128k_sampled_rows():
     assert torch.isfinite(buf.O.float()).all()
 
 
-def test_forward_32k_sampled_rows():
+@SHARED
+def test_forward_32k_sampled_rows(shared):
     """Qwen2.5-7B-shaped 32K forward (28 query / 4 KV heads), Bernoulli(0.2)."""
-    cfg, d, buf, sh, u16 = setup("qwen25_7b_32k")
+    cfg, d, buf, sh, u16 = setup("qwen25_7b_32k", shared=shared)
     rb, rh, rt, rows = rows_for_all_heads(cfg, d, seed=42)
     ref = oracle.forward_rows(sh, u16["Q"], u16["K"], u16["V"], d, rb, rh, rt)
     idx = torch.from_numpy(rows.astype(np.int64)).cuda()
@@ -87,9 +94,10 @@ def test_forward_32k_sampled_rows():
     check_close(got, want, "O (sampled rows, 32K)")
 
 
-def test_train_64k_forward_backward_sampled():
+@SHARED
+def test_train_64k_forward_backward_sampled(shared):
     """Training-step shape: L=65536, 28/4 heads, router logits ~ N(-1.4, 1) thresholded at 0 (about 8 % routed)."""
-    cfg, d, buf, sh, u16 = setup("train_64k", backward=True)
+    cfg, d, buf, sh, u16 = setup("train_64k", backward=True, shared=shared)
     assert 0.07 < d.mean() < 0.09
     rb, rh, rt, rows = rows_for_all_heads(cfg, d, seed=43)
     idx = torch.from_numpy(rows.astype(np.int64)).cuda()
@@ -112,10 +120,11 @@ def test_train_64k_forward_backward_sampled():
     check_close(to_f64(buf.dV[0].index_select(0, jt)[:, g]), dv, "dV (sampled keys, 64K)")
 
 
-def test_stress_128k_backward_identities_and_rows():
+@SHARED
+def test_stress_128k_backward_identities_and_rows(shared):
     """The benchmark's own workload (128K, clustered routing rho = 0.2, fwd + bwd): 1024 sampled dQ rows of every
     head, the dV column-sum identity, and finiteness of every output."""
-    cfg, d, buf, sh, u16 = setup("stress_128k", rho=0.2, backward=True, sweep=2)
+    cfg, d, buf, sh, u16 = setup("stress_128k", rho=0.2, backward=True, sweep=2, shared=shared)
     for t in (buf.O, buf.dQ, buf.dK, buf.dV):
         assert torch.isfinite(t.float()).all()
     rows = sample_rows(d[0], 1024, seed=44)

@@ -88,13 +88,36 @@ def test_shared_window_step_host_and_routed_forward(backward):
     if not backward:
         c.buf.lse_loc = torch.empty(B, Hq, L, dtype=torch.float32, device="cuda")
     c.run_forward()
-    want = c.buf.O.clone()
+    want = {"O": c.buf.O.clone()}
+    if backward:
+        run_backward(c)
+        want.update(dQ=c.buf.dQ.clone(), dK=c.buf.dK.clone(), dV=c.buf.dV.clone())
     host = {k: v.pin_memory() for k, v in c.host.items()}
     host["router"] = torch.from_numpy(d).pin_memory()
-    host["O"] = torch.empty_like(want, device="cpu").pin_memory()
-    if backward:
-        for k in ("dQ", "dK", "dV"):
-            host[k] = torch.empty_like(getattr(c.buf, k), device="cpu").pin_memory()
-    c.buf.O.zero_()
+    for k, w in want.items():
+        host[k] = torch.empty_like(w, device="cpu").pin_memory()
+        getattr(c.buf, k).zero_()
     l2a.l2a_step_host(c.p, host, c.buf, l2a.ROUTER_MASK_U8, 0.0)
-    assert torch.equal(host["O"].view(torch.int16), want.cpu().view(torch.int16))
+    for k, w in want.items():
+        assert torch.equal(host[k].view(torch.int16), w.cpu().view(torch.int16)), k
+
+
+def test_shared_window_split_backward_falls_back():
+    """With a separate gradient for the local output the two modules no longer share dP: the backward ignores the
+    flag there, bit-identical to the call without it."""
+    B, L, Hq, Hkv, D, W = 1, 900, 2, 1, 128, 200
+    d = synth.mask_bernoulli(B, L, 0.4, seed=6)
+    c = Case(B, L, Hq, Hkv, D, W, d, seed=41, backward=True)
+    c.run_forward()
+    run_backward(c)
+    want = {k: getattr(c.buf, k).clone() for k in ("dQ", "dK", "dV")}
+    b = c.buf
+    p = l2a.params(B, L, L, Hq, Hkv, D, W, flags=l2a.FLAG_SAVE_FOR_BWD | l2a.FLAG_SHARED_WINDOW)
+    dS_loc = b.dO.clone()
+    for t in (b.dQ, b.dK, b.dV):
+        t.fill_(float("nan"))
+    l2a.l2a_backward_split(p, b.Q, b.K, b.V, b.d_mask, b.q_idx, b.n_routed, b.prefix, b.dO, dS_loc, b.S_save, b.A_c,
+                           b.lse_loc, b.lse_glb, b.dQ, b.dK, b.dV, None, b.bwd_ws)
+    torch.cuda.synchronize()
+    for k, w in want.items():
+        assert torch.equal(getattr(b, k).view(torch.int16), w.view(torch.int16)), k
