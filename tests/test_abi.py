@@ -73,3 +73,14 @@ def test_stride_arguments_are_validated_on_the_host():
         with pytest.raises(l2a.L2AError) as e:
             l2a.l2a_workspace_bytes(l2a.params(**ok, q_stride=bad))
         assert e.value.code == -1
+
+
+def test_flag_and_router_constants_match_the_header():
+    """The binding's constants are the header's #defines (same names without the L2A_ prefix)."""
+    text = open(os.path.join(ROOT, "include", "l2a.h")).read()
+    defines = {m.group(1): int(m.group(2)) for m in re.finditer(r"#define\s+L2A_((?:FLAG|ROUTER)_[A-Z0-9_]+)\s+(\d+)u?", text)}
+    assert len([k for k in defines if k.startswith("FLAG_")]) >= 7 and "ROUTER_MASK_U8" in defines
+    for name, value in defines.items():
+        assert getattr(l2a, name) == value, name
+    flags = [v for k, v in defines.items() if k.startswith("FLAG_")]
+    assert len(set(flags)) == len(flags) and all(v & (v - 1) == 0 for v in flags)   # distinct single bits
