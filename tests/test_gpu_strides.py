@@ -15,10 +15,11 @@ def _bits(t):
     return t.contiguous().view(torch.int16)
 
 
+@pytest.mark.parametrize("extra", [0, l2a.FLAG_SHARED_WINDOW], ids=["plain", "shared_window"])
 @pytest.mark.parametrize("B,L,Hq,Hkv,D,W", [(2, 700, 4, 2, 128, 100), (1, 1300, 6, 2, 64, 300)])
-def test_strided_tensors_match_dense(B, L, Hq, Hkv, D, W):
+def test_strided_tensors_match_dense(B, L, Hq, Hkv, D, W, extra):
     d = synth.mask_bernoulli(B, L, 0.3, seed=5)
-    c = Case(B, L, Hq, Hkv, D, W, d, seed=77, backward=True)
+    c = Case(B, L, Hq, Hkv, D, W, d, seed=77, backward=True, flags=extra)
     c.run_forward()
     run_backward(c)
     b = c.buf
@@ -41,7 +42,7 @@ def test_strided_tensors_match_dense(B, L, Hq, Hkv, D, W):
     dObuf = torch.zeros((B, L, opitch), dtype=torch.bfloat16, device="cuda")
     dObuf[:, :, :wq] = b.dO.view(B, L, wq)
     st = (Lpad * tok, tok)
-    p = l2a.params(B, L, L, Hq, Hkv, D, W, flags=l2a.FLAG_SAVE_FOR_BWD, q_stride=st, k_stride=st, v_stride=st,
+    p = l2a.params(B, L, L, Hq, Hkv, D, W, flags=l2a.FLAG_SAVE_FOR_BWD | extra, q_stride=st, k_stride=st, v_stride=st,
                    o_stride=(L * opitch, opitch))
     b.S_save.fill_(float("nan"))
     l2a.l2a_forward(p, Q, K, V, b.d_mask, b.q_idx, b.n_routed, b.prefix, Obuf, b.S_save, b.A_c, b.lse_loc, b.lse_glb,
