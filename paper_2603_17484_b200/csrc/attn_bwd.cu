@@ -99,6 +99,18 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const bf16* __restrict__
     const uint4* ps = reinterpret_cast<const uint4*>(S + row) + lane;
     const uint4* pa = reinterpret_cast<const uint4*>(A_c + crow) + lane;
     float gate = 0.f;
+    // shared-window statistics: the two log-sum-exps of head (32 j + lane), fetched ahead of the passes that need them
+    float pre_loc[2] = {0.f, 0.f}, pre_glb[2] = {0.f, 0.f};
+    if (lse_eff != nullptr) {
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int h = 32 * j + lane;
+        if (h < Hq) {
+          pre_loc[j] = __ldg(&lse_loc[((int64_t)b * Hq + h) * L + t]);
+          if (routed) pre_glb[j] = __ldg(&lse_glb[((int64_t)b * Hq + h) * L + c]);
+        }
+      }
+    }
 #pragma unroll 4
     for (int p = 0; p < n_pass; ++p) {
       const int h = p * kHeadsPerPass + sub;
@@ -113,17 +125,24 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const bf16* __restrict__
         dl += __shfl_xor_sync(0xffffffffu, dl, off);
         dg += __shfl_xor_sync(0xffffffffu, dg, off);
       }
+      // (every lane takes part in the shuffles; heads beyond 64 fall back to loads in place)
+      float pre_l = __shfl_sync(0xffffffffu, (h & 32) ? pre_loc[1] : pre_loc[0], h & 31);
+      float pre_g = __shfl_sync(0xffffffffu, (h & 32) ? pre_glb[1] : pre_glb[0], h & 31);
       if (h < Hq && (lane % kLanesPerHead) == 0) {
         const int64_t it = ((int64_t)b * Hq + h) * L + t, ic = ((int64_t)b * Hq + h) * L + c;
+        if (lse_eff != nullptr && h >= 64) {
+          pre_l = lse_loc[it];
+          pre_g = routed ? lse_glb[ic] : 0.f;
+        }
         float dl_out = dl;
         if (lse_eff != nullptr) {
           // Shared-window backward.  Inside the window of a routed row P_glb = beta * P_loc with
           // beta = exp(lse_loc - lse_glb), and dP is the same product dO V^T for both modules, so the two
           // contributions add up to P' (dP - Delta') with P' = (1 + beta) P_loc and
           // Delta' = (Delta_loc + beta * Delta_glb) / (1 + beta): the local items carry them with these statistics.
-          float le = lse_loc[it];
+          float le = pre_l;
           if (routed) {
-            const float beta = __expf(le - lse_glb[ic]);
+            const float beta = __expf(le - pre_g);
             dl_out = (dl + beta * dg) / (1.0f + beta);
             le -= log1pf(beta);
           }
