@@ -16,26 +16,27 @@ def _bits(t):
     return t.cpu().view(torch.int16).numpy().view(np.uint16)
 
 
-def test_forward_routed_equals_the_four_calls():
+@pytest.mark.parametrize("extra", [0, l2a.FLAG_SHARED_WINDOW], ids=["plain", "shared_window"])
+def test_forward_routed_equals_the_four_calls(extra):
     B, L, Hq, Hkv, D, W = 2, 1300, 4, 2, 128, 160
     rng = np.random.default_rng(5)
     w = torch.from_numpy((rng.standard_normal(Hq * D) * 0.5).astype(np.float32)).cuda()
     bias = 0.1
     out = {}
     for mode in ("four_calls", "one_call"):
-        c = Case(B, L, Hq, Hkv, D, W, np.zeros((B, L), np.uint8), seed=31, backward=True)
+        c = Case(B, L, Hq, Hkv, D, W, np.zeros((B, L), np.uint8), seed=31, backward=True, flags=extra)
         b = c.buf
         logits = torch.empty((B, L), dtype=torch.float32, device="cuda")
         sum_sq = torch.empty((B,), dtype=torch.float32, device="cuda")
         b.O.fill_(float("nan"))
         if mode == "four_calls":
-            p1 = l2a.params(B, L, L, Hq, Hkv, D, W, flags=l2a.FLAG_SAVE_FOR_BWD | l2a.FLAG_SKIP_GLOBAL)
+            p1 = l2a.params(B, L, L, Hq, Hkv, D, W, flags=l2a.FLAG_SAVE_FOR_BWD | l2a.FLAG_SKIP_GLOBAL | extra)
             l2a.l2a_forward(p1, b.Q, b.K, b.V, b.d_mask, b.q_idx, b.n_routed, b.prefix, b.O, b.S_save, b.A_c,
                             b.lse_loc, b.lse_glb, b.fwd_ws)
             l2a.l2a_router_logits(p1, b.S_save, w, bias, logits, sum_sq)
             l2a.l2a_route_compact(p1, logits, l2a.ROUTER_LOGITS_F32, 0.0, b.d_mask, b.q_idx, b.n_routed, b.prefix,
                                   b.route_ws)
-            p2 = l2a.params(B, L, L, Hq, Hkv, D, W, flags=l2a.FLAG_SAVE_FOR_BWD | l2a.FLAG_GLOBAL_PHASE)
+            p2 = l2a.params(B, L, L, Hq, Hkv, D, W, flags=l2a.FLAG_SAVE_FOR_BWD | l2a.FLAG_GLOBAL_PHASE | extra)
             l2a.l2a_forward(p2, b.Q, b.K, b.V, b.d_mask, b.q_idx, b.n_routed, b.prefix, b.O, b.S_save, b.A_c,
                             b.lse_loc, b.lse_glb, b.fwd_ws)
         else:
