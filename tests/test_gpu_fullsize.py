@@ -79,11 +79,12 @@ def rows_for_all_heads(cfg, d, seed):
     return np.zeros_like(rt_all), rh, rt_all, rt
 
 
-def test_forward_128k_sampled_rows():
+@SHARED
+def test_forward_128k_sampled_rows(shared):
     """Qwen3-8B-shaped 128K prefill forward, Bernoulli(0.2): 4096 sampled rows of every head."""
-    cfg, d, buf, sh, u16 = setup("qwen3_8b_128k", rho=0.2, sweep=2)
+    cfg, d, buf, sh, u16 = setup("qwen3_8b_128k", rho=0.2, sweep=2, shared=shared)
     rb, rh, rt, rows = rows_for_all_heads(cfg, d, seed=41)
-    ref = oracle.forward_rows(sh, u16["Q"], u16["K"], u16["V"], d, rb, rh, rt)
+    ref = once("fwd128k", lambda: oracle.forward_rows(sh, u16["Q"], u16["K"], u16["V"], d, rb, rh, rt))
     idx = torch.from_numpy(rows.astype(np.int64)).cuda()
     got = to_f64(buf.O[0].index_select(0, idx))                      # [rows, Hq, D]
     want = ref["o"].reshape(cfg.Hq, rows.size, cfg.D).transpose(1, 0, 2)
