@@ -132,12 +132,12 @@ def test_train_64k_forward_backward_sampled(shared):
 
 @SHARED
 def test_stress_128k_backward_identities_and_rows(shared):
-    """The benchmark's own workload (128K, clustered routing rho = 0.2, fwd + bwd): 1024 sampled dQ rows of every
+    """The benchmark's own workload (128K, clustered routing rho = 0.2, fwd + bwd): 4096 sampled dQ rows of every
     head, the dV column-sum identity, and finiteness of every output."""
     cfg, d, buf, sh, u16 = setup("stress_128k", rho=0.2, backward=True, sweep=2, shared=shared)
     for t in (buf.O, buf.dQ, buf.dK, buf.dV):
         assert torch.isfinite(t.float()).all()
-    rows = sample_rows(d[0], 1024, seed=44)
+    rows = sample_rows(d[0], ROWS_PER_HEAD, seed=44)
     rh = np.repeat(np.arange(cfg.Hq, dtype=np.int32), rows.size)
     rt = np.tile(rows, cfg.Hq)
     want = once("dq128k", lambda: oracle.dq_rows(sh, u16["Q"], u16["K"], u16["V"], d, u16["dO"], np.zeros_like(rt), rh, rt))
