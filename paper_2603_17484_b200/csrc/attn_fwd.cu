@@ -337,20 +337,27 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         // pass 1: row maximum of this half (32 columns at a time: the scores are re-read from TMEM in pass 2
         // rather than kept in 64 registers)
         float mx = -INFINITY;
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t v[32];
-          tmem_ld32(s_addr + c * 32, v);
+        {
+          // both loads in flight before the one wait (nothing else is live in this pass)
+          uint32_t v0[32], v1[32];
+          tmem_ld32(s_addr, v0);
+          tmem_ld32(s_addr + 32, v1);
           tmem_ld_wait();
           if (partial) {
 #pragma unroll
             for (int e = 0; e < 32; ++e) {
-              const int kp = k0 + c * 32 + e;
-              if (kp <= pos && kp >= pos_lo) mx = fmaxf(mx, __uint_as_float(v[e]));
+              const int kp = k0 + e;
+              if (kp <= pos && kp >= pos_lo) mx = fmaxf(mx, __uint_as_float(v0[e]));
+              if (kp + 32 <= pos && kp + 32 >= pos_lo) mx = fmaxf(mx, __uint_as_float(v1[e]));
             }
           } else {
+            float mx1 = -INFINITY;
 #pragma unroll
-            for (int e = 0; e < 32; e += 2) mx = fmax3(mx, __uint_as_float(v[e]), __uint_as_float(v[e + 1]));
+            for (int e = 0; e < 32; e += 2) {
+              mx = fmax3(mx, __uint_as_float(v0[e]), __uint_as_float(v0[e + 1]));
+              mx1 = fmax3(mx1, __uint_as_float(v1[e]), __uint_as_float(v1[e + 1]));
+            }
+            mx = fmaxf(mx, mx1);
           }
         }
         // row maximum over both halves: publish mine, meet the other half, read theirs
