@@ -131,6 +131,28 @@ l2a_status l2a_workspace_bytes(const l2a_params* p, size_t* route_ws_bytes, size
                                size_t* bwd_ws_bytes);
 
 /*
+ * Self-test of the bounded device-side wait (the mechanism behind L2A_ERR_DEVICE_TIMEOUT).  Launches one small
+ * kernel in which a warp waits, with a limit of `limit_us` microseconds (1 .. 1000000), for an mbarrier arrival that
+ * never comes, while the other warps wait for something else: the first wait runs out, raises the CTA's abort flag,
+ * the other warps leave their waits on seeing it, and the CTA writes the status word of workspace `ws` (any 256-byte
+ * aligned device buffer of at least 256 bytes) -- the path every kernel of this library takes when a wait runs
+ * out.  Afterwards l2a_workspace_status(ws) returns L2A_ERR_DEVICE_TIMEOUT and the context stays usable.  Nothing
+ * traps, faults or spins without a limit.  Returns L2A_ERR_INVALID_ARG for a limit outside the range.
+ */
+l2a_status l2a_selftest_wait_timeout(void* ws, unsigned limit_us, void* stream);
+
+/*
+ * Self-test of the bounded device-side wait (the mechanism behind L2A_ERR_DEVICE_TIMEOUT).  Launches one small
+ * kernel in which a warp waits, with a limit of `limit_us` microseconds (1 .. 1000000), for an mbarrier arrival that
+ * never comes, while the other warps wait for something else: the first wait runs out, raises the CTA's abort flag,
+ * the other warps leave their waits on seeing it, and the CTA writes the status word of workspace `ws` (any 256-byte
+ * aligned device buffer of at least 256 bytes) -- the path every kernel of this library takes when a wait runs
+ * out.  Afterwards l2a_workspace_status(ws) returns L2A_ERR_DEVICE_TIMEOUT and the context stays usable.  Nothing
+ * traps, faults or spins without a limit.  Returns L2A_ERR_INVALID_ARG for a limit outside the range.
+ */
+l2a_status l2a_selftest_wait_timeout(void* ws, unsigned limit_us, void* stream);
+
+/*
  * Reads the status word the kernels of earlier calls left in workspace `ws` (any of the three).
  * Synchronises `stream`.  Returns L2A_OK, or L2A_ERR_DEVICE_TIMEOUT if a bounded device-side wait
  * ran out in some kernel that used this workspace since it was last used by a successful call.

@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include "l2a_common.cuh"
+#include "sm100_prims.cuh"
 
 namespace l2a {
 
@@ -107,6 +108,42 @@ l2a_status l2a_workspace_bytes(const l2a_params* p, size_t* route_ws_bytes, size
   if (fwd_ws_bytes) *fwd_ws_bytes = fwd_ws_size(p);
   if (bwd_ws_bytes) *bwd_ws_bytes = l2a::bwd_ws_size(p);
   return L2A_OK;
+}
+
+namespace l2a {
+namespace {
+// The path a kernel takes when one of its waits runs out, on its own: one warp waits (bounded) for an mbarrier
+// arrival that never comes, the other warps wait for the first one's outcome through the same abort flag, and the
+// CTA records the failure in the status word -- what every kernel of this library does at its end.
+__global__ void __launch_bounds__(128) wait_timeout_selftest_kernel(int* status, uint64_t limit_ns) {
+  __shared__ uint64_t never_arrives;
+  __shared__ uint64_t second;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&never_arrives, 1);
+    mbar_init(&second, 1);
+    abort_flag = 0;
+    fence_mbar_init();
+  }
+  __syncthreads();
+  volatile int* af = &abort_flag;
+  bool ok;
+  if (threadIdx.x < 32) ok = mbar_wait(&never_arrives, 0, af, limit_ns);   // gives up after limit_ns, raises the flag
+  else ok = mbar_wait(&second, 0, af, 1000 * limit_ns);                     // leaves as soon as the flag is up
+  __syncthreads();
+  if (threadIdx.x == 0 && abort_flag) atomicExch(status, 1);
+  (void)ok;
+}
+}  // namespace
+}  // namespace l2a
+
+l2a_status l2a_selftest_wait_timeout(void* ws, unsigned limit_us, void* stream) {
+  if (!ws || (reinterpret_cast<uintptr_t>(ws) % 256) != 0) return L2A_ERR_WORKSPACE;
+  if (limit_us == 0 || limit_us > 1000000u) return L2A_ERR_INVALID_ARG;   // at most one second
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(ws, 0, l2a::kWsHeaderBytes, s) != cudaSuccess) return L2A_ERR_CUDA;
+  l2a::wait_timeout_selftest_kernel<<<1, 128, 0, s>>>(static_cast<int*>(ws), (uint64_t)limit_us * 1000ull);
+  return cudaGetLastError() == cudaSuccess ? L2A_OK : L2A_ERR_CUDA;
 }
 
 l2a_status l2a_workspace_status(const void* ws, void* stream) {

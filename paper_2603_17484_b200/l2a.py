@@ -31,7 +31,7 @@ EXPORTS = (
     "l2a_version", "l2a_status_string", "l2a_workspace_bytes", "l2a_workspace_status",
     "l2a_route_compact", "l2a_forward", "l2a_backward", "l2a_step_host", "l2a_profile_next_call",
     "l2a_route_compact_static", "l2a_router_logits", "l2a_decode_workspace_bytes", "l2a_decode",
-    "l2a_backward_split", "l2a_router_backward", "l2a_forward_routed",
+    "l2a_backward_split", "l2a_router_backward", "l2a_forward_routed", "l2a_selftest_wait_timeout",
 )
 
 
@@ -117,6 +117,14 @@ def l2a_workspace_bytes(p: L2AParams) -> tuple[int, int, int]:
 
 def l2a_workspace_status(ws: torch.Tensor, stream=None) -> int:
     return lib().l2a_workspace_status(_ptr(ws), _stream(stream))
+
+
+def l2a_selftest_wait_timeout(ws: torch.Tensor, limit_us: int, stream=None, check=True) -> int:
+    """Runs the bounded-wait self-test kernel (a wait that nothing satisfies, limited to limit_us microseconds)."""
+    code = lib().l2a_selftest_wait_timeout(_ptr(ws), ctypes.c_uint(limit_us), _stream(stream))
+    if check:
+        _check(code, "l2a_selftest_wait_timeout")
+    return code
 
 
 def l2a_route_compact(p, router, router_kind, logit_threshold, d_mask, q_idx, n_routed, prefix, route_ws,
