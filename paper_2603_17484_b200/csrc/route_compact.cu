@@ -151,9 +151,9 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const bf16* __restrict
   }
 }
 
-// Router logit (Eq. 3).  The grid is sized to the machine: every warp owns a contiguous range of tokens and takes
-// four of them at a time, so that each 32-byte piece of w fetched (from L1) serves four 16-byte loads of S and
-// several rows are in flight per warp; fp32 accumulation.
+// Router logit (Eq. 3).  The grid is sized to the machine: the warps take groups of four tokens round-robin (the
+// whole grid reads one contiguous stretch of S at a time), four at a time so that each 32-byte piece of w fetched
+// (from L1) serves four 16-byte loads of S and several rows are in flight per warp; fp32 accumulation.
 constexpr int kRlTokens = 4;
 __global__ void __launch_bounds__(256) router_logits_kernel(const bf16* __restrict__ S, const float* __restrict__ w,
                                                             float bias, float* __restrict__ logits,
@@ -162,13 +162,14 @@ __global__ void __launch_bounds__(256) router_logits_kernel(const bf16* __restri
   const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
   const int64_t gw = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
-  const int64_t t_begin = n_tokens * gw / n_warps, t_end = n_tokens * (gw + 1) / n_warps;
+  const int64_t t_begin = gw * kRlTokens, t_end = n_tokens;
   const int n_chunks = row_elems / 8;
   const float4* w4 = reinterpret_cast<const float4*>(w);
-  // sum of sigmoid^2 of this warp's tokens, flushed with one atomic per batch entry the range touches
+  // sum of sigmoid^2 of this warp's tokens, flushed with one atomic per batch entry they touch (the batch index
+  // never decreases along a warp's tokens)
   float reg_sum = 0.f;
-  int64_t reg_b = t_begin / L;
-  for (int64_t token0 = t_begin; token0 < t_end; token0 += kRlTokens) {
+  int64_t reg_b = t_begin < t_end ? t_begin / L : 0;
+  for (int64_t token0 = t_begin; token0 < t_end; token0 += n_warps * kRlTokens) {
     const uint4* rows[kRlTokens];
     float acc[kRlTokens];
 #pragma unroll
