@@ -152,3 +152,22 @@ def test_stress_128k_backward_identities_and_rows(shared):
     # every dV entry carries a bf16 rounding of relative size 2^-9; they add up like a random walk
     scale = buf.dV[0].float().abs().mean().item() * 2.0 ** -9 * np.sqrt(cfg.L) * 8 + 1.0
     assert (got_sum - want_sum).abs().max().item() <= scale, ((got_sum - want_sum).abs().max().item(), scale)
+
+
+def test_stress_128k_shared_window_agrees_with_independent_modules_everywhere():
+    """Every element of O, dQ, dK, dV of the benchmark workload, computed with and without the shared-window fusion:
+    two bf16 results of the same quantity, each within the bound of the exact value, so within twice the bound of
+    each other (the sampled-row tests above tie both to the oracle; this one covers every tile of the launch)."""
+    outs = []
+    for shared in (False, True):
+        cfg, d, buf, sh, u16 = setup("stress_128k", rho=0.2, backward=True, sweep=2, shared=shared)
+        outs.append({k: getattr(buf, k).float() for k in ("O", "dQ", "dK", "dV")})
+        del buf
+        torch.cuda.empty_cache()
+    for k in ("O", "dQ", "dK", "dV"):
+        a, b = outs[0][k], outs[1][k]
+        err = (a - b).abs()
+        bound = 2 * (2e-2 + 2.0 ** -8 * a.abs())
+        n_over = int((err > bound).sum().item())
+        assert n_over <= max(1, int(1e-5 * err.numel())), (k, n_over, err.max().item())
+        assert err.mean().item() <= 2 * (2e-3 + 2.0 ** -9 * a.abs().mean().item()), (k, err.mean().item())
