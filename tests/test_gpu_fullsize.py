@@ -171,3 +171,33 @@ def test_stress_128k_shared_window_agrees_with_independent_modules_everywhere():
         n_over = int((err > bound).sum().item())
         assert n_over <= max(1, int(1e-5 * err.numel())), (k, n_over, err.max().item())
         assert err.mean().item() <= 2 * (2e-3 + 2.0 ** -9 * a.abs().mean().item()), (k, err.mean().item())
+
+
+@SHARED
+def test_forward_128k_constant_values_every_row(shared):
+    """V = c for every key (one vector per KV head): every soft-max average is c, so o_t = (1 + d_t) c for every row
+    of the 128K launch, whatever the scores are -- a check of every tile, mask edge and scatter of the forward."""
+    cfg = synth.CONFIGS["stress_128k"]
+    seed = synth.seed_for(synth.CONFIG_INDEX["stress_128k"], 3)
+    d, _ = synth.routing(cfg, seed, density=0.2)
+    p = l2a.params(cfg.B, cfg.L, cfg.L, cfg.Hq, cfg.Hkv, cfg.D, cfg.W,
+                   flags=l2a.FLAG_SAVE_FOR_BWD | (l2a.FLAG_SHARED_WINDOW if shared else 0))
+    buf = l2a.Buffers.allocate(p, backward=True)
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    buf.Q.copy_(torch.randn(buf.Q.shape, generator=g, device="cuda"))
+    buf.K.copy_(torch.randn(buf.K.shape, generator=g, device="cuda"))
+    c = torch.randn((cfg.Hkv, cfg.D), generator=g, device="cuda").to(torch.bfloat16)
+    buf.V.copy_(c.expand(cfg.B, cfg.L, cfg.Hkv, cfg.D))
+    buf.router.copy_(torch.from_numpy(d))
+    buf.O.fill_(float("nan"))
+    buf.route()
+    buf.forward()
+    torch.cuda.synchronize()
+    assert l2a.l2a_workspace_status(buf.fwd_ws) == 0
+    G = cfg.Hq // cfg.Hkv
+    want = c.float().repeat_interleave(G, dim=0)[None, None] * (1.0 + buf.d_mask.float())[:, :, None, None]
+    err = (buf.O.float() - want).abs()
+    bound = 2e-2 + 2.0 ** -8 * want.abs()
+    assert torch.isfinite(buf.O.float()).all()
+    assert int((err > bound).sum().item()) == 0, err.max().item()
+    assert err.mean().item() <= 2e-3 + 2.0 ** -9 * want.abs().mean().item()
