@@ -201,3 +201,24 @@ def test_forward_128k_constant_values_every_row(shared):
     assert torch.isfinite(buf.O.float()).all()
     assert int((err > bound).sum().item()) == 0, err.max().item()
     assert err.mean().item() <= 2e-3 + 2.0 ** -9 * want.abs().mean().item()
+
+
+@SHARED
+def test_stress_128k_backward_is_reproducible_and_linear_in_dO(shared):
+    """The default backward has no atomics: a second run gives the same bits in every element of the 128K launch, and
+    doubling dO (exact in bf16 and fp32) doubles every gradient element exactly.  Races, stale tiles or order-dependent
+    sums anywhere in the launch would show up here."""
+    cfg, d, buf, sh, u16 = setup("stress_128k", rho=0.2, backward=True, sweep=2, shared=shared)
+    first = {k: getattr(buf, k).clone() for k in ("dQ", "dK", "dV")}
+    for k in first:
+        getattr(buf, k).fill_(float("nan"))
+    buf.backward()
+    torch.cuda.synchronize()
+    for k, v in first.items():
+        assert torch.equal(getattr(buf, k).view(torch.int16), v.view(torch.int16)), k
+    buf.dO.mul_(2.0)
+    buf.backward()
+    torch.cuda.synchronize()
+    assert l2a.l2a_workspace_status(buf.bwd_ws) == 0
+    for k, v in first.items():
+        assert torch.equal(getattr(buf, k).float(), 2.0 * v.float()), k
