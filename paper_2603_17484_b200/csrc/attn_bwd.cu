@@ -1619,7 +1619,7 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   pe.mark(s);
   BwdArgs a;
   a.B = p->B; a.Lq = p->Lq; a.Lk = p->Lk; a.Hq = p->Hq; a.Hkv = p->Hkv; a.D = p->D;
-  a.window = p->window;
+  a.window = p->window < (1 << 30) ? p->window : (1 << 30);   // any window >= Lk is the same
   a.q_pos_offset = p->q_pos_offset;
   a.scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->D);
   a.scale_log2 = a.scale * kLog2e;

@@ -257,7 +257,7 @@ static l2a_status forward_range(const l2a_params* p, const void* Q, const void* 
 
   FwdArgs a;
   a.B = p->B; a.Lq = p->Lq; a.Lk = p->Lk; a.Hq = p->Hq; a.Hkv = p->Hkv; a.D = p->D;
-  a.window = p->window;
+  a.window = p->window < (1 << 30) ? p->window : (1 << 30);   // any window >= Lk is the same; keeps W + 1 in range
   a.q_pos_offset = p->q_pos_offset;
   a.scale_log2 = scale_of(p) * 1.4426950408889634f;
   a.q_idx = q_idx;

@@ -21,6 +21,7 @@ pytestmark = pytest.mark.gpu
     (1, 1000, 1000, 1, 1, 128, 0, 0.5),      # W = 0: the window is the token itself
     (1, 1300, 1300, 2, 2, 128, 127, 1.0),    # all routed, window edge one short of a key block
     (1, 1, 1, 1, 1, 128, 4, 1.0),
+    (1, 300, 300, 2, 1, 128, 2 ** 31 - 1, 0.5),   # the largest window the ABI accepts
 ])
 def test_shared_window_forward_backward(B, Lq, Lk, Hq, Hkv, D, W, rho):
     d = synth.mask_bernoulli(B, Lq, rho, seed=Lq + W)
