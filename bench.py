@@ -245,6 +245,61 @@ def run_router(args):
         "gpu_launches": steps}), flush=True)
 
 
+def run_paper_table(args):
+    """The paper's short-context kernel table (its App. D: sparse Global Attention kernel + preprocessing at 4096 and
+    8192 tokens, 28 heads, d = 128, by sparsity = 1 - routed fraction), on this build: route/compact + gather + global
+    forward only (L2A_FLAG_SKIP_LOCAL), and the same with the global backward.  Context beside the paper's H200
+    figures, not the headline metric; these inputs fit in L2, as they do in the paper's table."""
+    from paper_2603_17484_b200 import l2a
+    torch.cuda.set_device(0)
+    Hq, Hkv, D = 28, 4, 128
+    steps, warm = max(args.steps, 20), max(3, args.warmup)
+    rows = []
+    for L in (4096, 8192):
+        for sparsity in (0.0, 0.2, 0.5, 0.8, 0.9, 0.95):
+            d = np.ones((1, L), np.uint8) if sparsity == 0.0 else synth.mask_bernoulli(1, L, 1.0 - sparsity, seed=L + int(100 * sparsity))
+            fl = l2a.FLAG_SAVE_FOR_BWD
+            p_all = l2a.params(1, L, L, Hq, Hkv, D, L, flags=fl)
+            buf = l2a.Buffers.allocate(p_all, backward=True)
+            for t in (buf.Q, buf.K, buf.V, buf.dO):
+                t.normal_()
+            buf.router.copy_(torch.from_numpy(d))
+            buf.route(); buf.forward()          # S_save, lse_loc for the backward call's signature
+            p_glb = l2a.params(1, L, L, Hq, Hkv, D, L, flags=l2a.FLAG_SKIP_LOCAL)
+            p_glb_b = l2a.params(1, L, L, Hq, Hkv, D, L, flags=fl | l2a.FLAG_SKIP_LOCAL)
+
+            def fwd():
+                buf.route()
+                l2a.l2a_forward(p_glb, buf.Q, buf.K, buf.V, buf.d_mask, buf.q_idx, buf.n_routed, buf.prefix, buf.O,
+                                None, None, None, None, buf.fwd_ws)
+
+            def bwd():
+                l2a.l2a_backward(p_glb_b, buf.Q, buf.K, buf.V, buf.d_mask, buf.q_idx, buf.n_routed, buf.prefix, buf.dO,
+                                 None, buf.A_c, None, buf.lse_glb, buf.dQ, buf.dK, buf.dV, None, buf.bwd_ws)
+
+            def timed(fn):
+                for _ in range(warm):
+                    fn()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                e0.record()
+                for _ in range(steps):
+                    fn()
+                e1.record()
+                torch.cuda.synchronize()
+                return e0.elapsed_time(e1) / steps
+            rows.append({"L": L, "sparsity": sparsity, "routed": int(d.sum()), "fwd_ms": timed(fwd), "bwd_ms": timed(bwd)})
+            del buf
+    print(json.dumps({
+        "metric": "sparse Global Attention kernel + preprocessing, short contexts (paper's kernel table)", "unit": "ms",
+        "value": rows[-1]["fwd_ms"], "n_gpus": 1, "steps": steps, "warmup": warm, "higher_is_better": False,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "paper_kernel_table", "B": 1, "Hq": Hq, "Hkv": Hkv, "D": D,
+                   "l2_policy": "inputs fit in L2, as in the paper's table; no flush",
+                   "note": "forward = route/compact + gather + global forward; backward = global backward of the same rows"},
+        "rows": rows, "gpu_launches": 4 * steps}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -265,6 +320,8 @@ def main():
     ap.add_argument("--decode", action="store_true", help="measure the decode step instead (HBM roofline)")
     ap.add_argument("--decode-batch", type=int, default=16)
     ap.add_argument("--router", action="store_true", help="measure the router kernels instead (HBM roofline)")
+    ap.add_argument("--paper-table", action="store_true",
+                    help="the paper's short-context kernel table on this build (context, not the headline)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -274,6 +331,8 @@ def main():
         return run_decode(args)
     if args.router:
         return run_router(args)
+    if args.paper_table:
+        return run_paper_table(args)
 
     from paper_2603_17484_b200 import l2a
 
