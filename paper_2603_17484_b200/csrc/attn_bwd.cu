@@ -183,7 +183,8 @@ struct BwdArgs {
   int skip_local, skip_global;   // gradients of one module only (the other module has its own Q/K/V)
   int kb_begin, kb_count;        // dK/dV kernel: key blocks [kb_begin, kb_begin + kb_count) of every KV head
   RowStrides dq_st, dk_st, dv_st;   // strides of the gradient tensors in elements
-  float* dq_acc;                 // fused mode: fp32 [B, Lq, Hq, D] accumulator of dQ
+  float* dq_acc_loc;             // five-GEMM mode: fp32 dQ accumulators (layout: see bwd_fused_kernel), by row tile
+  float* dq_acc_glb;             //                 and by compact tile; NULL when that module is skipped
   int vis_shift;                 // global items see the keys 0 .. pos - vis_shift: 0, or W + 1 when the window's share of
                                  // the global gradient is carried by the local items (shared-window backward)
   const int32_t* q_idx;
@@ -963,15 +964,21 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 }
 
 // ================================================================================================
-// Fused backward kernel (L2A_FLAG_FUSED_DQ): the dK/dV kernel above plus the fifth GEMM, dQ(i) = dS(i) K, so that S and
-// dP are computed once (five GEMMs per tile pair instead of seven).  dQ(i) is a fresh 128 x D accumulator per item:
-// it borrows the S^T columns (S^T(i) is in registers by then), is read out by the compute warps (lane = query row)
-// and added to an fp32 dQ buffer in global memory with red.global.add.v4.f32 -- local and global contributions
-// and all key blocks meet there, in no fixed order, so dQ is not bit-reproducible from run to run in this mode.
-// dS is needed twice: transposed in TMEM (A operand of dK, as above) and in shared memory, [key][query], read
-// MN-major as the A operand of dQ; it takes the place of the third Q stage.
-//   TMEM: dV [0,D) | dK [D,2D) | T [256,384): S^T(i), then dQ(i) | U [384,512): dP^T(i), then P^T(i) | dS^T(i).
-//   MMA order per item i:  dQ(i) | dV(i) | dK(i) | S^T(i+1) (after dQ(i) was read out) | dP^T(i+1).
+// Five-GEMM backward kernel: the key/value-stationary kernel above plus the fifth GEMM, dQ(i) = dS(i) K, so that
+// S and dP are computed once per tile pair.  dQ(i) is a fresh 128 x D accumulator per item; the compute warps read
+// it out (lane = query row) and add it into an fp32 accumulator in global memory whose layout is private to this
+// file: per (batch, head, 128-row tile) one block of 128 x D floats ordered [warp 16][piece D/16][lane 32][4], so
+// that every red.global.add.v4.f32 of a warp covers 512 contiguous bytes.  Local items add into the accumulator
+// indexed by row tile, global items into the one indexed by compact tile; dq_merge_kernel forms the bf16 dQ.
+// All key blocks meet in those accumulators in no fixed order: dQ is not bit-reproducible from run to run
+// (dK, dV are).
+//   TMEM: dV [0,D) | dK [D,2D) | T [256,384): S^T(i), then P^T(i) (bf16, quarter-local) | U [384,512): dP^T(i),
+//         then dQ(i).
+//   Shared memory: K, V resident; Q and dO in two-stage rings; dS(i) (bf16, [key][query], swizzled like a TMA
+//   tile) -- the A operand of both dK += dS^T Q (read K-major) and dQ = dS K (read MN-major).
+//   MMA order per item i:  dK(i-1) | dV(i) | dQ(i) | S^T(i+1) | dP^T(i+1).  Two loops run through the order with
+//   slack: T: S^T -> P -> dV -> S^T and U: dP^T -> dS -> dQ -> read-out -> dP^T; dK(i-1) fills the pipe while the
+//   exponentials of item i run.
 template <int D>
 struct FusedSmem {
   static constexpr int kTileBytes = 128 * D * 2;
@@ -990,10 +997,11 @@ struct FusedBarriers {
   uint64_t q_full[2], q_empty[2];
   uint64_t do_full[2], do_empty[2];
   uint64_t st_full[2], st_empty[2];
-  uint64_t s_full, dp_full, pds_full, dq_full, t_free, final_bar;
+  uint64_t s_full, dp_full, p_full, ds_full, ds_free, dq_full, u_free, final_bar;
   uint32_t tmem_base;
   int abort_flag;
 };
+static_assert(sizeof(FusedBarriers) <= 256, "barrier block");
 
 template <int D>
 __global__ void __launch_bounds__(kDkvThreads, 1)
@@ -1019,7 +1027,7 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
   uint8_t* sQ = smem + SM::kQOff;
   uint8_t* sDO = smem + SM::kDoOff;
   FusedBarriers* bar = reinterpret_cast<FusedBarriers*>(smem + SM::kBarOff);
-  uint8_t* sDS = smem + SM::kDsOff;          // dS (bf16, [key][query]) for dQ = dS K
+  uint8_t* sDS = smem + SM::kDsOff;          // dS (bf16, [key][query])
   volatile int* abort_flag = &bar->abort_flag;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -1042,16 +1050,18 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 
   if (tid == 0) {
     mbar_init(&bar->kv_full, 1);
-    for (int s = 0; s < 2; ++s) { mbar_init(&bar->q_full[s], 1); mbar_init(&bar->q_empty[s], 1); }
     for (int s = 0; s < 2; ++s) {
+      mbar_init(&bar->q_full[s], 1); mbar_init(&bar->q_empty[s], 1);
       mbar_init(&bar->do_full[s], 1); mbar_init(&bar->do_empty[s], 1);
       mbar_init(&bar->st_full[s], 32); mbar_init(&bar->st_empty[s], kComputeWarps * 32);
     }
     mbar_init(&bar->s_full, 1);
     mbar_init(&bar->dp_full, 1);
-    mbar_init(&bar->pds_full, kComputeWarps * 32);   // P^T, dS^T in TMEM and dS in shared memory
+    mbar_init(&bar->p_full, kComputeWarps * 32);     // P^T(i) is in TMEM
+    mbar_init(&bar->ds_full, kComputeWarps * 32);    // dS(i) is in shared memory and dP^T(i) has been read
+    mbar_init(&bar->ds_free, 1);                     // dQ(i) and dK(i) have consumed dS(i)
     mbar_init(&bar->dq_full, 1);                     // dQ(i) is in TMEM
-    mbar_init(&bar->t_free, kComputeWarps * 32);     // dQ(i) has been read out: the columns may take S^T(i+1)
+    mbar_init(&bar->u_free, kComputeWarps * 32);     // dQ(i) has been read out: the columns may take dP^T(i+1)
     mbar_init(&bar->final_bar, 1);
     bar->abort_flag = 0;
     fence_mbar_init();
@@ -1078,18 +1088,17 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       tma_load_4d(sK, &mapK, &bar->kv_full, 0, k0, g * (D / 64), b);
       tma_load_4d(sV, &mapV, &bar->kv_full, 0, k0, g * (D / 64), b);
       ItemCursor cur(plan, g * G);
-      int qs = 0;
-      uint32_t qph = 0;
       for (int i = 0; i < plan.total; ++i) {
         const int glb = cur.glb(), row0 = cur.tile() * kTileM, hc = cur.h * (D / 64);
         cur.next();
-        if (!mbar_wait(&bar->q_empty[qs], qph ^ 1, abort_flag)) break;
-        mbar_expect_tx(&bar->q_full[qs], SM::kTileBytes);
-        tma_load_4d(sQ + qs * SM::kTileBytes, glb ? &mapQc : &mapQ, &bar->q_full[qs], 0, row0, hc, b);
-        if (!mbar_wait(&bar->do_empty[i & 1], ((i >> 1) & 1) ^ 1, abort_flag)) break;
-        mbar_expect_tx(&bar->do_full[i & 1], SM::kTileBytes);
-        tma_load_4d(sDO + (i & 1) * SM::kTileBytes, glb ? &mapDOc : &mapDO, &bar->do_full[i & 1], 0, row0, hc, b);
-        if (++qs == 2) { qs = 0; qph ^= 1; }
+        const int st = i & 1;
+        const uint32_t ph = ((i >> 1) & 1) ^ 1;
+        if (!mbar_wait(&bar->q_empty[st], ph, abort_flag)) break;
+        mbar_expect_tx(&bar->q_full[st], SM::kTileBytes);
+        tma_load_4d(sQ + st * SM::kTileBytes, glb ? &mapQc : &mapQ, &bar->q_full[st], 0, row0, hc, b);
+        if (!mbar_wait(&bar->do_empty[st], ph, abort_flag)) break;
+        mbar_expect_tx(&bar->do_full[st], SM::kTileBytes);
+        tma_load_4d(sDO + st * SM::kTileBytes, glb ? &mapDOc : &mapDO, &bar->do_full[st], 0, row0, hc, b);
       }
     }
     __syncwarp();
@@ -1155,6 +1164,7 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       const uint64_t dk = smem_desc_sw128(smem_u32(sK), 16, 1024), dv = smem_desc_sw128(smem_u32(sV), 16, 1024);
       const uint64_t dkm = smem_desc_sw128(smem_u32(sK), kBoxBytes, 1024);            // K as MN-major B of dQ
       const uint64_t dsm = smem_desc_sw128(smem_u32(sDS), kBoxBytes, 1024);           // dS as MN-major A of dQ
+      const uint64_t dsk = smem_desc_sw128(smem_u32(sDS), 16, 1024);                  // dS^T as K-major A of dK
       const uint64_t dq_base = smem_desc_sw128(smem_u32(sQ), 16, 1024);
       const uint64_t ddo_base = smem_desc_sw128(smem_u32(sDO), 16, 1024);
       const uint64_t dqm_base = smem_desc_sw128(smem_u32(sQ), kBoxBytes, 1024);      // Q / dO as MN-major B
@@ -1168,7 +1178,7 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         }
         tc_commit(&bar->s_full, leader);
       };
-      auto issue_dP = [&](int ds) {   // dP^T = V dO^T
+      auto issue_dP = [&](int ds) {   // dP^T = V dO^T into the U columns
         const uint64_t dod = ddo_base + ds * kStageStep;
 #pragma unroll
         for (int kk = 0; kk < kKSteps; ++kk) {
@@ -1177,27 +1187,29 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         }
         tc_commit(&bar->dp_full, leader);
       };
-      auto issue_dQ = [&]() {         // dQ(i) = dS K into the T columns (a fresh accumulator for every item)
+      auto issue_dQ = [&]() {         // dQ(i) = dS K into the U columns (a fresh accumulator for every item)
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
-          mma_ss(tmem + 256, dsm + ((kk * 2048) >> 4), dkm + ((kk * 2048) >> 4), idesc_dq, kk > 0, leader);
+          mma_ss(tmem + 384, dsm + ((kk * 2048) >> 4), dkm + ((kk * 2048) >> 4), idesc_dq, kk > 0, leader);
         tc_commit(&bar->dq_full, leader);
       };
-      auto issue_dV = [&](int ds, bool first) {   // dV += P^T dO
+      auto issue_dV = [&](int ds, bool first) {   // dV += P^T dO, P^T from the T columns
         const uint64_t dod = ddom_base + ds * kStageStep;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
-          mma_ts(tmem, tmem + 384 + (kk >> 1) * 32 + (kk & 1) * 8, dod + ((kk * 2048) >> 4), idesc_acc,
+          mma_ts(tmem, tmem + 256 + (kk >> 1) * 32 + (kk & 1) * 8, dod + ((kk * 2048) >> 4), idesc_acc,
                  (kk > 0 || !first) ? 1u : 0u, leader);
         tc_commit(&bar->do_empty[ds], leader);
       };
-      auto issue_dK = [&](int qs, bool first) {   // dK += dS^T Q
+      auto issue_dK = [&](int qs, bool first) {   // dK += dS^T Q, dS^T from shared memory
         const uint64_t qd = dqm_base + qs * kStageStep;
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-          mma_ts(tmem + D, tmem + 384 + (kk >> 1) * 32 + 16 + (kk & 1) * 8, qd + ((kk * 2048) >> 4), idesc_acc,
-                 (kk > 0 || !first) ? 1u : 0u, leader);
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint32_t c = ((kk >> 2) * kBoxBytes + (kk & 3) * 32) >> 4;
+          mma_ss(tmem + D, dsk + c, qd + ((kk * 2048) >> 4), idesc_acc, (kk > 0 || !first) ? 1u : 0u, leader);
+        }
         tc_commit(&bar->q_empty[qs], leader);
+        tc_commit(&bar->ds_free, leader);
       };
       bool ok = mbar_spin_warp(&bar->kv_full, 0, abort_flag) && mbar_spin_warp(&bar->q_full[0], 0, abort_flag) &&
                 mbar_spin_warp(&bar->do_full[0], 0, abort_flag);
@@ -1207,36 +1219,82 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         issue_dP(0);
       }
       for (int i = 0; ok && i < plan.total; ++i) {
-        const int qs = i & 1;
-        if (!mbar_spin_warp(&bar->pds_full, i & 1, abort_flag)) { ok = false; break; }
+        const bool more = i + 1 < plan.total;
+        if (i > 0) issue_dK((i - 1) & 1, i == 1);     // its dS was waited for before dQ(i-1)
+        if (!mbar_spin_warp(&bar->p_full, i & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        issue_dQ();                 // first: the compute warps read it out while dV and dK run
         issue_dV(i & 1, i == 0);
-        issue_dK(qs, i == 0);
-        if (i + 1 < plan.total) {
-          const int qn = (i + 1) & 1;
-          // S^T(i+1) reuses the columns of dQ(i): wait for its read-out; dP^T(i+1) follows dV(i), dK(i) in order
-          if (!mbar_spin_warp(&bar->t_free, i & 1, abort_flag) ||
-              !mbar_spin_warp(&bar->q_full[qn], ((i + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+        if (!mbar_spin_warp(&bar->ds_full, i & 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        issue_dQ();
+        if (more) {
+          const int sn = (i + 1) & 1;
+          const uint32_t phn = ((i + 1) >> 1) & 1;
+          // S^T(i+1) overwrites P^T(i): dV(i) precedes it in issue order
+          if (!mbar_spin_warp(&bar->q_full[sn], phn, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          issue_S(qn);
-          if (!mbar_spin_warp(&bar->do_full[(i + 1) & 1], ((i + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+          issue_S(sn);
+          // dP^T(i+1) overwrites dQ(i): wait for its read-out
+          if (!mbar_spin_warp(&bar->u_free, i & 1, abort_flag) ||
+              !mbar_spin_warp(&bar->do_full[sn], phn, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          issue_dP((i + 1) & 1);
+          issue_dP(sn);
         }
       }
-      if (ok) tc_commit(&bar->final_bar, leader);
+      if (ok) {
+        issue_dK((plan.total - 1) & 1, plan.total == 1);
+        tc_commit(&bar->final_bar, leader);
+      }
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------------ P^T / dS^T and epilogue
+    // ------------------------------------------------------------------ P^T, dS, dQ read-out and epilogue
     const int q = warp >> 2;                           // query-column quarter of this warp
     const int kr = (warp & 3) * 32 + lane;             // key inside the block == TMEM lane
     const int kp = k0 + kr;
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const uint32_t s_addr = tmem + lane_base + 256 + q * 32;
     const uint32_t dp_addr = tmem + lane_base + 384 + q * 32;
+    constexpr int kCols = D / 4;                       // dQ columns per quarter: 32 (D = 128) or 16 (D = 64)
+    const uint32_t dq_addr = tmem + lane_base + 384 + ((q * kCols) & ~31);
+    const int sub = (D == 64) ? (q & 1) * 16 : 0;
+    const int n_tiles = (a.Lq + kTileM - 1) / kTileM;
+    float* acc_prev = nullptr;                         // accumulator block of the previous item's query tile
     bool ok = true;
+    // dQ(i) read-out: lane == query row; each warp adds its 32 rows x D/4 columns as D/16 pieces of 512 bytes
+    auto drain = [&](int i_prev) -> bool {
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->dq_full, i_prev & 1, abort_flag))) return false;
+      tc_fence_after();
+      uint32_t v[32];
+      tmem_ld32(dq_addr, v);
+      tmem_ld_wait();
+      tc_fence_before();
+      mbar_arrive(&bar->u_free);       // the values are in registers: dP^T(i+1) may overwrite the columns
+      float* dst = acc_prev + warp * (8 * D) + lane * 4;
+#if defined(L2A_DIAG_ST)
+#pragma unroll
+      for (int c = 0; c < D / 16; ++c) {
+        const int k = sub + 4 * c;
+        asm volatile("st.global.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + c * 128), "f"(__uint_as_float(v[k])),
+                     "f"(__uint_as_float(v[k + 1])), "f"(__uint_as_float(v[k + 2])), "f"(__uint_as_float(v[k + 3]))
+                     : "memory");
+      }
+#elif !defined(L2A_DIAG_NO_RED)
+#ifdef L2A_DIAG_QUARTER
+      if (q == 0)
+#endif
+#pragma unroll
+      for (int c = 0; c < D / 16; ++c) {
+        const int k = sub + 4 * c;
+        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + c * 128), "f"(__uint_as_float(v[k])),
+                     "f"(__uint_as_float(v[k + 1])), "f"(__uint_as_float(v[k + 2])), "f"(__uint_as_float(v[k + 3]))
+                     : "memory");
+      }
+#else
+      if (v[0] == 0x12345678u && dst == nullptr) *dst = 0.f;
+#endif
+      return true;
+    };
     for (int i = 0; i < plan.total; ++i) {
       const int s = i & 1;
       // this item's row statistics go to registers before the scores are waited for
@@ -1251,6 +1309,11 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       }
       const bool masked = st_flags[q] != 0;
       const int item_glb = st_flags[4], item_row0 = st_flags[5], item_h = st_flags[6];
+      float* acc_cur = (item_glb ? a.dq_acc_glb : a.dq_acc_loc) +
+                       (((int64_t)b * a.Hq + item_h) * n_tiles + (item_row0 >> 7)) * (int64_t)(kTileM * D);
+      // the previous item's dQ leaves TMEM while this item's scores are still being computed
+      if (i > 0 && !drain(i - 1)) { ok = false; break; }
+      acc_prev = acc_cur;
       if (!__all_sync(0xffffffffu, mbar_wait(&bar->s_full, i & 1, abort_flag))) { ok = false; break; }
       tc_fence_after();
       uint32_t pp[16];
@@ -1268,17 +1331,16 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
             pp[e] = pack_bf16(fast_exp2(x.x), fast_exp2(x.y));
           }
         } else {
-          const int glb = st_flags[4], row0 = st_flags[5];
-          const int w_eff = glb ? 0x3fffffff : a.window;
-          const int n_rows = glb ? n_c : a.Lq;
+          const int w_eff = item_glb ? 0x3fffffff : a.window;
+          const int n_rows = item_glb ? n_c : a.Lq;
           const int32_t* qi = a.q_idx + (int64_t)b * a.Lq;
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
             int pos[2];
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
-              const int row = row0 + q * 32 + e + u;
-              pos[u] = row < n_rows ? (glb ? __ldg(&qi[row]) - a.vis_shift : row) + a.q_pos_offset : -1;
+              const int row = item_row0 + q * 32 + e + u;
+              pos[u] = row < n_rows ? (item_glb ? __ldg(&qi[row]) - a.vis_shift : row) + a.q_pos_offset : -1;
             }
             float p0 = fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, -st[e]));
             float p1 = fast_exp2(fmaf(__uint_as_float(sv[e + 1]), a.scale_log2, -st[e + 1]));
@@ -1288,6 +1350,10 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
           }
         }
       }
+      tmem_st16(s_addr, pp);     // P^T over the first half of this quarter's own S^T columns
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(&bar->p_full);
       // Delta of the same rows, again ahead of the wait; after this the statistics slot may be refilled
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
@@ -1311,11 +1377,9 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
           pd[e] = pack_bf16(ds.x, ds.y);
         }
       }
-      // P^T and dS^T go to this quarter's own 32 columns of the dP^T region (first 16 / next 16): A operands of dV
-      // and dK.  dS also goes to shared memory, [key][query] with the 128-byte swizzle of a TMA tile: read
-      // MN-major it is the A operand of dQ = dS K.
-      tmem_st16(dp_addr, pp);
-      tmem_st16(dp_addr + 16, pd);
+      // dS goes to shared memory, [key][query] with the 128-byte swizzle of a TMA tile (two boxes of 64 queries); the
+      // tile of the previous item must have been consumed by dQ(i-1) and dK(i-1)
+      if (i > 0 && !__all_sync(0xffffffffu, mbar_wait(&bar->ds_free, (i - 1) & 1, abort_flag))) { ok = false; break; }
       {
         const uint32_t row = smem_u32(sDS) + (q >> 1) * kBoxBytes + kr * 128;
         const int chunk0 = (q & 1) * 4;
@@ -1324,56 +1388,11 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((chunk0 + c) ^ (kr & 7)) << 4)),
                        "r"(pd[4 * c]), "r"(pd[4 * c + 1]), "r"(pd[4 * c + 2]), "r"(pd[4 * c + 3]) : "memory");
       }
-      tmem_st_wait();
       fence_async_smem();        // the MMA reads the tile through the async proxy
-      tc_fence_before();
-      mbar_arrive(&bar->pds_full);
-      // ---- dQ(i): read the 128 x D accumulator out of TMEM (lane = query row) and add it to the fp32 dQ buffer
-      if (!__all_sync(0xffffffffu, mbar_wait(&bar->dq_full, i & 1, abort_flag))) { ok = false; break; }
-      tc_fence_after();
-      {
-        constexpr int kCols = D / 4;     // 32 (D = 128) or 16 (D = 64) columns per quarter
-        uint32_t v[32];
-        tmem_ld32(tmem + lane_base + 256 + ((q * kCols) & ~31), v);
-        tmem_ld_wait();
-        tc_fence_before();
-        mbar_arrive(&bar->t_free);       // the values are in registers: S^T(i+1) may overwrite the columns
-        // Reduction into the fp32 dQ buffer.  Lane == query row would make every red instruction touch 32 rows with
-        // 16 bytes each (half a sector per row): instead each warp transposes its 32 x 16-column pieces through
-        // shared memory, so that one instruction covers 8 rows with 64 contiguous bytes each.  The scratch is the
-        // 2 KB of the dS tile that this warp itself wrote (the dQ MMA that read them has completed, and nobody else
-        // writes them), addressed with the same swizzle, which keeps both directions free of bank conflicts.
-        const int r = item_row0 + kr;    // query row of this thread (lane == row inside the tile)
-        const int n_rows = item_glb ? n_c : a.Lq;
-        const int t_mine = r < n_rows ? (item_glb ? __ldg(&a.q_idx[(int64_t)b * a.Lq + r]) : r) : -1;
-        const uint32_t scratch = smem_u32(sDS) + (q >> 1) * kBoxBytes + (kr - lane) * 128;
-        const int chunk0 = (q & 1) * 4;
-        const int sub = (D == 64) ? (q & 1) * 16 : 0;
-        float* acc_head = a.dq_acc + (int64_t)b * a.Lq * a.Hq * D + (int64_t)item_h * D + q * kCols;
-#pragma unroll
-        for (int half = 0; half < kCols / 16; ++half) {
-          __syncwarp();
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const int k = sub + half * 16 + 4 * c;
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(scratch + lane * 128 + (((chunk0 + c) ^ (lane & 7)) << 4)),
-                         "r"(v[k]), "r"(v[k + 1]), "r"(v[k + 2]), "r"(v[k + 3]) : "memory");
-          }
-          __syncwarp();
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int R = j * 8 + (lane >> 2), cl = lane & 3;
-            const float4 x = lds128(scratch + R * 128 + (((chunk0 + cl) ^ (R & 7)) << 4));
-            const int t = __shfl_sync(0xffffffffu, t_mine, R);
-            if (t >= 0) {
-              float* dst = acc_head + (int64_t)t * a.Hq * D + half * 16 + cl * 4;
-              asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(x.x * a.scale),
-                           "f"(x.y * a.scale), "f"(x.z * a.scale), "f"(x.w * a.scale) : "memory");
-            }
-          }
-        }
-      }
+      tc_fence_before();         // orders the dP^T read above before the dQ MMA that overwrites those columns
+      mbar_arrive(&bar->ds_full);
     }
+    if (ok && plan.total > 0 && !drain(plan.total - 1)) ok = false;
     // epilogue: quarters 0,1 store the two column halves of dV, quarters 2,3 those of dK
     if (ok && __all_sync(0xffffffffu, mbar_wait(&bar->final_bar, 0, abort_flag))) {
       tc_fence_after();
@@ -1413,18 +1432,67 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
   if (warp == 17) tmem_dealloc(tmem, 512);
 }
 
+// Zeroes the fp32 dQ accumulators: every row tile of the local one, the compact tiles below n_routed of the global one.
+__global__ void __launch_bounds__(256) dq_zero_kernel(float* __restrict__ acc_loc, float* __restrict__ acc_glb,
+                                                      const int32_t* __restrict__ n_routed, int B, int Hq, int n_tiles,
+                                                      int tile_floats) {
+  const int per = B * Hq * n_tiles;
+  for (int item = blockIdx.x; item < 2 * per; item += gridDim.x) {
+    const int which = item >= per, rem = which ? item - per : item;
+    float* base = which ? acc_glb : acc_loc;
+    if (base == nullptr) continue;
+    if (which && (rem % n_tiles) * kTileM >= n_routed[rem / (n_tiles * Hq)]) continue;
+    float4* p = reinterpret_cast<float4*>(base + (int64_t)rem * tile_floats);
+    for (int k = threadIdx.x; k < tile_floats / 4; k += blockDim.x) p[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+}
 
-// fp32 dQ accumulator -> bf16 dQ (the accumulated values already carry the soft-max scale)
-__global__ void __launch_bounds__(256) dq_convert_kernel(const float* __restrict__ acc, bf16* __restrict__ dQ, int B, int L,
-                                                         int row_elems, int64_t bs, int64_t ts) {
-  const int64_t chunks_per_row = row_elems / 8;
-  const int64_t n = (int64_t)B * L * chunks_per_row;
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
-    const int64_t row = i / chunks_per_row, c = i % chunks_per_row;
-    const float4 x = __ldg(reinterpret_cast<const float4*>(acc) + 2 * i), y = __ldg(reinterpret_cast<const float4*>(acc) + 2 * i + 1);
-    const int64_t b = row / L, t = row % L;
-    *reinterpret_cast<uint4*>(dQ + b * bs + t * ts + c * 8) =
-        make_uint4(pack_bf16(x.x, x.y), pack_bf16(x.z, x.w), pack_bf16(y.x, y.y), pack_bf16(y.z, y.w));
+// fp32 dQ accumulators -> bf16 dQ: dQ_t = scale * (local(t) + d_t * global(prefix[t])).  One CTA per (batch, row tile,
+// head); the accumulator blocks are read in their own order (512 contiguous bytes per warp), the bf16 rows leave
+// through shared memory as whole 2 D-byte segments.
+template <int D>
+__global__ void __launch_bounds__(256) dq_merge_kernel(const float* __restrict__ acc_loc, const float* __restrict__ acc_glb,
+                                                       const uint8_t* __restrict__ d_mask,
+                                                       const int32_t* __restrict__ prefix, bf16* __restrict__ dQ, int B,
+                                                       int L, int Hq, float scale, int64_t bs, int64_t ts) {
+  constexpr int kChunks = D / 8;             // 16-byte chunks per bf16 row
+  constexpr int kRowBytes = D * 2 + 16;      // padded: conflict-free 16-byte accesses down a column
+  __shared__ __align__(16) uint8_t tile_s[kTileM * kRowBytes];
+  const int n_tiles = (L + kTileM - 1) / kTileM;
+  const int h = blockIdx.x % Hq;
+  const int tile = (blockIdx.x / Hq) % n_tiles;
+  const int b = blockIdx.x / (Hq * n_tiles);
+  const int64_t tile_floats = kTileM * D;
+  const float* loc = acc_loc ? acc_loc + (((int64_t)b * Hq + h) * n_tiles + tile) * tile_floats : nullptr;
+  for (int idx = threadIdx.x; idx < kTileM * kChunks; idx += blockDim.x) {
+    const int lane = idx & 31, rq = (idx >> 5) & 3, k = idx >> 7;
+    const int r = rq * 32 + lane, t = tile * kTileM + r;
+    if (t >= L) continue;
+    const int d0 = 8 * k, q = d0 / (D / 4), c = (d0 % (D / 4)) / 4;
+    float4 x = make_float4(0.f, 0.f, 0.f, 0.f), y = x;
+    if (loc) {
+      const float4* p = reinterpret_cast<const float4*>(loc + (q * 4 + rq) * (8 * D) + c * 128 + lane * 4);
+      x = __ldg(p); y = __ldg(p + 32);
+    }
+    if (acc_glb && d_mask[(int64_t)b * L + t]) {
+      const int cr = prefix[(int64_t)b * (L + 1) + t];
+      const float4* p = reinterpret_cast<const float4*>(
+          acc_glb + (((int64_t)b * Hq + h) * n_tiles + (cr >> 7)) * tile_floats + (q * 4 + ((cr & 127) >> 5)) * (8 * D) +
+          c * 128 + (cr & 31) * 4);
+      const float4 gx = __ldg(p), gy = __ldg(p + 32);
+      x.x += gx.x; x.y += gx.y; x.z += gx.z; x.w += gx.w;
+      y.x += gy.x; y.y += gy.y; y.z += gy.z; y.w += gy.w;
+    }
+    *reinterpret_cast<uint4*>(tile_s + r * kRowBytes + k * 16) =
+        make_uint4(pack_bf16(x.x * scale, x.y * scale), pack_bf16(x.z * scale, x.w * scale),
+                   pack_bf16(y.x * scale, y.y * scale), pack_bf16(y.z * scale, y.w * scale));
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < kTileM * kChunks; idx += blockDim.x) {
+    const int r = idx / kChunks, k = idx % kChunks, t = tile * kTileM + r;
+    if (t < L)
+      *reinterpret_cast<uint4*>(dQ + b * bs + t * ts + (int64_t)h * D + k * 8) =
+          *reinterpret_cast<const uint4*>(tile_s + r * kRowBytes + k * 16);
   }
 }
 
@@ -1485,33 +1553,36 @@ int dkv_split_block(int n_kblocks) { return n_kblocks >= 8 ? (3 * n_kblocks) / 4
 template <int D>
 cudaError_t launch_bwd_fused(const BwdArgs& base, const CUtensorMap& mapQ, const CUtensorMap& mapDO,
                              const CUtensorMap& mapQc, const CUtensorMap& mapDOc, const CUtensorMap& mapK,
-                             const CUtensorMap& mapV, cudaStream_t s) {
+                             const CUtensorMap& mapV, const uint8_t* d_mask, cudaStream_t s) {
   cudaError_t e = cudaFuncSetAttribute(bwd_fused_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        FusedSmem<D>::kTotal);
   if (e != cudaSuccess) return e;
-  const size_t acc = (size_t)base.B * base.Lq * base.Hq * D * sizeof(float);
-  e = cudaMemsetAsync(base.dq_acc, 0, acc, s);
-  if (e != cudaSuccess) return e;
-  phase_events().mark(s);     // (no local dQ launch in this mode)
-  phase_events().mark(s);     // (no global dQ launch)
+  int device = 0, sms = 148;
+  if (cudaGetDevice(&device) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+  const int n_tiles = (base.Lq + kTileM - 1) / kTileM;
+  dq_zero_kernel<<<sms * 8, 256, 0, s>>>(base.dq_acc_loc, base.dq_acc_glb, base.n_routed, base.B, base.Hq, n_tiles,
+                                         kTileM * D);
+  phase_events().mark(s);
   BwdArgs a = base;
   const int n_kblocks = (base.Lk + kTileN - 1) / kTileN;
   a.kb_begin = 0;
   a.kb_count = n_kblocks;
   bwd_fused_kernel<D><<<(unsigned)n_kblocks * base.B * base.Hkv, kDkvThreads, FusedSmem<D>::kTotal, s>>>(
       mapQ, mapDO, mapQc, mapDOc, mapK, mapV, a);
-  int device = 0, sms = 148;
-  if (cudaGetDevice(&device) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
-  dq_convert_kernel<<<sms * 8, 256, 0, s>>>(base.dq_acc, base.dQ, base.B, base.Lq, base.Hq * D, base.dq_st.b,
-                                            base.dq_st.t);
+  phase_events().mark(s);
+  dq_merge_kernel<D><<<(unsigned)(n_tiles * base.B * base.Hq), 256, 0, s>>>(
+      base.dq_acc_loc, base.dq_acc_glb, d_mask, base.prefix, base.dQ, base.B, base.Lq, base.Hq, base.scale,
+      base.dq_st.b, base.dq_st.t);
   phase_events().mark(s);
   return cudaGetLastError();
 }
 
+// one fp32 dQ accumulator: whole 128-row tiles
 size_t acc_bytes(const l2a_params* p) {
-  return (p->flags & L2A_FLAG_FUSED_DQ) ? align_up((size_t)p->B * p->Lq * p->Hq * p->D * sizeof(float), 256) : 0;
+  return (p->flags & L2A_FLAG_FUSED_DQ)
+             ? align_up((size_t)p->B * p->Hq * ceil_div(p->Lq, kTileM) * kTileM * p->D * sizeof(float), 256) : 0;
 }
-size_t bwd_ws_size(const l2a_params* p) { return kWsHeaderBytes + 2 * rows_bytes(p) + 3 * stat_bytes(p) + acc_bytes(p); }
+size_t bwd_ws_size(const l2a_params* p) { return kWsHeaderBytes + 2 * rows_bytes(p) + 3 * stat_bytes(p) + 2 * acc_bytes(p); }
 
 }  // namespace l2a
 
@@ -1550,7 +1621,6 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   if (!skip_global && (!d_mask || !q_idx || !n_routed || !prefix || !A_c || !lse_glb)) return L2A_ERR_INVALID_ARG;
   if (!skip_local && (!S_save || !lse_loc)) return L2A_ERR_INVALID_ARG;
   if (force_all && (skip_local || skip_global)) return L2A_ERR_INVALID_ARG;
-  if ((p->flags & L2A_FLAG_FUSED_DQ) && (skip_local || skip_global || force_all)) return L2A_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(dO) || !aligned16(S_save) || !aligned16(A_c) ||
       !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
     return L2A_ERR_INVALID_ARG;
@@ -1563,12 +1633,13 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   float* delta_loc = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p));
   float* delta_glb = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + stat_bytes(p));
   float* lse_c = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + 2 * stat_bytes(p));
-  float* dq_acc = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + 3 * stat_bytes(p));
+  float* dq_acc_loc = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + 3 * stat_bytes(p));
+  float* dq_acc_glb = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + 3 * stat_bytes(p) + acc_bytes(p));
   const bool fused = p->flags & L2A_FLAG_FUSED_DQ;
   // Shared-window backward: the window's share of a routed row's global gradient rides on the local items (see
   // bwd_delta_kernel).  Needs the same gradient for both outputs; the flag permits it, other modes just ignore it.
   const bool share = (p->flags & L2A_FLAG_SHARED_WINDOW) && dS_loc == dO && !skip_local && !skip_global &&
-                     !force_all && !fused;
+                     !force_all;
 
   CUtensorMap mapQ, mapDO, mapQc, mapDOc, mapK, mapV;
   const RowStrides qs = resolve_strides(p->q_stride, p->Lq, p->Hq * p->D);
@@ -1631,12 +1702,13 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   a.vis_shift = share ? (p->window < (1 << 30) ? p->window : (1 << 30)) + 1 : 0; a.delta_loc = delta_loc; a.delta_glb = delta_glb;
   a.dQ = static_cast<bf16*>(dQ); a.dK = static_cast<bf16*>(dK); a.dV = static_cast<bf16*>(dV);
   a.dq_st = qs; a.dk_st = ks; a.dv_st = vs;
-  a.dq_acc = fused ? dq_acc : nullptr;
+  a.dq_acc_loc = fused && !skip_local ? dq_acc_loc : nullptr;
+  a.dq_acc_glb = fused && !skip_global ? dq_acc_glb : nullptr;
   a.status = reinterpret_cast<int*>(ws);
   cudaError_t e;
   if (fused)
-    e = p->D == 128 ? launch_bwd_fused<128>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, s)
-                    : launch_bwd_fused<64>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, s);
+    e = p->D == 128 ? launch_bwd_fused<128>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, skip_global ? nullptr : d_mask, s)
+                    : launch_bwd_fused<64>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, skip_global ? nullptr : d_mask, s);
   else
     e = p->D == 128 ? launch_bwd_kernels<128>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, s)
                     : launch_bwd_kernels<64>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, s);
