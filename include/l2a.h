@@ -10,8 +10,11 @@
  *
  * Conventions shared by every call
  *   - Every pointer is a DEVICE pointer unless its comment says "host".  The caller owns all
- *     buffers, including the workspaces; the library allocates no device memory, keeps no state
- *     between calls, and never synchronises the stream (only l2a_workspace_status does).
+ *     buffers, including the workspaces; the library allocates no device memory and never
+ *     synchronises the stream (only l2a_workspace_status and l2a_step_host do).  State kept between
+ *     calls: per-device facts looked up once (SM count, kernel attributes); the fixed device array
+ *     and its cached address of l2a_route_compact_static; the per-thread helper streams and events of
+ *     l2a_step_host; the one-shot event registration of l2a_profile_next_call.
  *   - Tensors are contiguous bf16:  Q, O, dO, dQ, S_save, A_c : [B, Lq, Hq, D]
  *                                   K, V, dK, dV              : [B, Lk, Hkv, D]
  *     D contiguous, base pointers 16-byte aligned.  D is 64 or 128.  Hq % Hkv == 0 (GQA: query
@@ -56,35 +59,28 @@ typedef enum {
                                   /* the routed rows' global attention runs and is added into O.       */
                                   /* Lets the caller compute the router decision from S in between     */
                                   /* (Eq. 2 -> 3 -> 4 -> 5 in the order the layer defines them).       */
-#define L2A_FLAG_FUSED_DQ 32u      /* backward, experimental: five GEMMs per tile pair instead of seven -- dQ is  */
-                                  /* produced inside the dK/dV kernel and summed in an fp32 buffer with atomic   */
-                                  /* reductions, then rounded to bf16.  Same tolerance as the default path; dK   */
-                                  /* and dV are bit-identical to it, dQ is not bit-reproducible from run to run. */
-                                  /* The backward workspace grows by B * Lq * Hq * D * 4 bytes (pass the same    */
-                                  /* flags to l2a_workspace_bytes).  Not combined with L2A_FLAG_SKIP_LOCAL,        */
-                                  /* L2A_FLAG_SKIP_GLOBAL or L2A_FLAG_FORCE_ALL_GLOBAL (invalid argument).  On   */
-                                  /* B200 the reductions' L2 traffic makes it slower than the default at long    */
-                                  /* sequences, so it is off by default.                                         */
-#define L2A_FLAG_SHARED_WINDOW 64u /* forward, shared projections (the "L2A-shared" variant of the paper's ablations:  */
-                                  /* one Q/K/V set feeds both modules, which is what this interface always passes):  */
-                                  /* a routed row's scores against the keys inside its window are the ones the Local */
-                                  /* pass has already reduced, so Global Attention covers only the keys BEFORE the   */
-                                  /* window (positions 0 .. t-W-1) and is merged with the local result,              */
-                                  /*   a_t = (e^{lse_out} o_out + e^{lse_loc} s_t) / (e^{lse_out} + e^{lse_loc}),     */
-                                  /* which is the softmax over the whole prefix.  Saves rho * W pairs per head.      */
-                                  /* s_t enters as the stored bf16 value (one extra rounding of relative size 2^-9   */
-                                  /* on the window's share of a_t; same tolerance).  Needs lse_loc (also without     */
-                                  /* L2A_FLAG_SAVE_FOR_BWD); not combined with L2A_FLAG_SKIP_LOCAL or                */
-                                  /* L2A_FLAG_FORCE_ALL_GLOBAL; ignored by a call that has L2A_FLAG_SKIP_GLOBAL.     */
-                                  /* A_c, lse_glb and O mean the same as without it, so the backward does not depend */
-                                  /* on how the forward was run.  Passed to l2a_backward, the flag allows the same    */
-                                  /* sharing there: inside the window P_glb = beta_t P_loc with                       */
-                                  /* beta_t = exp(lse_loc - lse_glb) and dP = dO V^T is common to both modules, so    */
-                                  /* the local tile pairs carry both gradients (row statistics                        */
-                                  /* lse' = lse_loc - log(1 + beta), Delta' = (Delta_loc + beta Delta_glb)/(1 + beta)) */
-                                  /* and the global ones stop before the window.  Used only when both outputs get the */
-                                  /* same gradient (not l2a_backward_split with its own dS_loc) and without           */
-                                  /* L2A_FLAG_FUSED_DQ / FORCE_ALL_GLOBAL / SKIP_*; otherwise ignored.                */
+#define L2A_FLAG_SHARED_WINDOW 64u /* Only for callers that really pass ONE Q/K/V set to both modules (the benchmark     */
+                                  /* configurations do; in the paper's layer Global Attention reads the local output   */
+                                  /* s_t through its own projections, so its Q/K/V differ from the local module's and   */
+                                  /* the flag does not apply).  With one set, a routed row's scores against the keys    */
+                                  /* inside its window are the ones the Local pass has already reduced, so Global       */
+                                  /* Attention covers only the keys BEFORE the window (positions 0 .. t-W-1) and is     */
+                                  /* merged with the local result,                                                      */
+                                  /*   a_t = (e^{lse_out} o_out + e^{lse_loc} s_t) / (e^{lse_out} + e^{lse_loc}),       */
+                                  /* which is the softmax over the whole prefix.  Saves rho * W pairs per head.         */
+                                  /* s_t enters as the stored bf16 value (one extra rounding of relative size 2^-9      */
+                                  /* on the window's share of a_t; same tolerance).  Needs lse_loc (also without        */
+                                  /* L2A_FLAG_SAVE_FOR_BWD); not combined with L2A_FLAG_SKIP_LOCAL or                   */
+                                  /* L2A_FLAG_FORCE_ALL_GLOBAL; ignored by a call that has L2A_FLAG_SKIP_GLOBAL.        */
+                                  /* A_c, lse_glb and O mean the same as without it, so the backward does not depend    */
+                                  /* on how the forward was run.  Passed to l2a_backward, the flag allows the same       */
+                                  /* sharing there: inside the window P_glb = beta_t P_loc with                          */
+                                  /* beta_t = exp(lse_loc - lse_glb) and dP = dO V^T is common to both modules, so       */
+                                  /* the local tile pairs carry both gradients (row statistics                           */
+                                  /* lse' = lse_loc - log(1 + beta), Delta' = (Delta_loc + beta Delta_glb)/(1 + beta))   */
+                                  /* and the global ones stop before the window.  Used only when both outputs get the    */
+                                  /* same gradient (not l2a_backward_split with its own dS_loc) and without              */
+                                  /* FORCE_ALL_GLOBAL / SKIP_*; otherwise ignored.                                       */
 #define L2A_FLAG_FORCE_ALL_GLOBAL 8u /* training iterations that invoke Global Attention for every    */
                                   /* token regardless of d_t (Section 3.3: done with a small       */
                                   /* probability so that masked tokens' routers get a gradient).   */
@@ -142,17 +138,6 @@ l2a_status l2a_workspace_bytes(const l2a_params* p, size_t* route_ws_bytes, size
 l2a_status l2a_selftest_wait_timeout(void* ws, unsigned limit_us, void* stream);
 
 /*
- * Self-test of the bounded device-side wait (the mechanism behind L2A_ERR_DEVICE_TIMEOUT).  Launches one small
- * kernel in which a warp waits, with a limit of `limit_us` microseconds (1 .. 1000000), for an mbarrier arrival that
- * never comes, while the other warps wait for something else: the first wait runs out, raises the CTA's abort flag,
- * the other warps leave their waits on seeing it, and the CTA writes the status word of workspace `ws` (any 256-byte
- * aligned device buffer of at least 256 bytes) -- the path every kernel of this library takes when a wait runs
- * out.  Afterwards l2a_workspace_status(ws) returns L2A_ERR_DEVICE_TIMEOUT and the context stays usable.  Nothing
- * traps, faults or spins without a limit.  Returns L2A_ERR_INVALID_ARG for a limit outside the range.
- */
-l2a_status l2a_selftest_wait_timeout(void* ws, unsigned limit_us, void* stream);
-
-/*
  * Reads the status word the kernels of earlier calls left in workspace `ws` (any of the three).
  * Synchronises `stream`.  Returns L2A_OK, or L2A_ERR_DEVICE_TIMEOUT if a bounded device-side wait
  * ran out in some kernel that used this workspace since it was last used by a successful call.
@@ -160,8 +145,8 @@ l2a_status l2a_selftest_wait_timeout(void* ws, unsigned limit_us, void* stream);
 l2a_status l2a_workspace_status(const void* ws, void* stream);
 
 /*
- * Routing decision and query compaction (Eq. 3; Section 3.2 "consolidated into a compact,
- * contiguous buffer ... original sequence positions recorded"; Algorithm 1, step 1).
+ * Routing decision and query compaction (Eq. 3; Section 3.2: the routed queries are gathered into one
+ * dense buffer and the sequence position of each is kept; Algorithm 1, step 1).
  *
  *   router      in : [B, Lq] uint8 mask, fp32 logits or bf16 logits, per router_kind.  For logits the decision
  *                    is taken on the logit in fp32, d = (z >= logit_threshold); threshold 0 is
@@ -242,13 +227,16 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
  *   dO          in : bf16 [B, Lq, Hq, D], gradient of the loss w.r.t. O.
  *   S_save, A_c, lse_loc, lse_glb
  *               in : as written by l2a_forward with L2A_FLAG_SAVE_FOR_BWD.
- *   dQ          out: bf16 [B, Lq, Hq, D].
- *   dK, dV      out: bf16 [B, Lk, Hkv, D].
+ *   dQ          out: bf16 [B, Lq, Hq, D].  The contributions of the key blocks meet in fp32 accumulators in the
+ *                    workspace through atomic additions, in no fixed order: two runs agree to fp32 rounding of
+ *                    the sums (and almost always bit for bit after the bf16 rounding), not by construction.
+ *   dK, dV      out: bf16 [B, Lk, Hkv, D].  Accumulated on chip in a fixed order: bit-reproducible.
  *   dgate       out: optional fp32 [B, Lq] (may be NULL): sum over heads of dO_t . a_t -- the
  *                    loss-dependent term of the straight-through router gradient (Eq. 7) -- for
  *                    the rows whose global output was computed: routed rows (0 elsewhere), or
  *                    every row with L2A_FLAG_FORCE_ALL_GLOBAL.
- *   bwd_ws         : workspace of at least bwd_ws_bytes.
+ *   bwd_ws         : workspace of at least bwd_ws_bytes (compact copies of Q and dO, row statistics, and two fp32
+ *                    dQ accumulators of B * Hq * ceil(Lq / 128) * 128 * D floats each).
  */
 l2a_status l2a_backward(const l2a_params* p, const void* Q, const void* K, const void* V,
                         const uint8_t* d_mask, const int32_t* q_idx, const int32_t* n_routed,
@@ -402,11 +390,12 @@ l2a_status l2a_route_compact_static(const l2a_params* p, const void* router, int
  * k-th phase boundary and then clears the registration.  Phase boundaries:
  *   l2a_forward : 0 start | 1 after the query gather | 2 after the local kernel | 3 after the
  *                 global kernel
- *   l2a_backward: 0 start | 1 after the gathers | 2 after the Delta kernel | 3 after the local dQ
- *                 kernel | 4 after the global dQ kernel (dQ is final) | 5 after the dK/dV kernel.
- *                 With 7 events the dK/dV kernel runs as two launches (key rows below and from
- *                 128 * floor(3 * ceil(Lk / 128) / 4), when Lk >= 1024): 5 after the first, 6 after the second
- * This is the only per-thread state the library keeps.
+ *   l2a_backward: 0 start | 1 after the gathers | 2 after the Delta kernel and the clearing of the dQ accumulators |
+ *                 3 after the five-GEMM kernel | 4 after the dQ merge (everything final).
+ *                 With 7 events the kernel runs as two launches over key-block ranges (keys below and from
+ *                 128 * floor(3 * ceil(Lk / 128) / 4), when Lk >= 1024), each followed by the merge of the dQ rows
+ *                 it completes: 3 / 4 after the first kernel / merge (dK, dV of the first range's keys and dQ of the
+ *                 rows that see only those keys are final), 5 / 6 after the second.
  */
 l2a_status l2a_profile_next_call(void* const* events, int n_events);
 

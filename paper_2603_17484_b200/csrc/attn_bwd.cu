@@ -9,15 +9,14 @@
 //
 // Kernels
 //   bwd_delta_kernel : Delta_loc (all rows), Delta_glb (compact rows), optional dgate.  HBM bound.
-//   bwd_dkv_kernel   : key/value-stationary.  One CTA owns a block of 128 keys of one KV head and
-//                      walks every query tile that can see it -- local band tiles of the G query heads,
-//                      then the compact routed tiles from the first one at or after the block -- and
-//                      accumulates dK, dV in TMEM (no atomics, one bf16 store).  The scores are built
-//                      transposed (keys on TMEM lanes) so P^T and dS^T feed the second pair of MMAs
-//                      straight from TMEM.  Each tile is processed as two 64-column halves so that the
-//                      MMAs of one half overlap the exponentials of the other.
-//   bwd_dq_kernel    : query-stationary, the forward's iteration space; local mode writes dQ, global mode
-//                      adds the routed rows' global term at their positions.
+//   dq_zero_kernel   : clears the fp32 dQ accumulators.
+//   bwd_kernel       : key/value-stationary, five GEMMs per (query tile, key block) pair.  One CTA owns a block of
+//                      128 keys of one KV head and walks every query tile that can see it -- local band tiles of
+//                      the G query heads, then the compact routed tiles from the first one at or after the block.
+//                      dK, dV accumulate in TMEM (no atomics, one bf16 store); the scores are built transposed (keys
+//                      on TMEM lanes) so that P^T feeds dV straight from TMEM; dQ(i) = dS(i) K is a fresh tile per
+//                      item that the compute warps add into fp32 accumulators in global memory.
+//   dq_merge_kernel  : dQ = scale * (local accumulator + routed rows' global accumulator), rounded to bf16 once.
 #include "l2a_common.cuh"
 #include "sm100_prims.cuh"
 
@@ -27,29 +26,6 @@ namespace {
 
 constexpr int kBoxBytes = 128 * 128;
 constexpr float kLog2e = 1.4426950408889634f;
-
-// Optional per-role clock tracing of one CTA of the dK/dV kernel (development builds only: -DL2A_TRACE=<block>).
-#ifndef L2A_TRACE_WARP
-#define L2A_TRACE_WARP 0   // the compute warp whose phases are recorded
-#endif
-#ifdef L2A_TRACE
-__device__ long long g_trace[4][8192];
-#define L2A_TRACE_POINT(role, idx)                                                              \
-  do {                                                                                          \
-    if (blockIdx.x == (L2A_TRACE) && (idx) < 8192) g_trace[role][idx] = clock64();              \
-  } while (0)
-#else
-#define L2A_TRACE_POINT(role, idx)
-#endif
-// same for one CTA of the dQ kernel (-DL2A_TRACE=<any> -DL2A_TRACE_DQ=<block>), roles 0 (MMA warp) and 1 (compute warp)
-#if defined(L2A_TRACE) && defined(L2A_TRACE_DQ)
-#define L2A_TRACE_DQ_POINT(role, idx)                                                           \
-  do {                                                                                          \
-    if (blockIdx.x == (L2A_TRACE_DQ) && (idx) < 8192) g_trace[role][idx] = clock64();           \
-  } while (0)
-#else
-#define L2A_TRACE_DQ_POINT(role, idx)
-#endif
 
 // ------------------------------------------------------------------------------------------------
 // Delta / dgate preprocess.  The grid is one resident wave; the warps take the tokens round-robin, so that at any
@@ -179,11 +155,10 @@ struct BwdArgs {
   int B, Lq, Lk, Hq, Hkv, D;
   int window, q_pos_offset;
   float scale, scale_log2;
-  int global_mode;  // dq kernel only
   int skip_local, skip_global;   // gradients of one module only (the other module has its own Q/K/V)
-  int kb_begin, kb_count;        // dK/dV kernel: key blocks [kb_begin, kb_begin + kb_count) of every KV head
+  int kb_begin, kb_count;        // key blocks [kb_begin, kb_begin + kb_count) of every KV head
   RowStrides dq_st, dk_st, dv_st;   // strides of the gradient tensors in elements
-  float* dq_acc_loc;             // five-GEMM mode: fp32 dQ accumulators (layout: see bwd_fused_kernel), by row tile
+  float* dq_acc_loc;             // fp32 dQ accumulators (layout: see bwd_kernel), by row tile
   float* dq_acc_glb;             //                 and by compact tile; NULL when that module is skipped
   int vis_shift;                 // global items see the keys 0 .. pos - vis_shift: 0, or W + 1 when the window's share of
                                  // the global gradient is carried by the local items (shared-window backward)
@@ -201,354 +176,16 @@ struct BwdArgs {
 };
 
 // ================================================================================================
-// Thread roles of the two tensor-core kernels below:
-//   warps 0-15 : compute.  Warp w owns TMEM lanes 32*(w%4)..+31 (its thread's query row / key) and the
+// Thread roles of the tensor-core kernel below:
+//   warps 0-15 : compute.  Warp w owns TMEM lanes 32*(w%4)..+31 (its thread's key, or query row of dQ) and the
 //                32 score columns of quarter w/4, so that 16 warps hide each other's TMEM and MUFU latency.
 //   warp 16    : TMA producer          warp 17 : tcgen05 MMA issuer, TMEM owner
-//   warp 18    : (dK/dV kernel only) stages the row statistics of each query tile
+//   warp 18    : stages the row statistics of each query tile
 constexpr int kComputeWarps = 16;
-constexpr int kDqThreads = (kComputeWarps + 3) * 32;    // 608: + TMA producer + two MMA issuers
 constexpr int kDkvThreads = (kComputeWarps + 3) * 32;   // 608
 
 __device__ __forceinline__ float bf16lo_to_f32(uint32_t packed) { return __uint_as_float(packed << 16); }
 __device__ __forceinline__ float bf16hi_to_f32(uint32_t packed) { return __uint_as_float(packed & 0xffff0000u); }
-
-// ================================================================================================
-// dQ kernel: one 128-row query tile per CTA; Q and dO stay in shared memory, K/V blocks stream.
-//   TMEM: dQ [0,D) | S [128,256) | dP (two buffers) [256,384) [384,512).
-//   The scores go to registers at once (barrier s_taken), so one S buffer is enough; dS (bf16) is written over the
-//   dP buffer of its key block (quarter q puts its 16 packed columns at the start of its own 32 columns) and is the
-//   A operand of dQ += dS K.  With two dP buffers nothing the compute warps wait for depends on an MMA that waits
-//   for them: S(j+1) and dP(j+1) are produced a block ahead, dQ(j) only consumes.
-//   Two warps issue the MMAs, on different scheduler partitions: warp 17 the dQ stream, warp 18 the S / dP stream.
-//   A single issuer leaves a gap between consecutive MMAs (its next instruction is prepared only after the
-//   previous one was accepted: measured 105-125 clk per MMA inside this kernel against 64 in a lean stream); with
-//   two independent streams one MMA is always waiting at the pipe (74 clk per MMA measured).
-template <int D>
-struct DqSmem {
-  static constexpr int kTileBytes = 128 * D * 2;
-  static constexpr int kKStages = 3;
-  static constexpr int kVStages = 2;
-  static constexpr int kQOff = 0;
-  static constexpr int kDoOff = kTileBytes;
-  static constexpr int kKOff = 2 * kTileBytes;
-  static constexpr int kVOff = kKOff + kKStages * kTileBytes;
-  static constexpr int kBarOff = kVOff + kVStages * kTileBytes;
-  static constexpr int kTotal = kBarOff + 256 + 1024;
-};
-struct DqBarriers {
-  uint64_t q_full;
-  uint64_t k_full[3], k_empty[3], v_full[2], v_empty[2];
-  uint64_t s_full, s_taken, dp_full[2], ds_full[2], dq_done[2], final_bar;
-  uint32_t tmem_base;
-  int abort_flag;
-};
-
-template <int D>
-__global__ void __launch_bounds__(kDqThreads, 1)
-bwd_dq_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapDO,
-              const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, const BwdArgs a) {
-  using SM = DqSmem<D>;
-  constexpr int kKSteps = D / 16;
-  const int n_tiles = (a.Lq + kTileM - 1) / kTileM;
-  const int h = blockIdx.x % a.Hq;
-  const int rest = blockIdx.x / a.Hq;
-  const int b = rest % a.B;
-  const int ti = n_tiles - 1 - rest / a.B;
-  const int g = h / (a.Hq / a.Hkv);
-  const int n_rows = a.global_mode ? a.n_routed[b] : a.Lq;
-  const int row0 = ti * kTileM;
-  if (row0 >= n_rows) return;
-  const int32_t* q_idx_b = a.q_idx + (int64_t)b * a.Lq;
-  const int w_eff = a.global_mode ? 0x3fffffff : a.window;
-  const int last = min(row0 + kTileM - 1, n_rows - 1);
-  const int vis_shift = a.global_mode ? a.vis_shift : 0;
-  const int min_pos = (a.global_mode ? q_idx_b[row0] : row0) + a.q_pos_offset - vis_shift;   // last visible key
-  const int max_pos = (a.global_mode ? q_idx_b[last] : last) + a.q_pos_offset - vis_shift;
-  if (max_pos < 0) return;    // (shared-window backward) no row of the tile has a key before its window
-  const int jlo = (min_pos - w_eff > 0) ? (min_pos - w_eff) / kTileN : 0;
-  const int jhi = max_pos / kTileN;
-  const int n_blocks = jhi - jlo + 1;
-
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sQ = smem + SM::kQOff;
-  uint8_t* sDO = smem + SM::kDoOff;
-  uint8_t* sK = smem + SM::kKOff;
-  uint8_t* sV = smem + SM::kVOff;
-  DqBarriers* bar = reinterpret_cast<DqBarriers*>(smem + SM::kBarOff);
-  volatile int* abort_flag = &bar->abort_flag;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-
-  if (tid == 0) {
-    mbar_init(&bar->q_full, 1);
-    for (int s = 0; s < 3; ++s) { mbar_init(&bar->k_full[s], 1); mbar_init(&bar->k_empty[s], 1); }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&bar->v_full[s], 1); mbar_init(&bar->v_empty[s], 1);
-      // per dP buffer, so that a waiter can never be a whole phase behind the barrier it polls
-      mbar_init(&bar->dp_full[s], 1);
-      mbar_init(&bar->ds_full[s], kComputeWarps * 32);
-      mbar_init(&bar->dq_done[s], 1);               // dQ(j) has consumed dS(j): the buffer is free again
-    }
-    mbar_init(&bar->s_full, 1);
-    mbar_init(&bar->s_taken, kComputeWarps * 32);   // every compute thread holds its scores in registers
-    mbar_init(&bar->final_bar, 1);
-    bar->abort_flag = 0;
-    fence_mbar_init();
-  }
-  if (warp == 17) { tmem_alloc(&bar->tmem_base, 512); tmem_relinquish(); }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = bar->tmem_base;
-  if (tmem != 0) {
-    // all 512 columns were requested, so the allocation must start at column 0; the MMA warp relies on it to
-    // keep its TMEM operand addresses compile-time constants
-    __syncthreads();
-    if (warp == 17) tmem_dealloc(tmem, 512);
-    if (tid == 0) atomicExch(a.status, 3);
-    return;
-  }
-
-  if (warp == 16) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      tma_prefetch_desc(&mapQ); tma_prefetch_desc(&mapDO); tma_prefetch_desc(&mapK); tma_prefetch_desc(&mapV);
-      mbar_expect_tx(&bar->q_full, 2 * SM::kTileBytes);
-      tma_load_4d(sQ, &mapQ, &bar->q_full, 0, row0, h * (D / 64), b);
-      tma_load_4d(sDO, &mapDO, &bar->q_full, 0, row0, h * (D / 64), b);
-      for (int it = 0; it < n_blocks; ++it) {
-        const int j = jlo + it;
-        const int ks = it % 3, vs = it & 1;
-        if (!mbar_wait(&bar->k_empty[ks], ((it / 3) & 1) ^ 1, abort_flag)) break;
-        mbar_expect_tx(&bar->k_full[ks], SM::kTileBytes);
-        tma_load_4d(sK + ks * SM::kTileBytes, &mapK, &bar->k_full[ks], 0, j * kTileN, g * (D / 64), b);
-        if (!mbar_wait(&bar->v_empty[vs], ((it >> 1) & 1) ^ 1, abort_flag)) break;
-        mbar_expect_tx(&bar->v_full[vs], SM::kTileBytes);
-        tma_load_4d(sV + vs * SM::kTileBytes, &mapV, &bar->v_full[vs], 0, j * kTileN, g * (D / 64), b);
-      }
-    }
-    __syncwarp();
-  } else if (warp == 17 || warp == 18) {
-    // ------------------------------------------------------------------ MMA issuers
-    // (whole warp runs the loop; only the tcgen05 instructions are predicated on lane 0)
-    {
-      const uint32_t leader = (lane == 0);
-      constexpr uint32_t tmem = 0;   // checked above: TMEM operand addresses are immediates in this loop
-      constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);
-      constexpr uint32_t idesc_dq = idesc_bf16_f32(128, D, 0, 1);
-      const uint64_t dq = smem_desc_sw128(smem_u32(sQ), 16, 1024), ddo = smem_desc_sw128(smem_u32(sDO), 16, 1024);
-      const uint64_t dk_base = smem_desc_sw128(smem_u32(sK), 16, 1024);            // K-major view of a K stage
-      const uint64_t dkm_base = smem_desc_sw128(smem_u32(sK), kBoxBytes, 1024);    // same bytes as MN-major B
-      const uint64_t dv_base = smem_desc_sw128(smem_u32(sV), 16, 1024);
-      constexpr uint32_t kStageStep = SM::kTileBytes >> 4;
-      auto issue_S = [&](int it) {   // S(it) = Q K^T
-        const uint64_t kd = dk_base + (it % 3) * kStageStep;
-#pragma unroll
-        for (int kk = 0; kk < kKSteps; ++kk) {
-          const uint32_t c = ((kk >> 2) * kBoxBytes + (kk & 3) * 32) >> 4;
-          mma_ss(tmem + 128, dq + c, kd + c, idesc_s, kk > 0, leader);
-        }
-        tc_commit(&bar->s_full, leader);
-      };
-      auto issue_dP = [&](int it) {  // dP(it) = dO V^T into dP buffer it&1
-        const uint64_t vd = dv_base + (it & 1) * kStageStep;
-        const uint32_t buf = tmem + 256 + (it & 1) * 128;
-#pragma unroll
-        for (int kk = 0; kk < kKSteps; ++kk) {
-          const uint32_t c = ((kk >> 2) * kBoxBytes + (kk & 3) * 32) >> 4;
-          mma_ss(buf, ddo + c, vd + c, idesc_s, kk > 0, leader);
-        }
-        tc_commit(&bar->dp_full[it & 1], leader);
-        tc_commit(&bar->v_empty[it & 1], leader);
-      };
-      auto issue_dQ = [&](int it) {  // dQ += dS(it) K
-        const uint64_t kd = dkm_base + (it % 3) * kStageStep;
-        const uint32_t buf = tmem + 256 + (it & 1) * 128;
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-          mma_ts(tmem, buf + (kk >> 1) * 32 + (kk & 1) * 8, kd + ((kk * 2048) >> 4), idesc_dq,
-                 (kk > 0 || it > 0) ? 1u : 0u, leader);
-        tc_commit(&bar->k_empty[it % 3], leader);
-        tc_commit(&bar->dq_done[it & 1], leader);
-      };
-      if (warp == 17) {
-        // ---- consumer stream: dQ(it) as soon as dS(it) is in TMEM
-        bool ok = true;
-        for (int it = 0; ok && it < n_blocks; ++it) {
-          if (!mbar_spin_warp(&bar->ds_full[it & 1], (it >> 1) & 1, abort_flag)) { ok = false; break; }
-          if (lane == 0) L2A_TRACE_DQ_POINT(0, 4 * it);
-          tc_fence_after();
-          issue_dQ(it);
-          if (lane == 0) L2A_TRACE_DQ_POINT(0, 4 * it + 1);
-        }
-        if (ok) tc_commit(&bar->final_bar, leader);
-      } else {
-        // ---- producer stream: S(it+1) once the scores of block it are in registers, dP(it+1) once its buffer is free
-        bool ok = mbar_spin_warp(&bar->q_full, 0, abort_flag) && mbar_spin_warp(&bar->k_full[0], 0, abort_flag) &&
-                  mbar_spin_warp(&bar->v_full[0], 0, abort_flag);
-        if (ok) {
-          tc_fence_after();
-          issue_S(0);
-          issue_dP(0);
-        }
-        for (int it = 0; ok && it + 1 < n_blocks; ++it) {
-          if (!mbar_spin_warp(&bar->s_taken, it & 1, abort_flag) ||
-              !mbar_spin_warp(&bar->k_full[(it + 1) % 3], ((it + 1) / 3) & 1, abort_flag)) { ok = false; break; }
-          tc_fence_after();
-          issue_S(it + 1);
-          if (lane == 0) L2A_TRACE_DQ_POINT(0, 4 * it + 2);
-          // dP(it+1) overwrites the buffer that held dS(it-1)
-          if (it >= 1 && !mbar_spin_warp(&bar->dq_done[(it - 1) & 1], ((it - 1) >> 1) & 1, abort_flag)) { ok = false; break; }
-          if (!mbar_spin_warp(&bar->v_full[(it + 1) & 1], ((it + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
-          tc_fence_after();
-          issue_dP(it + 1);
-          if (lane == 0) L2A_TRACE_DQ_POINT(0, 4 * it + 3);
-        }
-      }
-    }
-    __syncwarp();
-  } else {
-    // ------------------------------------------------------------------ P, dS and epilogue
-    const int q = warp >> 2;                        // column quarter
-    const int r = (warp & 3) * 32 + lane;           // query row == TMEM lane
-    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    const int row = row0 + r;
-    const bool valid = row < n_rows;
-    const int seq_row = valid ? (a.global_mode ? q_idx_b[row] : row) : -1;
-    const int pos = valid ? seq_row + a.q_pos_offset - vis_shift : -1;
-    const int pos_lo = valid ? pos - w_eff : 0x7fffffff;
-    const int64_t stat_idx = ((int64_t)b * a.Hq + h) * a.Lq + (valid ? row : 0);
-    const float lse2 = valid ? (a.global_mode ? a.lse_glb : a.lse_loc)[stat_idx] * kLog2e : 0.f;
-    const float delta = valid ? (a.global_mode ? a.delta_glb : a.delta_loc)[stat_idx] : 0.f;
-    const bool ragged = (last - row0 + 1 < kTileM);
-    bool ok = true;
-    for (int it = 0; it < n_blocks; ++it) {
-      if (!__all_sync(0xffffffffu, mbar_wait(&bar->s_full, it & 1, abort_flag))) { ok = false; break; }
-      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_DQ_POINT(1, 4 * it);
-      tc_fence_after();
-      const int k0 = (jlo + it) * kTileN + q * 32;   // first key of this quarter
-      const bool partial = (k0 + 31 > min_pos) || (k0 < max_pos - w_eff) || ragged;
-      uint32_t sv[32];
-      tmem_ld32(tmem + lane_base + 128 + q * 32, sv);
-      tmem_ld_wait();
-      tc_fence_before();
-      mbar_arrive(&bar->s_taken);      // the S columns may be overwritten by the next block's scores
-      if (!partial) {
-#pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          const float2 x = __ffma2_rn(make_float2(__uint_as_float(sv[e]), __uint_as_float(sv[e + 1])),
-                                      make_float2(a.scale_log2, a.scale_log2), make_float2(-lse2, -lse2));
-          sv[e] = __float_as_uint(fast_exp2(x.x));
-          sv[e + 1] = __float_as_uint(fast_exp2(x.y));
-        }
-      } else {
-#pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const int kp = k0 + e;
-          const float p = fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, -lse2));
-          sv[e] = __float_as_uint((kp <= pos && kp >= pos_lo) ? p : 0.f);
-        }
-      }
-      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_DQ_POINT(1, 4 * it + 1);
-      if (!__all_sync(0xffffffffu, mbar_wait(&bar->dp_full[it & 1], (it >> 1) & 1, abort_flag))) { ok = false; break; }
-      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_DQ_POINT(1, 4 * it + 2);
-      tc_fence_after();
-      const uint32_t dp_addr = tmem + lane_base + 256 + (it & 1) * 128 + q * 32;
-      uint32_t dv[32];
-      tmem_ld32(dp_addr, dv);
-      tmem_ld_wait();
-      uint32_t pk[16];
-#pragma unroll
-      for (int e = 0; e < 16; ++e) {
-        const float2 t = __fadd2_rn(make_float2(__uint_as_float(dv[2 * e]), __uint_as_float(dv[2 * e + 1])),
-                                    make_float2(-delta, -delta));
-        const float2 ds = __fmul2_rn(make_float2(__uint_as_float(sv[2 * e]), __uint_as_float(sv[2 * e + 1])), t);
-        pk[e] = pack_bf16(ds.x, ds.y);
-      }
-      tmem_st16(dp_addr, pk);
-      tmem_st_wait();
-      tc_fence_before();
-      mbar_arrive(&bar->ds_full[it & 1]);
-      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_DQ_POINT(1, 4 * it + 3);
-    }
-    // epilogue: quarter q stores D/4 columns of dQ
-    if (ok && __all_sync(0xffffffffu, mbar_wait(&bar->final_bar, 0, abort_flag))) {
-      tc_fence_after();
-      constexpr int kCols = D / 4;     // 32 (D = 128) or 16 (D = 64)
-      bf16* dst = valid ? a.dQ + b * a.dq_st.b + seq_row * a.dq_st.t + (int64_t)h * D + q * kCols : nullptr;
-      uint32_t v[32];
-      tmem_ld32(tmem + lane_base + (q * kCols & ~31), v);   // D = 64: quarters 0,1 / 2,3 share a 32-column load
-      tmem_ld_wait();
-      if (dst) {
-        constexpr int kOff = 0;
-        (void)kOff;
-        const int sub = (D == 64) ? (q & 1) * 16 : 0;
-#pragma unroll
-        for (int c8 = 0; c8 < kCols / 8; ++c8) {
-          float f[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[sub + c8 * 8 + e]) * a.scale;
-          uint4* d4 = reinterpret_cast<uint4*>(dst + c8 * 8);
-          if (a.global_mode) {
-            const uint4 old = *d4;
-            const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              f[2 * k] += bf16lo_to_f32(ow[k]);
-              f[2 * k + 1] += bf16hi_to_f32(ow[k]);
-            }
-          }
-          *d4 = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
-        }
-      }
-    }
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (bar->abort_flag) {
-    const uint64_t t0 = globaltimer_ns();
-    while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
-    if (tid == 0) atomicExch(a.status, 1);
-    __syncthreads();
-  }
-  if (warp == 17) tmem_dealloc(tmem, 512);
-}
-
-// ================================================================================================
-// dK/dV kernel: one block of 128 keys of one KV head per CTA; K and V stay in shared memory, the Q and dO
-// tiles of every query tile that can see the block stream through their own rings (Q: 3 stages, released by
-// the item's last MMA; dO: 2 stages, released earlier), so that the next tile is always resident.
-//   TMEM: dV [0,D) | dK [D,2D) | S^T [256,384) | dP^T [384,512).
-//   P^T / dS^T (bf16): quarter q puts its 16 packed columns at the start of its own 32 columns of S^T / dP^T;
-//   they are the A operands of dV += P^T dO and dK += dS^T Q.
-//   MMA order per item i:  dV(i) | S^T(i+1) | dK(i) | dP^T(i+1): the exponentials of item i+1 run under dK(i) and
-//   dP^T(i+1), its dS under dV(i+1) and S^T(i+2).
-//   Shared memory is used to the last kilobyte (7 tiles of 32 KB at D = 128): the dynamic segment must start
-//   1024-byte aligned, which the kernel checks instead of padding.
-template <int D>
-struct DkvSmem {
-  static constexpr int kTileBytes = 128 * D * 2;
-  static constexpr int kQStages = 3;
-  static constexpr int kDoStages = 2;
-  static constexpr int kKOff = 0;
-  static constexpr int kVOff = kTileBytes;
-  static constexpr int kQOff = 2 * kTileBytes;
-  static constexpr int kDoOff = kQOff + kQStages * kTileBytes;
-  static constexpr int kStatOff = kDoOff + kDoStages * kTileBytes;   // 2 slots x {lse2[128], delta[128], flags[8]}
-  static constexpr int kStatSlot = (2 * 128 + 8) * 4;
-  static constexpr int kBarOff = kStatOff + 2 * kStatSlot;
-  static constexpr int kTotal = kBarOff + 256;
-};
-struct DkvBarriers {
-  uint64_t kv_full;
-  uint64_t q_full[3], q_empty[3];
-  uint64_t do_full[2], do_empty[2];
-  uint64_t st_full[2], st_empty[2];
-  uint64_t s_full, dp_full, p_full, ds_full, final_bar;
-  uint32_t tmem_base;
-  int abort_flag;
-};
 
 struct ItemPlan {
   int loc_t0, loc_nt;   // first local query tile, number of local tiles
@@ -557,11 +194,11 @@ struct ItemPlan {
   int total;            // per_head * G
 };
 
-__device__ __forceinline__ ItemPlan make_plan(const BwdArgs& a, int b, int k0) {
+__device__ __forceinline__ ItemPlan make_plan(const BwdArgs& a, int b, int k0, int span = kTileN) {
   ItemPlan p;
-  // local: rows t with position in [k0, k0 + 127 + W]
+  // local: rows t with position in [k0, k0 + span - 1 + W]
   int tmin = k0 - a.q_pos_offset;
-  const long long tmax_ll = (long long)k0 + kTileN - 1 + a.window - a.q_pos_offset;
+  const long long tmax_ll = (long long)k0 + span - 1 + a.window - a.q_pos_offset;
   int tmax = tmax_ll > a.Lq - 1 ? a.Lq - 1 : (int)tmax_ll;
   if (tmin < 0) tmin = 0;
   if (tmax < tmin || a.skip_local) { p.loc_t0 = 0; p.loc_nt = 0; }
@@ -591,378 +228,6 @@ struct ItemCursor {
   __device__ __forceinline__ void next() { if (++r == per_head) { r = 0; ++h; } }
 };
 
-template <int D>
-__global__ void __launch_bounds__(kDkvThreads, 1)
-bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapDO,
-               const __grid_constant__ CUtensorMap mapQc, const __grid_constant__ CUtensorMap mapDOc,
-               const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, const BwdArgs a) {
-  using SM = DkvSmem<D>;
-  constexpr int kKSteps = D / 16;
-  // key blocks ascending (most work first) inside one KV head; KV heads outermost so that the CTAs
-  // running together share the same query tiles in L2
-  const int j = a.kb_begin + blockIdx.x % a.kb_count;
-  const int rest = blockIdx.x / a.kb_count;
-  const int b = rest % a.B;
-  const int g = rest / a.B;
-  const int G = a.Hq / a.Hkv;
-  const int k0 = j * kTileN;
-  const ItemPlan plan = make_plan(a, b, k0);
-  const int n_c = a.skip_global ? 0 : a.n_routed[b];   // the routing arrays may be NULL when the global part is skipped
-
-  extern __shared__ __align__(1024) uint8_t smem[];
-  uint8_t* sK = smem + SM::kKOff;
-  uint8_t* sV = smem + SM::kVOff;
-  uint8_t* sQ = smem + SM::kQOff;
-  uint8_t* sDO = smem + SM::kDoOff;
-  DkvBarriers* bar = reinterpret_cast<DkvBarriers*>(smem + SM::kBarOff);
-  volatile int* abort_flag = &bar->abort_flag;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-
-  if ((smem_u32(smem) & 1023u) != 0) {   // the swizzled tiles need a 1024-byte aligned base: refuse to run otherwise
-    if (tid == 0) atomicExch(a.status, 2);
-    return;
-  }
-  if (plan.total == 0) {
-    // no query can see these keys: their gradients are zero
-    for (int i = tid; i < kTileN * (D / 8); i += blockDim.x) {
-      const int kr = i / (D / 8), c8 = i % (D / 8);
-      if (k0 + kr < a.Lk) {
-        const int64_t o = (int64_t)g * D + c8 * 8;
-        *reinterpret_cast<uint4*>(a.dK + b * a.dk_st.b + (k0 + kr) * a.dk_st.t + o) = make_uint4(0, 0, 0, 0);
-        *reinterpret_cast<uint4*>(a.dV + b * a.dv_st.b + (k0 + kr) * a.dv_st.t + o) = make_uint4(0, 0, 0, 0);
-      }
-    }
-    return;
-  }
-
-  if (tid == 0) {
-    mbar_init(&bar->kv_full, 1);
-    for (int s = 0; s < 3; ++s) { mbar_init(&bar->q_full[s], 1); mbar_init(&bar->q_empty[s], 1); }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&bar->do_full[s], 1); mbar_init(&bar->do_empty[s], 1);
-      mbar_init(&bar->st_full[s], 32); mbar_init(&bar->st_empty[s], kComputeWarps * 32);
-    }
-    mbar_init(&bar->s_full, 1);
-    mbar_init(&bar->dp_full, 1);
-    mbar_init(&bar->p_full, kComputeWarps * 32);
-    mbar_init(&bar->ds_full, kComputeWarps * 32);
-    mbar_init(&bar->final_bar, 1);
-    bar->abort_flag = 0;
-    fence_mbar_init();
-  }
-  if (warp == 17) { tmem_alloc(&bar->tmem_base, 512); tmem_relinquish(); }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = bar->tmem_base;
-  if (tmem != 0) {
-    // all 512 columns were requested, so the allocation must start at column 0; the MMA warp relies on it to
-    // keep its TMEM operand addresses compile-time constants
-    __syncthreads();
-    if (warp == 17) tmem_dealloc(tmem, 512);
-    if (tid == 0) atomicExch(a.status, 3);
-    return;
-  }
-
-  if (warp == 16) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      tma_prefetch_desc(&mapQ); tma_prefetch_desc(&mapDO); tma_prefetch_desc(&mapQc); tma_prefetch_desc(&mapDOc);
-      mbar_expect_tx(&bar->kv_full, 2 * SM::kTileBytes);
-      tma_load_4d(sK, &mapK, &bar->kv_full, 0, k0, g * (D / 64), b);
-      tma_load_4d(sV, &mapV, &bar->kv_full, 0, k0, g * (D / 64), b);
-      ItemCursor cur(plan, g * G);
-      int qs = 0;
-      uint32_t qph = 0;
-      for (int i = 0; i < plan.total; ++i) {
-        const int glb = cur.glb(), row0 = cur.tile() * kTileM, hc = cur.h * (D / 64);
-        cur.next();
-        if (!mbar_wait(&bar->q_empty[qs], qph ^ 1, abort_flag)) break;
-        L2A_TRACE_POINT(3, 2 * i);
-        mbar_expect_tx(&bar->q_full[qs], SM::kTileBytes);
-        tma_load_4d(sQ + qs * SM::kTileBytes, glb ? &mapQc : &mapQ, &bar->q_full[qs], 0, row0, hc, b);
-        if (!mbar_wait(&bar->do_empty[i & 1], ((i >> 1) & 1) ^ 1, abort_flag)) break;
-        mbar_expect_tx(&bar->do_full[i & 1], SM::kTileBytes);
-        tma_load_4d(sDO + (i & 1) * SM::kTileBytes, glb ? &mapDOc : &mapDO, &bar->do_full[i & 1], 0, row0, hc, b);
-        L2A_TRACE_POINT(3, 2 * i + 1);
-        if (++qs == 3) { qs = 0; qph ^= 1; }
-      }
-    }
-    __syncwarp();
-  } else if (warp == 18) {
-    // ------------------------------------------------------------------ row statistics of each item
-    // lse * log2(e) and Delta of the item's 128 query rows, plus per-quarter mask flags, go to shared memory.
-    // The global loads of item i+1 are issued before waiting for its slot, so their latency is hidden.
-    float r_lse[4], r_delta[4];
-    int r_pos[4], r_glb = 0, r_row0 = 0;
-    ItemCursor cur(plan, g * G);
-    auto load_item = [&]() {
-      const int h = cur.h, glb = cur.glb(), row0 = cur.tile() * kTileM;
-      cur.next();
-      const int n_rows = glb ? n_c : a.Lq;
-      const float* lse = glb ? a.lse_glb : a.lse_loc;
-      const float* dl = glb ? a.delta_glb : a.delta_loc;
-      r_glb = glb;
-      r_row0 = row0;
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int row = row0 + q * 32 + lane;
-        const bool valid = row < n_rows;
-        const int64_t si = ((int64_t)b * a.Hq + h) * a.Lq + (valid ? row : 0);
-        r_lse[q] = valid ? __ldg(&lse[si]) * kLog2e : 0.f;
-        r_delta[q] = valid ? __ldg(&dl[si]) : 0.f;
-        r_pos[q] = valid ? (glb ? __ldg(&a.q_idx[(int64_t)b * a.Lq + row]) - a.vis_shift : row) + a.q_pos_offset : -1;
-      }
-    };
-    load_item();
-    for (int i = 0; i < plan.total; ++i) {
-      const int s = i & 1;
-      if (!__all_sync(0xffffffffu, mbar_wait(&bar->st_empty[s], ((i >> 1) & 1) ^ 1, abort_flag))) break;
-      float* st_lse = reinterpret_cast<float*>(smem + SM::kStatOff + s * SM::kStatSlot);
-      float* st_delta = st_lse + 128;
-      int* st_flags = reinterpret_cast<int*>(st_delta + 128);
-      const int w_eff = r_glb ? 0x3fffffff : a.window;
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int col = q * 32 + lane;
-        st_lse[col] = r_lse[q];
-        st_delta[col] = -r_delta[q];   // negated: dS = P * (dP + (-Delta)) with packed f32x2 arithmetic
-        // quarter q needs the element mask unless every (key, query) pair of it is visible
-        const bool lane_ok = r_pos[q] >= 0 && (k0 + kTileN - 1 <= r_pos[q]) && (k0 >= r_pos[q] - w_eff);
-        const bool interior = __all_sync(0xffffffffu, lane_ok);
-        if (lane == 0) st_flags[q] = interior ? 0 : 1;
-      }
-      if (lane == 0) { st_flags[4] = r_glb; st_flags[5] = r_row0; }
-      __syncwarp();
-      mbar_arrive(&bar->st_full[s]);
-      if (i + 1 < plan.total) load_item();
-    }
-  } else if (warp == 17) {
-    // ------------------------------------------------------------------ MMA issuer
-    // (whole warp runs the loop; only the tcgen05 instructions are predicated on lane 0)
-    {
-      const uint32_t leader = (lane == 0);
-      constexpr uint32_t tmem = 0;   // checked above: TMEM operand addresses are immediates in this loop
-      constexpr uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);
-      constexpr uint32_t idesc_acc = idesc_bf16_f32(128, D, 0, 1);
-      constexpr uint32_t kStageStep = SM::kTileBytes >> 4;
-      const uint64_t dk = smem_desc_sw128(smem_u32(sK), 16, 1024), dv = smem_desc_sw128(smem_u32(sV), 16, 1024);
-      const uint64_t dq_base = smem_desc_sw128(smem_u32(sQ), 16, 1024);
-      const uint64_t ddo_base = smem_desc_sw128(smem_u32(sDO), 16, 1024);
-      const uint64_t dqm_base = smem_desc_sw128(smem_u32(sQ), kBoxBytes, 1024);      // Q / dO as MN-major B
-      const uint64_t ddom_base = smem_desc_sw128(smem_u32(sDO), kBoxBytes, 1024);
-      auto issue_S = [&](int qs) {    // S^T = K Q^T
-        const uint64_t qd = dq_base + qs * kStageStep;
-#pragma unroll
-        for (int kk = 0; kk < kKSteps; ++kk) {
-          const uint32_t c = ((kk >> 2) * kBoxBytes + (kk & 3) * 32) >> 4;
-          mma_ss(tmem + 256, dk + c, qd + c, idesc_s, kk > 0, leader);
-        }
-        tc_commit(&bar->s_full, leader);
-      };
-      auto issue_dP = [&](int ds) {   // dP^T = V dO^T
-        const uint64_t dod = ddo_base + ds * kStageStep;
-#pragma unroll
-        for (int kk = 0; kk < kKSteps; ++kk) {
-          const uint32_t c = ((kk >> 2) * kBoxBytes + (kk & 3) * 32) >> 4;
-          mma_ss(tmem + 384, dv + c, dod + c, idesc_s, kk > 0, leader);
-        }
-        tc_commit(&bar->dp_full, leader);
-      };
-      auto issue_dV = [&](int ds, bool first) {   // dV += P^T dO
-        const uint64_t dod = ddom_base + ds * kStageStep;
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-          mma_ts(tmem, tmem + 256 + (kk >> 1) * 32 + (kk & 1) * 8, dod + ((kk * 2048) >> 4), idesc_acc,
-                 (kk > 0 || !first) ? 1u : 0u, leader);
-        tc_commit(&bar->do_empty[ds], leader);
-      };
-      auto issue_dK = [&](int qs, bool first) {   // dK += dS^T Q
-        const uint64_t qd = dqm_base + qs * kStageStep;
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-          mma_ts(tmem + D, tmem + 384 + (kk >> 1) * 32 + (kk & 1) * 8, qd + ((kk * 2048) >> 4), idesc_acc,
-                 (kk > 0 || !first) ? 1u : 0u, leader);
-        tc_commit(&bar->q_empty[qs], leader);
-      };
-      bool ok = mbar_spin_warp(&bar->kv_full, 0, abort_flag) && mbar_spin_warp(&bar->q_full[0], 0, abort_flag) &&
-                mbar_spin_warp(&bar->do_full[0], 0, abort_flag);
-      if (ok) {
-        tc_fence_after();
-        issue_S(0);
-        issue_dP(0);
-      }
-      int qs = 0;           // Q stage of item i
-      uint32_t qph = 0;     // its phase parity
-      for (int i = 0; ok && i < plan.total; ++i) {
-        const bool more = i + 1 < plan.total;
-        int qn = qs + 1;
-        uint32_t qphn = qph;
-        if (qn == 3) { qn = 0; qphn ^= 1; }
-        if (!mbar_spin_warp(&bar->p_full, i & 1, abort_flag)) { ok = false; break; }
-        if (lane == 0) L2A_TRACE_POINT(0, 4 * i);
-        tc_fence_after();
-        issue_dV(i & 1, i == 0);
-        if (lane == 0) L2A_TRACE_POINT(2, 4 * i + 3);
-        if (more) {
-          if (!mbar_spin_warp(&bar->q_full[qn], qphn, abort_flag)) { ok = false; break; }
-          if (lane == 0) L2A_TRACE_POINT(0, 4 * i + 1);
-          tc_fence_after();
-          issue_S(qn);
-        }
-        if (!mbar_spin_warp(&bar->ds_full, i & 1, abort_flag)) { ok = false; break; }
-        if (lane == 0) L2A_TRACE_POINT(0, 4 * i + 2);
-        tc_fence_after();
-        issue_dK(qs, i == 0);
-        if (more) {
-          if (!mbar_spin_warp(&bar->do_full[(i + 1) & 1], ((i + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
-          tc_fence_after();
-          issue_dP((i + 1) & 1);
-        }
-        if (lane == 0) L2A_TRACE_POINT(0, 4 * i + 3);
-        qs = qn;
-        qph = qphn;
-      }
-      if (ok) tc_commit(&bar->final_bar, leader);
-    }
-    __syncwarp();
-  } else {
-    // ------------------------------------------------------------------ P^T / dS^T and epilogue
-    const int q = warp >> 2;                           // query-column quarter of this warp
-    const int kr = (warp & 3) * 32 + lane;             // key inside the block == TMEM lane
-    const int kp = k0 + kr;
-    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    const uint32_t s_addr = tmem + lane_base + 256 + q * 32;
-    const uint32_t dp_addr = tmem + lane_base + 384 + q * 32;
-    bool ok = true;
-    for (int i = 0; i < plan.total; ++i) {
-      const int s = i & 1;
-      // this item's row statistics go to registers before the scores are waited for
-      if (!__all_sync(0xffffffffu, mbar_wait(&bar->st_full[s], (i >> 1) & 1, abort_flag))) { ok = false; break; }
-      const uint32_t st_base = smem_u32(smem + SM::kStatOff + s * SM::kStatSlot);
-      const int* st_flags = reinterpret_cast<const int*>(smem + SM::kStatOff + s * SM::kStatSlot) + 2 * 128;
-      float st[32];
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        const float4 v = lds128(st_base + (q * 32 + c * 4) * 4);
-        st[4 * c] = v.x; st[4 * c + 1] = v.y; st[4 * c + 2] = v.z; st[4 * c + 3] = v.w;
-      }
-      const bool masked = st_flags[q] != 0;
-      if (!__all_sync(0xffffffffu, mbar_wait(&bar->s_full, i & 1, abort_flag))) { ok = false; break; }
-      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_POINT(1, 4 * i);
-      tc_fence_after();
-      uint32_t pp[16];
-      {
-        uint32_t sv[32];
-        tmem_ld32(s_addr, sv);
-        tmem_ld_wait();
-        if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_POINT(2, 4 * i);
-        // the element mask is needed only for the few tiles that straddle the causal diagonal or a window edge:
-        // two loop versions, so that the common one has no branches
-        if (!masked) {
-#pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const float2 x = __ffma2_rn(make_float2(__uint_as_float(sv[2 * e]), __uint_as_float(sv[2 * e + 1])),
-                                        make_float2(a.scale_log2, a.scale_log2), make_float2(-st[2 * e], -st[2 * e + 1]));
-            pp[e] = pack_bf16(fast_exp2(x.x), fast_exp2(x.y));
-          }
-        } else {
-          const int glb = st_flags[4], row0 = st_flags[5];
-          const int w_eff = glb ? 0x3fffffff : a.window;
-          const int n_rows = glb ? n_c : a.Lq;
-          const int32_t* qi = a.q_idx + (int64_t)b * a.Lq;
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            int pos[2];
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-              const int row = row0 + q * 32 + e + u;
-              pos[u] = row < n_rows ? (glb ? __ldg(&qi[row]) - a.vis_shift : row) + a.q_pos_offset : -1;
-            }
-            float p0 = fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, -st[e]));
-            float p1 = fast_exp2(fmaf(__uint_as_float(sv[e + 1]), a.scale_log2, -st[e + 1]));
-            p0 = (kp <= pos[0] && kp >= pos[0] - w_eff) ? p0 : 0.f;
-            p1 = (kp <= pos[1] && kp >= pos[1] - w_eff) ? p1 : 0.f;
-            pp[e >> 1] = pack_bf16(p0, p1);
-          }
-        }
-      }
-      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_POINT(2, 4 * i + 1);
-      tmem_st16(s_addr, pp);     // P^T over the first half of this quarter's own S^T columns
-      tmem_st_wait();
-      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_POINT(2, 4 * i + 2);
-      tc_fence_before();
-      mbar_arrive(&bar->p_full);
-      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_POINT(1, 4 * i + 1);
-      // Delta of the same rows, again ahead of the wait; after this the statistics slot may be refilled
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        const float4 v = lds128(st_base + (128 + q * 32 + c * 4) * 4);
-        st[4 * c] = v.x; st[4 * c + 1] = v.y; st[4 * c + 2] = v.z; st[4 * c + 3] = v.w;
-      }
-      mbar_arrive(&bar->st_empty[s]);
-      if (!__all_sync(0xffffffffu, mbar_wait(&bar->dp_full, i & 1, abort_flag))) { ok = false; break; }
-      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_POINT(1, 4 * i + 2);
-      tc_fence_after();
-      uint32_t pd[16];
-      {
-        uint32_t dv[32];
-        tmem_ld32(dp_addr, dv);
-        tmem_ld_wait();
-#pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          // dS uses the bf16-rounded P, the same value the dV product sees; st[] holds -Delta
-          const float2 t = __fadd2_rn(make_float2(__uint_as_float(dv[2 * e]), __uint_as_float(dv[2 * e + 1])),
-                                      make_float2(st[2 * e], st[2 * e + 1]));
-          const float2 ds = __fmul2_rn(make_float2(bf16lo_to_f32(pp[e]), bf16hi_to_f32(pp[e])), t);
-          pd[e] = pack_bf16(ds.x, ds.y);
-        }
-      }
-      tmem_st16(dp_addr, pd);    // dS^T over the first half of this quarter's own dP^T columns
-      tmem_st_wait();
-      tc_fence_before();
-      mbar_arrive(&bar->ds_full);
-      if (warp == L2A_TRACE_WARP && lane == 0) L2A_TRACE_POINT(1, 4 * i + 3);
-    }
-    // epilogue: quarters 0,1 store the two column halves of dV, quarters 2,3 those of dK
-    if (ok && __all_sync(0xffffffffu, mbar_wait(&bar->final_bar, 0, abort_flag))) {
-      tc_fence_after();
-      const bool valid = kp < a.Lk;
-      const int which = q >> 1, half = q & 1;
-      const RowStrides st = which == 0 ? a.dv_st : a.dk_st;
-      const int64_t o = b * st.b + (valid ? kp : 0) * st.t + (int64_t)g * D + half * (D / 2);
-      bf16* dst = (which == 0 ? a.dV : a.dK) + o;
-      const float mul = which == 0 ? 1.0f : a.scale;
-#pragma unroll
-      for (int c = 0; c < D / 64; ++c) {
-        uint32_t v[32];
-        tmem_ld32(tmem + lane_base + which * D + half * (D / 2) + c * 32, v);
-        tmem_ld_wait();
-        if (valid) {
-          uint4* d4 = reinterpret_cast<uint4*>(dst + c * 32);
-#pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            float f[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[8 * x + e]) * mul;
-            d4[x] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
-                               pack_bf16(f[6], f[7]));
-          }
-        }
-      }
-    }
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (bar->abort_flag) {
-    const uint64_t t0 = globaltimer_ns();
-    while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
-    if (tid == 0) atomicExch(a.status, 1);
-    __syncthreads();
-  }
-  if (warp == 17) tmem_dealloc(tmem, 512);
-}
-
 // ================================================================================================
 // Five-GEMM backward kernel: the key/value-stationary kernel above plus the fifth GEMM, dQ(i) = dS(i) K, so that
 // S and dP are computed once per tile pair.  dQ(i) is a fresh 128 x D accumulator per item; the compute warps read
@@ -980,7 +245,7 @@ bwd_dkv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 //   slack: T: S^T -> P -> dV -> S^T and U: dP^T -> dS -> dQ -> read-out -> dP^T; dK(i-1) fills the pipe while the
 //   exponentials of item i run.
 template <int D>
-struct FusedSmem {
+struct BwdSmem {
   static constexpr int kTileBytes = 128 * D * 2;
   static constexpr int kKOff = 0;
   static constexpr int kVOff = kTileBytes;
@@ -992,7 +257,7 @@ struct FusedSmem {
   static constexpr int kBarOff = kStatOff + 2 * kStatSlot;
   static constexpr int kTotal = kBarOff + 256;
 };
-struct FusedBarriers {
+struct BwdBarriers {
   uint64_t kv_full;
   uint64_t q_full[2], q_empty[2];
   uint64_t do_full[2], do_empty[2];
@@ -1001,14 +266,14 @@ struct FusedBarriers {
   uint32_t tmem_base;
   int abort_flag;
 };
-static_assert(sizeof(FusedBarriers) <= 256, "barrier block");
+static_assert(sizeof(BwdBarriers) <= 256, "barrier block");
 
 template <int D>
 __global__ void __launch_bounds__(kDkvThreads, 1)
-bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapDO,
+bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapDO,
                const __grid_constant__ CUtensorMap mapQc, const __grid_constant__ CUtensorMap mapDOc,
                const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, const BwdArgs a) {
-  using SM = FusedSmem<D>;
+  using SM = BwdSmem<D>;
   constexpr int kKSteps = D / 16;
   // key blocks ascending (most work first) inside one KV head; KV heads outermost so that the CTAs
   // running together share the same query tiles in L2
@@ -1026,7 +291,7 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
   uint8_t* sV = smem + SM::kVOff;
   uint8_t* sQ = smem + SM::kQOff;
   uint8_t* sDO = smem + SM::kDoOff;
-  FusedBarriers* bar = reinterpret_cast<FusedBarriers*>(smem + SM::kBarOff);
+  BwdBarriers* bar = reinterpret_cast<BwdBarriers*>(smem + SM::kBarOff);
   uint8_t* sDS = smem + SM::kDsOff;          // dS (bf16, [key][query])
   volatile int* abort_flag = &bar->abort_flag;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -1271,18 +536,6 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       tc_fence_before();
       mbar_arrive(&bar->u_free);       // the values are in registers: dP^T(i+1) may overwrite the columns
       float* dst = acc_prev + warp * (8 * D) + lane * 4;
-#if defined(L2A_DIAG_ST)
-#pragma unroll
-      for (int c = 0; c < D / 16; ++c) {
-        const int k = sub + 4 * c;
-        asm volatile("st.global.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + c * 128), "f"(__uint_as_float(v[k])),
-                     "f"(__uint_as_float(v[k + 1])), "f"(__uint_as_float(v[k + 2])), "f"(__uint_as_float(v[k + 3]))
-                     : "memory");
-      }
-#elif !defined(L2A_DIAG_NO_RED)
-#ifdef L2A_DIAG_QUARTER
-      if (q == 0)
-#endif
 #pragma unroll
       for (int c = 0; c < D / 16; ++c) {
         const int k = sub + 4 * c;
@@ -1290,9 +543,6 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                      "f"(__uint_as_float(v[k + 1])), "f"(__uint_as_float(v[k + 2])), "f"(__uint_as_float(v[k + 3]))
                      : "memory");
       }
-#else
-      if (v[0] == 0x12345678u && dst == nullptr) *dst = 0.f;
-#endif
       return true;
     };
     for (int i = 0; i < plan.total; ++i) {
@@ -1447,21 +697,22 @@ __global__ void __launch_bounds__(256) dq_zero_kernel(float* __restrict__ acc_lo
   }
 }
 
-// fp32 dQ accumulators -> bf16 dQ: dQ_t = scale * (local(t) + d_t * global(prefix[t])).  One CTA per (batch, row tile,
-// head); the accumulator blocks are read in their own order (512 contiguous bytes per warp), the bf16 rows leave
+// fp32 dQ accumulators -> bf16 dQ: dQ_t = scale * (local(t) + d_t * global(prefix[t])), for the row tiles
+// [tile_begin, tile_begin + tile_count).  One CTA per (batch, row tile, head); the accumulator blocks are read in their own order (512 contiguous bytes per warp), the bf16 rows leave
 // through shared memory as whole 2 D-byte segments.
 template <int D>
 __global__ void __launch_bounds__(256) dq_merge_kernel(const float* __restrict__ acc_loc, const float* __restrict__ acc_glb,
                                                        const uint8_t* __restrict__ d_mask,
                                                        const int32_t* __restrict__ prefix, bf16* __restrict__ dQ, int B,
-                                                       int L, int Hq, float scale, int64_t bs, int64_t ts) {
+                                                       int L, int Hq, float scale, int64_t bs, int64_t ts,
+                                                       int tile_begin, int tile_count) {
   constexpr int kChunks = D / 8;             // 16-byte chunks per bf16 row
   constexpr int kRowBytes = D * 2 + 16;      // padded: conflict-free 16-byte accesses down a column
   __shared__ __align__(16) uint8_t tile_s[kTileM * kRowBytes];
   const int n_tiles = (L + kTileM - 1) / kTileM;
   const int h = blockIdx.x % Hq;
-  const int tile = (blockIdx.x / Hq) % n_tiles;
-  const int b = blockIdx.x / (Hq * n_tiles);
+  const int tile = tile_begin + (blockIdx.x / Hq) % tile_count;
+  const int b = blockIdx.x / (Hq * tile_count);
   const int64_t tile_floats = kTileM * D;
   const float* loc = acc_loc ? acc_loc + (((int64_t)b * Hq + h) * n_tiles + tile) * tile_floats : nullptr;
   for (int idx = threadIdx.x; idx < kTileM * kChunks; idx += blockDim.x) {
@@ -1496,103 +747,80 @@ __global__ void __launch_bounds__(256) dq_merge_kernel(const float* __restrict__
   }
 }
 
+}  // namespace
+int delta_ctas_per_sm(int D) {
+  int per_sm = 0;
+  const cudaError_t e = D == 128 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bwd_delta_kernel<128>, 256, 0)
+                                 : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bwd_delta_kernel<64>, 256, 0);
+  return (e != cudaSuccess || per_sm < 1) ? 1 : per_sm;
+}
+namespace {
+
 size_t rows_bytes(const l2a_params* p) { return align_up((size_t)p->B * p->Lq * p->Hq * p->D * sizeof(bf16), 256); }
 size_t stat_bytes(const l2a_params* p) { return align_up((size_t)p->B * p->Hq * p->Lq * sizeof(float), 256); }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+}  // namespace
+
+int dkv_split_block(int n_kblocks) { return n_kblocks >= 8 ? (3 * n_kblocks) / 4 : 0; }
+
+// First row tile whose dQ still receives contributions from the key blocks at or after `split`: a row at position p
+// only meets keys <= p, so after the key blocks below `split` the rows with p < 128 * split are final.
+int dq_final_tiles(int split, int q_pos_offset, int n_tiles) {
+  const long long rows = (long long)split * kTileN - q_pos_offset;
+  if (rows <= 0) return 0;
+  const long long t = rows / kTileM;
+  return t > n_tiles ? n_tiles : (int)t;
+}
+
 template <int D>
-cudaError_t launch_bwd_kernels(const BwdArgs& base, const CUtensorMap& mapQ, const CUtensorMap& mapDO,
-                               const CUtensorMap& mapQc, const CUtensorMap& mapDOc, const CUtensorMap& mapK,
-                               const CUtensorMap& mapV, cudaStream_t s) {
-  cudaError_t e;
-  e = cudaFuncSetAttribute(bwd_dkv_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, DkvSmem<D>::kTotal);
+cudaError_t launch_bwd(const BwdArgs& base, const CUtensorMap& mapQ, const CUtensorMap& mapDO,
+                       const CUtensorMap& mapQc, const CUtensorMap& mapDOc, const CUtensorMap& mapK,
+                       const CUtensorMap& mapV, const uint8_t* d_mask, cudaStream_t s) {
+  const DeviceInfo* dev = device_info();
+  if (dev == nullptr) return cudaErrorUnknown;
+  static PerDeviceOnce once;
+  cudaError_t e = once.run([] {
+    return cudaFuncSetAttribute(bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::kTotal);
+  });
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(bwd_dq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqSmem<D>::kTotal);
-  if (e != cudaSuccess) return e;
-  // dQ first: it is the largest result (Hq / Hkv times dK or dV), so a caller that ships results to the host as
-  // they complete can move it while the dK/dV kernel, the longest of the three, is still running
-  const unsigned n_tiles = (base.Lq + kTileM - 1) / kTileM;
-  BwdArgs a = base;
-  a.global_mode = 0;
-  if (!base.skip_local) {
-    bwd_dq_kernel<D><<<n_tiles * base.B * base.Hq, kDqThreads, DqSmem<D>::kTotal, s>>>(mapQ, mapDO, mapK, mapV, a);
-  } else {
-    // the global launch adds into dQ at the routed positions: every other row of dQ is zero
-    for (int b = 0; b < base.B; ++b) {
-      e = cudaMemset2DAsync(base.dQ + b * base.dq_st.b, (size_t)base.dq_st.t * sizeof(bf16), 0,
-                            (size_t)base.Hq * D * sizeof(bf16), base.Lq, s);
-      if (e != cudaSuccess) return e;
-    }
-  }
-  phase_events().mark(s);
-  a.global_mode = 1;
-  if (!base.skip_global)
-    bwd_dq_kernel<D><<<n_tiles * base.B * base.Hq, kDqThreads, DqSmem<D>::kTotal, s>>>(mapQc, mapDOc, mapK, mapV, a);
+  const int n_tiles = (base.Lq + kTileM - 1) / kTileM;
+  dq_zero_kernel<<<dev->sms * 8, 256, 0, s>>>(base.dq_acc_loc, base.dq_acc_glb, base.n_routed, base.B, base.Hq, n_tiles,
+                                              kTileM * D);
   phase_events().mark(s);
   const int n_kblocks = (base.Lk + kTileN - 1) / kTileN;
-  // A caller that registered a seventh phase event wants the first three quarters of dK / dV early (to move them
-  // while the rest is computed): two launches over key-block ranges, a boundary in between.
+  // A caller that registered seven phase events wants the gradients of the early rows while the rest is computed (to
+  // move them to the host): two launches over key-block ranges, each followed by the merge of the dQ rows it finishes.
   const int split = phase_events().n >= 7 ? dkv_split_block(n_kblocks) : 0;
-  a = base;
+  const int t_split = split > 0 ? dq_final_tiles(split, base.q_pos_offset, n_tiles) : n_tiles;
   for (int part = 0; part < 2; ++part) {
+    if (part == 1 && split == 0) break;
+    BwdArgs a = base;
     a.kb_begin = part == 0 ? 0 : split;
     a.kb_count = part == 0 ? (split > 0 ? split : n_kblocks) : n_kblocks - split;
-    if (part == 1 && split == 0) break;
-    bwd_dkv_kernel<D><<<(unsigned)a.kb_count * base.B * base.Hkv, kDkvThreads, DkvSmem<D>::kTotal, s>>>(
+    bwd_kernel<D><<<(unsigned)a.kb_count * base.B * base.Hkv, kDkvThreads, BwdSmem<D>::kTotal, s>>>(
         mapQ, mapDO, mapQc, mapDOc, mapK, mapV, a);
+    phase_events().mark(s);
+    const int t0 = part == 0 ? 0 : t_split, t1 = part == 0 ? t_split : n_tiles;
+    if (t1 > t0)
+      dq_merge_kernel<D><<<(unsigned)((t1 - t0) * base.B * base.Hq), 256, 0, s>>>(
+          base.dq_acc_loc, base.dq_acc_glb, d_mask, base.prefix, base.dQ, base.B, base.Lq, base.Hq, base.scale,
+          base.dq_st.b, base.dq_st.t, t0, t1 - t0);
     phase_events().mark(s);
   }
   return cudaGetLastError();
 }
 
-}  // namespace
-
-int dkv_split_block(int n_kblocks) { return n_kblocks >= 8 ? (3 * n_kblocks) / 4 : 0; }
-
-template <int D>
-cudaError_t launch_bwd_fused(const BwdArgs& base, const CUtensorMap& mapQ, const CUtensorMap& mapDO,
-                             const CUtensorMap& mapQc, const CUtensorMap& mapDOc, const CUtensorMap& mapK,
-                             const CUtensorMap& mapV, const uint8_t* d_mask, cudaStream_t s) {
-  cudaError_t e = cudaFuncSetAttribute(bwd_fused_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       FusedSmem<D>::kTotal);
-  if (e != cudaSuccess) return e;
-  int device = 0, sms = 148;
-  if (cudaGetDevice(&device) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
-  const int n_tiles = (base.Lq + kTileM - 1) / kTileM;
-  dq_zero_kernel<<<sms * 8, 256, 0, s>>>(base.dq_acc_loc, base.dq_acc_glb, base.n_routed, base.B, base.Hq, n_tiles,
-                                         kTileM * D);
-  phase_events().mark(s);
-  BwdArgs a = base;
-  const int n_kblocks = (base.Lk + kTileN - 1) / kTileN;
-  a.kb_begin = 0;
-  a.kb_count = n_kblocks;
-  bwd_fused_kernel<D><<<(unsigned)n_kblocks * base.B * base.Hkv, kDkvThreads, FusedSmem<D>::kTotal, s>>>(
-      mapQ, mapDO, mapQc, mapDOc, mapK, mapV, a);
-  phase_events().mark(s);
-  dq_merge_kernel<D><<<(unsigned)(n_tiles * base.B * base.Hq), 256, 0, s>>>(
-      base.dq_acc_loc, base.dq_acc_glb, d_mask, base.prefix, base.dQ, base.B, base.Lq, base.Hq, base.scale,
-      base.dq_st.b, base.dq_st.t);
-  phase_events().mark(s);
-  return cudaGetLastError();
-}
-
 // one fp32 dQ accumulator: whole 128-row tiles
 size_t acc_bytes(const l2a_params* p) {
-  return (p->flags & L2A_FLAG_FUSED_DQ)
-             ? align_up((size_t)p->B * p->Hq * ceil_div(p->Lq, kTileM) * kTileM * p->D * sizeof(float), 256) : 0;
+  return align_up((size_t)p->B * p->Hq * ceil_div(p->Lq, kTileM) * kTileM * p->D * sizeof(float), 256);
 }
 size_t bwd_ws_size(const l2a_params* p) { return kWsHeaderBytes + 2 * rows_bytes(p) + 3 * stat_bytes(p) + 2 * acc_bytes(p); }
 
 }  // namespace l2a
 
 using namespace l2a;
-
-#ifdef L2A_TRACE
-extern "C" int l2a_debug_read_trace(long long* host) {
-  return (int)cudaMemcpyFromSymbol(host, g_trace, sizeof(g_trace));
-}
-#endif
 
 extern "C" l2a_status l2a_backward(const l2a_params* p, const void* Q, const void* K, const void* V,
                                    const uint8_t* d_mask, const int32_t* q_idx, const int32_t* n_routed,
@@ -1635,7 +863,6 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   float* lse_c = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + 2 * stat_bytes(p));
   float* dq_acc_loc = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + 3 * stat_bytes(p));
   float* dq_acc_glb = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p) + 3 * stat_bytes(p) + acc_bytes(p));
-  const bool fused = p->flags & L2A_FLAG_FUSED_DQ;
   // Shared-window backward: the window's share of a routed row's global gradient rides on the local items (see
   // bwd_delta_kernel).  Needs the same gradient for both outputs; the flag permits it, other modes just ignore it.
   const bool share = (p->flags & L2A_FLAG_SHARED_WINDOW) && dS_loc == dO && !skip_local && !skip_global &&
@@ -1668,11 +895,10 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   pe.mark(s);
   {
     // one resident wave of 8-warp CTAs; the warps take the tokens round-robin
-    int device = 0, sms = 148, per_sm = 0;
-    if (cudaGetDevice(&device) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    const DeviceInfo* dev = device_info();
+    if (dev == nullptr) return L2A_ERR_CUDA;
     auto kern = p->D == 128 ? bwd_delta_kernel<128> : bwd_delta_kernel<64>;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 256, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
-    int64_t blocks = (int64_t)sms * per_sm;
+    int64_t blocks = (int64_t)dev->sms * (p->D == 128 ? dev->delta_ctas_128 : dev->delta_ctas_64);
     const int64_t max_blocks = ((int64_t)p->B * p->Lq + 7) / 8;
     if (blocks > max_blocks) blocks = max_blocks;
     kern<<<(unsigned)blocks, 256, 0, s>>>(static_cast<const bf16*>(dO), static_cast<const bf16*>(dS_loc),
@@ -1687,14 +913,12 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
       if (cudaGetLastError() != cudaSuccess) return L2A_ERR_CUDA;
     }
   }
-  pe.mark(s);
   BwdArgs a;
   a.B = p->B; a.Lq = p->Lq; a.Lk = p->Lk; a.Hq = p->Hq; a.Hkv = p->Hkv; a.D = p->D;
   a.window = p->window < (1 << 30) ? p->window : (1 << 30);   // any window >= Lk is the same
   a.q_pos_offset = p->q_pos_offset;
   a.scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->D);
   a.scale_log2 = a.scale * kLog2e;
-  a.global_mode = 0;
   a.skip_local = skip_local ? 1 : 0;
   a.skip_global = skip_global ? 1 : 0;
   a.q_idx = q_idx; a.n_routed = n_routed; a.prefix = prefix;
@@ -1702,15 +926,11 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   a.vis_shift = share ? (p->window < (1 << 30) ? p->window : (1 << 30)) + 1 : 0; a.delta_loc = delta_loc; a.delta_glb = delta_glb;
   a.dQ = static_cast<bf16*>(dQ); a.dK = static_cast<bf16*>(dK); a.dV = static_cast<bf16*>(dV);
   a.dq_st = qs; a.dk_st = ks; a.dv_st = vs;
-  a.dq_acc_loc = fused && !skip_local ? dq_acc_loc : nullptr;
-  a.dq_acc_glb = fused && !skip_global ? dq_acc_glb : nullptr;
+  a.dq_acc_loc = !skip_local ? dq_acc_loc : nullptr;
+  a.dq_acc_glb = !skip_global ? dq_acc_glb : nullptr;
   a.status = reinterpret_cast<int*>(ws);
-  cudaError_t e;
-  if (fused)
-    e = p->D == 128 ? launch_bwd_fused<128>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, skip_global ? nullptr : d_mask, s)
-                    : launch_bwd_fused<64>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, skip_global ? nullptr : d_mask, s);
-  else
-    e = p->D == 128 ? launch_bwd_kernels<128>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, s)
-                    : launch_bwd_kernels<64>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, s);
+  const cudaError_t e =
+      p->D == 128 ? launch_bwd<128>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, skip_global ? nullptr : d_mask, s)
+                  : launch_bwd<64>(a, mapQ, mapDO, mapQc, mapDOc, mapK, mapV, skip_global ? nullptr : d_mask, s);
   return e == cudaSuccess ? L2A_OK : L2A_ERR_CUDA;
 }

@@ -27,20 +27,6 @@ namespace l2a {
 
 namespace {
 
-// Optional clock tracing of one CTA (development builds only: -DL2A_TRACE_FWD=<block>).
-#ifdef L2A_TRACE_FWD
-__device__ long long g_trace_fwd[4][8192];
-#define L2A_FWD_TRACE(role, idx)                                                                   \
-  do {                                                                                             \
-    if (blockIdx.x == (L2A_TRACE_FWD) && (idx) < 8192) g_trace_fwd[role][idx] = clock64();         \
-  } while (0)
-#else
-#define L2A_FWD_TRACE(role, idx)
-#endif
-#ifndef L2A_TRACE_FWD_WARP
-#define L2A_TRACE_FWD_WARP 0
-#endif
-
 constexpr int kNumTiles = 2;
 constexpr int kStages = 2;
 constexpr int kSoftmaxWarps = 16;
@@ -268,7 +254,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             uint32_t& pc = t ? p_cnt1 : p_cnt0;
             if (!mbar_spin_warp(&bar->p_full[t], pc & 1, abort_flag)) { ok = false; }
             else {
-              if (lane == 0) L2A_FWD_TRACE(0, 4 * (j - jlo) + 2 * t);
               ++pc;
               if (!v_ready) {
                 if (!mbar_spin_warp(&bar->v_full[s], ph, abort_flag)) ok = false;
@@ -289,7 +274,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
             if (ok) {
               tc_fence_after();
               issue_qk(t, sn);
-              if (lane == 0) L2A_FWD_TRACE(0, 4 * (j - jlo) + 2 * t + 1);
             }
           }
         }
@@ -330,7 +314,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         const int j = my.lo + i;
         // warp-uniform outcome: the TMEM loads/stores below are warp-collective
         if (!__all_sync(0xffffffffu, mbar_wait(&bar->s_full[t], i & 1, abort_flag))) { ok = false; break; }
-        if (warp == L2A_TRACE_FWD_WARP && lane == 0) L2A_FWD_TRACE(1, 4 * i);
         tc_fence_after();
         const int k0 = j * kTileN + hf * 64;
         const bool partial = (k0 + 63 > my.min_pos - vis_shift) || (k0 < my.max_pos - w_eff);
@@ -363,10 +346,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         // row maximum over both halves: publish mine, meet the other half, read theirs
         float* slot = xch + (((i & 1) * kNumTiles + t) * 2) * kTileM;
         slot[hf * kTileM + r] = mx;
-        if (warp == L2A_TRACE_FWD_WARP && lane == 0) L2A_FWD_TRACE(1, 4 * i + 1);
         mbar_arrive(&bar->xch[t]);
         if (!__all_sync(0xffffffffu, mbar_wait(&bar->xch[t], i & 1, abort_flag))) { ok = false; break; }
-        if (warp == L2A_TRACE_FWD_WARP && lane == 0) L2A_FWD_TRACE(1, 4 * i + 2);
         mx = fmaxf(mx, slot[(hf ^ 1) * kTileM + r]);
         const float m_new = fmaxf(m_use, mx * a.scale_log2);
 
@@ -426,7 +407,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         tmem_st_wait();
         tc_fence_before();
         mbar_arrive(&bar->p_full[t]);
-        if (warp == L2A_TRACE_FWD_WARP && lane == 0) L2A_FWD_TRACE(1, 4 * i + 3);
       }
 
       // ---- epilogue: O / l, log-sum-exp, store (local) or scatter + combine (global)
@@ -536,25 +516,23 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
 
 }  // namespace
 
-#ifdef L2A_TRACE_FWD
-}  // namespace l2a
-extern "C" int l2a_debug_read_trace_fwd(long long* host) {
-  return (int)cudaMemcpyFromSymbol(host, l2a::g_trace_fwd, sizeof(l2a::g_trace_fwd));
-}
-namespace l2a {
-#endif
-
 cudaError_t launch_attn_fwd(const FwdArgs& a, const CUtensorMap& mapQ, const CUtensorMap& mapK,
                             const CUtensorMap& mapV, cudaStream_t stream) {
   const unsigned grid = (unsigned)(a.pair_end - a.pair_begin) * a.Hq * a.B;
   if (a.pair_end <= a.pair_begin) return cudaSuccess;
   cudaError_t e;
   if (a.D == 128) {
-    e = cudaFuncSetAttribute(attn_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<128>::kTotal);
+    static PerDeviceOnce once;
+    e = once.run([] {
+      return cudaFuncSetAttribute(attn_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<128>::kTotal);
+    });
     if (e != cudaSuccess) return e;
     attn_fwd_kernel<128><<<grid, kFwdThreads, FwdSmem<128>::kTotal, stream>>>(mapQ, mapK, mapV, a);
   } else {
-    e = cudaFuncSetAttribute(attn_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<64>::kTotal);
+    static PerDeviceOnce once;
+    e = once.run([] {
+      return cudaFuncSetAttribute(attn_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<64>::kTotal);
+    });
     if (e != cudaSuccess) return e;
     attn_fwd_kernel<64><<<grid, kFwdThreads, FwdSmem<64>::kTotal, stream>>>(mapQ, mapK, mapV, a);
   }

@@ -61,6 +61,23 @@ PhaseEvents& phase_events() {
   return pe;
 }
 
+const DeviceInfo* device_info() {
+  static DeviceInfo info[PerDeviceOnce::kMaxDevices];
+  static PerDeviceOnce once;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= PerDeviceOnce::kMaxDevices) return nullptr;
+  const cudaError_t e = once.run([dev] {
+    DeviceInfo d;
+    cudaError_t r = cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev);
+    if (r != cudaSuccess) return r;
+    d.delta_ctas_64 = delta_ctas_per_sm(64);
+    d.delta_ctas_128 = delta_ctas_per_sm(128);
+    info[dev] = d;
+    return cudaSuccess;
+  });
+  return e == cudaSuccess ? &info[dev] : nullptr;
+}
+
 bool encode_rows_map(CUtensorMap* map, const void* base, int batch, int rows, int row_elems, int box_rows,
                      int head_dim, int64_t batch_stride, int64_t token_stride) {
   encode_tiled_fn enc = get_encode();
@@ -127,12 +144,11 @@ __global__ void __launch_bounds__(128) wait_timeout_selftest_kernel(int* status,
   }
   __syncthreads();
   volatile int* af = &abort_flag;
-  bool ok;
-  if (threadIdx.x < 32) ok = mbar_wait(&never_arrives, 0, af, limit_ns);   // gives up after limit_ns, raises the flag
-  else ok = mbar_wait(&second, 0, af, 1000 * limit_ns);                     // leaves as soon as the flag is up
+  const uint64_t second_limit = 1000 * limit_ns < kWaitLimitNs ? 1000 * limit_ns : kWaitLimitNs;
+  if (threadIdx.x < 32) mbar_wait(&never_arrives, 0, af, limit_ns);   // gives up after limit_ns, raises the flag
+  else mbar_wait(&second, 0, af, second_limit);                        // leaves as soon as the flag is up
   __syncthreads();
   if (threadIdx.x == 0 && abort_flag) atomicExch(status, 1);
-  (void)ok;
 }
 }  // namespace
 }  // namespace l2a
@@ -535,9 +551,9 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
   L2A_TRY(cudaMemcpyAsync(host->O, dev->O, qb, cudaMemcpyDeviceToHost, aux.out));
   if (bwd) {
     L2A_TRY(cudaStreamWaitEvent(s, aux.up, 0));
-    // phase boundary 4 of the backward = both dQ kernels have finished: dQ can leave while dK/dV are computed;
-    // with seven events the dK/dV kernel runs as two launches and boundary 5 says that the key rows of the first
-    // one are final
+    // With seven phase events the backward runs as two key-block ranges; boundary 4 says that the gradients of the
+    // early rows (dK, dV of the first range's keys, dQ of the rows that only see those keys) are final: they leave
+    // on the download stream while the second range is computed, the rest after the last kernel.
     void* phase_events[7];
     for (int i = 0; i < 7; ++i) phase_events[i] = aux.phase[i];
     st = l2a_profile_next_call(phase_events, 7);
@@ -546,21 +562,30 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
                       dev->S_save, dev->A_c, dev->lse_loc, dev->lse_glb, dev->dQ, dev->dK, dev->dV, nullptr,
                       dev->bwd_ws, dev->bwd_ws_bytes, stream);
     if (st != L2A_OK) return st;
-    L2A_TRY(cudaStreamWaitEvent(aux.out, aux.phase[4], 0));
-    L2A_TRY(cudaMemcpyAsync(host->dQ, dev->dQ, qb, cudaMemcpyDeviceToHost, aux.out));
-    const int64_t split_rows = (int64_t)dkv_split_block(ceil_div(p->Lk, kTileN)) * kTileN;   // 0: one launch
-    const size_t krow = (size_t)p->Hkv * p->D * sizeof(bf16);
-    if (split_rows > 0) L2A_TRY(cudaStreamWaitEvent(aux.out, aux.phase[5], 0));
+    const int split = dkv_split_block(ceil_div(p->Lk, kTileN));   // 0: one launch
+    const int64_t k_early = (int64_t)split * kTileN;
+    int64_t q_early = (int64_t)dq_final_tiles(split, p->q_pos_offset, ceil_div(p->Lq, kTileM)) * kTileM;
+    if (q_early > p->Lq) q_early = p->Lq;
+    const size_t krow = (size_t)p->Hkv * p->D * sizeof(bf16), qrow = (size_t)p->Hq * p->D * sizeof(bf16);
+    if (split > 0) L2A_TRY(cudaStreamWaitEvent(aux.out, aux.phase[4], 0));
     for (int b = 0; b < p->B; ++b) {
-      const size_t base = (size_t)b * p->Lk * krow, early = (size_t)split_rows * krow, late = (size_t)p->Lk * krow - early;
-      uint8_t *hk = static_cast<uint8_t*>(host->dK) + base, *hv = static_cast<uint8_t*>(host->dV) + base;
-      const uint8_t *gk = static_cast<const uint8_t*>(dev->dK) + base, *gv = static_cast<const uint8_t*>(dev->dV) + base;
-      if (early > 0) {
-        L2A_TRY(cudaMemcpyAsync(hk, gk, early, cudaMemcpyDeviceToHost, aux.out));
-        L2A_TRY(cudaMemcpyAsync(hv, gv, early, cudaMemcpyDeviceToHost, aux.out));
+      const size_t kbase = (size_t)b * p->Lk * krow, kearly = (size_t)k_early * krow, kall = (size_t)p->Lk * krow;
+      const size_t qbase = (size_t)b * p->Lq * qrow, qearly = (size_t)q_early * qrow, qall = (size_t)p->Lq * qrow;
+      uint8_t *hk = static_cast<uint8_t*>(host->dK) + kbase, *hv = static_cast<uint8_t*>(host->dV) + kbase;
+      uint8_t* hq = static_cast<uint8_t*>(host->dQ) + qbase;
+      const uint8_t *gk = static_cast<const uint8_t*>(dev->dK) + kbase, *gv = static_cast<const uint8_t*>(dev->dV) + kbase;
+      const uint8_t* gq = static_cast<const uint8_t*>(dev->dQ) + qbase;
+      if (split > 0 && qearly > 0) L2A_TRY(cudaMemcpyAsync(hq, gq, qearly, cudaMemcpyDeviceToHost, aux.out));
+      if (split > 0 && kearly > 0) {
+        L2A_TRY(cudaMemcpyAsync(hk, gk, kearly, cudaMemcpyDeviceToHost, aux.out));
+        L2A_TRY(cudaMemcpyAsync(hv, gv, kearly, cudaMemcpyDeviceToHost, aux.out));
       }
-      L2A_TRY(cudaMemcpyAsync(hk + early, gk + early, late, cudaMemcpyDeviceToHost, s));
-      L2A_TRY(cudaMemcpyAsync(hv + early, gv + early, late, cudaMemcpyDeviceToHost, s));
+      const size_t qoff = split > 0 ? qearly : 0, koff = split > 0 ? kearly : 0;
+      if (qall > qoff) L2A_TRY(cudaMemcpyAsync(hq + qoff, gq + qoff, qall - qoff, cudaMemcpyDeviceToHost, s));
+      if (kall > koff) {
+        L2A_TRY(cudaMemcpyAsync(hk + koff, gk + koff, kall - koff, cudaMemcpyDeviceToHost, s));
+        L2A_TRY(cudaMemcpyAsync(hv + koff, gv + koff, kall - koff, cudaMemcpyDeviceToHost, s));
+      }
     }
   }
   L2A_TRY(cudaEventRecord(aux.down, aux.out));

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/l2a.h"
 
 namespace l2a {
@@ -102,8 +104,35 @@ struct FwdArgs {
   const float* lse_loc;      // [B,Hq,Lq] by row; read only when shared_window is set
 };
 size_t bwd_ws_size(const l2a_params* p);
-// First key block of the second dK/dV launch when the backward is asked for the early boundary (0: not split).
+// First key block of the second backward launch when the caller asked for the early boundary (0: not split), and the
+// number of leading 128-row tiles of dQ that are final after the first launch.
 int dkv_split_block(int n_kblocks);
+int dq_final_tiles(int split, int q_pos_offset, int n_tiles);
+
+// Facts about the current device that the launchers need, looked up once per device and cached.
+struct DeviceInfo {
+  int sms;
+  int delta_ctas_64, delta_ctas_128;   // resident CTAs per SM of the Delta kernel
+};
+const DeviceInfo* device_info();       // NULL if the CUDA runtime fails
+int delta_ctas_per_sm(int D);          // defined with the backward
+// Runs fn() once per device (per call site owning the object): for cudaFuncSetAttribute and the like.
+struct PerDeviceOnce {
+  static constexpr int kMaxDevices = 64;
+  std::atomic<int> done[kMaxDevices];
+  PerDeviceOnce() { for (auto& d : done) d.store(0); }
+  template <class F>
+  cudaError_t run(F fn) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return fn();
+    if (done[dev].load(std::memory_order_acquire)) return cudaSuccess;
+    e = fn();                         // idempotent: two threads racing here both succeed
+    if (e == cudaSuccess) done[dev].store(1, std::memory_order_release);
+    return e;
+  }
+};
 
 // One-shot, thread-local registration of phase-boundary events (see l2a_profile_next_call).
 struct PhaseEvents {

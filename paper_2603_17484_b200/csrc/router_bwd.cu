@@ -32,9 +32,9 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
 // and adds its dW partial sums once.
 __global__ void __launch_bounds__(kRbMaxThreads)
 router_backward_kernel(const bf16* __restrict__ S, const float* __restrict__ w, const float* __restrict__ logits,
-                       const float* __restrict__ dgate, float coeff, const bf16* __restrict__ dO,
+                       const float* __restrict__ dgate, float coeff, const bf16* dO /* may alias dS */,
                        float* __restrict__ dz_out, float* __restrict__ dw, float* __restrict__ dbias,
-                       bf16* __restrict__ dS, int64_t n_tokens, int row_elems) {
+                       bf16* dS, int64_t n_tokens, int row_elems) {
   __shared__ float dz_s[kRbTokens];
   const int tid = threadIdx.x;
   const int64_t t_begin = n_tokens * blockIdx.x / gridDim.x, t_end = n_tokens * (blockIdx.x + 1) / gridDim.x;
@@ -90,7 +90,7 @@ router_backward_kernel(const bf16* __restrict__ S, const float* __restrict__ w, 
         for (int t = 0; t < nt; ++t) {
           float sv[8], ov[8];
           unpack8(__ldg(&S4[(int64_t)t * n_chunks]), sv);
-          unpack8(__ldg(&dO4[(int64_t)t * n_chunks]), ov);
+          unpack8(dO4[(int64_t)t * n_chunks], ov);   // plain load: dS may be written in place
           const float dz = dz_s[t];
 #pragma unroll
           for (int e = 0; e < 8; ++e) {

@@ -21,7 +21,6 @@ FLAG_SKIP_LOCAL = 2
 FLAG_SKIP_GLOBAL = 4
 FLAG_FORCE_ALL_GLOBAL = 8
 FLAG_GLOBAL_PHASE = 16
-FLAG_FUSED_DQ = 32
 FLAG_SHARED_WINDOW = 64
 ROUTER_MASK_U8 = 0
 ROUTER_LOGITS_F32 = 1

@@ -6,16 +6,17 @@ max abs error <= 2e-2 and mean abs error <= 2e-3.  A bf16 number of magnitude |x
 2^-7 |x| apart at worst, so storing the exact result already costs up to 2^-8 |x| (more than 2e-2 once
 |x| >= 5.12; dK/dV of early keys sum over thousands of queries and get there).  The bounds therefore
 apply to the value before that final rounding: |err| <= 2e-2 + 2^-8 |want| element-wise and
-mean|err| <= 2e-3 + 2^-9 mean|want|.
+mean|err| <= 2e-3 + 2^-9 mean|want|.  Forward outputs are held to exactly that.
 
-Gradients additionally inherit the bf16 rounding of the MMA operands P and dS (relative 2^-9 each, standard
-flash-attention practice): an element of dQ picks up scale * 2^-9 * sum_j |dS_ij| |k_j|.  With N(0,1) inputs dO.v has
-standard deviation sqrt(D) ~ 11, so the very first rows (two or three keys, P ~ 0.5) can carry |dS| ~ 10, where bf16
-is spaced 0.0625 apart, and a dQ element can be off by ~0.03 (reproduced by emulating the kernel's roundings in
-numpy).  A dK element of an early key sums such terms over every row and every query head of its group: with G = 8,
-D = 64 (scale 1/8) and ~500 terms of |dS| ~ 3 its noise has a standard deviation of ~0.01, so the largest of
-~10^4 elements reaches 0.03-0.04.  Gradient checks therefore let a fraction of at most 1e-5 of the elements (rounded
-up to a whole element) exceed the bound, and none by more than a factor of two."""
+Gradients additionally inherit the bf16 rounding of the MMA operands P and dS (relative 2^-9 each, the
+reading taken where the paper is silent on rounding: fp32 scores and soft-max, bf16 tensor-core operands).
+tests/test_rounding_model.py applies exactly these roundings to the oracle's fp64 arithmetic on the shapes of
+tests/test_gpu_backward.py: the excursions they cause beyond the bound are rare (at most one element in 2.6e5) and
+small (at most 1.03 x the bound).  Gradient checks therefore let a fraction of at most 1e-5 of the elements (rounded up
+to a whole element) exceed the bound, none by more than a factor of 1.5.
+
+Every comparison also records how many elements exceed the plain 2e-2 and the bound; the session prints the table
+(tests/conftest.py)."""
 import math
 
 import numpy as np
@@ -33,8 +34,11 @@ def to_f64(t: torch.Tensor) -> np.ndarray:
     return t.detach().float().cpu().numpy().astype(np.float64)
 
 
+STATS = []   # (what, elements, over plain 2e-2, over the bound, largest err / bound): printed at the end of the session
+
+
 def check_close(got: np.ndarray, want: np.ndarray, what: str, max_abs=MAX_ABS, mean_abs=MEAN_ABS, outlier_frac=0.0,
-                extra_outliers=0):
+                cap=1.5):
     assert got.shape == want.shape, (what, got.shape, want.shape)
     assert np.isfinite(got).all(), f"{what}: non-finite values in the GPU result"
     if got.size == 0:
@@ -44,9 +48,13 @@ def check_close(got: np.ndarray, want: np.ndarray, what: str, max_abs=MAX_ABS, m
     excess = err - bound
     i = np.unravel_index(np.argmax(excess), err.shape)
     n_over = int((excess > 0).sum())
-    msg = f"{what}: abs err {err[i]:.4g} at {i} (got {got[i]}, want {want[i]}), max abs err {err.max():.4g}, {n_over} over"
-    assert n_over <= math.ceil(outlier_frac * err.size) + extra_outliers, msg
-    assert (err <= 2.0 * bound).all(), msg
+    n_plain = int((err > max_abs).sum())
+    ratio = float((err / bound).max())
+    STATS.append((what, int(err.size), n_plain, n_over, ratio))
+    msg = (f"{what}: abs err {err[i]:.4g} at {i} (got {got[i]}, want {want[i]}), max abs err {err.max():.4g}, "
+           f"{n_over} over the bound, {n_plain} over {max_abs}, largest err/bound {ratio:.3f}")
+    assert n_over <= math.ceil(outlier_frac * err.size), msg
+    assert ratio <= cap, msg
     mean_tol = mean_abs + 2.0 ** -9 * np.abs(want).mean()
     assert err.mean() <= mean_tol, f"{what}: mean abs err {err.mean():.4g} > {mean_tol:.4g}"
 
@@ -110,11 +118,11 @@ class Case:
         if self.backward:
             check_close(to_f64(b.S_save), ref["s"], "S_save")
             check_close(to_f64(b.lse_loc), ref["lse_loc"], "lse_loc", LSE_ABS, LSE_ABS)
-            A_c, lse_glb = to_f64(b.A_c), to_f64(b.lse_glb)
             for bi in range(self.shape.B):
                 rows = q_idx[bi, :n[bi]]
-                check_close(A_c[bi, :n[bi]], ref["a"][bi, rows], "A_c")
-                check_close(lse_glb[bi, :, :n[bi]], ref["lse_glb"][bi][:, rows], "lse_glb", LSE_ABS, LSE_ABS)
+                # rows past the routed count are never written: slice on the device before converting
+                check_close(to_f64(b.A_c[bi, :n[bi]]), ref["a"][bi, rows], "A_c")
+                check_close(to_f64(b.lse_glb[bi, :, :n[bi]]), ref["lse_glb"][bi][:, rows], "lse_glb", LSE_ABS, LSE_ABS)
         return ref
 
 
@@ -128,13 +136,22 @@ def run_backward(case: "Case", with_dgate=True):
     return b
 
 
-def check_backward_full(case: "Case", dq_first_rows=0):
-    """dq_first_rows: elements of dQ per (batch entry, head) that may exceed the bound (by less than a factor of two)
-    on top of the 1e-5 fraction.  The fused backward forms dS from the bf16-rounded P (the dQ kernel of the
-    seven-GEMM path keeps P in fp32), so the rows with two or three keys, where |dS| ~ 10, carry sqrt(2) more noise."""
+def check_backward_full(case: "Case"):
     b = case.buf
     dQ, dK, dV = oracle.backward_full(case.shape, case.u16("Q"), case.u16("K"), case.u16("V"), case.d, case.u16("dO"))
-    check_close(to_f64(b.dQ), dQ, "dQ", outlier_frac=1e-5, extra_outliers=dq_first_rows * dQ.shape[0] * dQ.shape[2])
+    check_close(to_f64(b.dQ), dQ, "dQ", outlier_frac=1e-5)
     check_close(to_f64(b.dK), dK, "dK", outlier_frac=1e-5)
     check_close(to_f64(b.dV), dV, "dV", outlier_frac=1e-5)
     return dQ, dK, dV
+
+
+def check_same_or_rounding(a: torch.Tensor, b: torch.Tensor, what: str):
+    """Two runs of a result whose fp32 sums are taken in no fixed order: equal up to the bf16 rounding of sums that
+    differ in their last fp32 bits (one bf16 step on a few elements at most; where terms cancel, the difference is that
+    of the fp32 sums themselves, far below 1e-4)."""
+    x, y = a.float(), b.float()
+    diff = (x - y).abs()
+    step = 2.0 ** -7 * torch.maximum(x.abs(), y.abs()) + 1e-4
+    assert bool((diff <= step).all()), (what, float((diff / step).max()))
+    frac = float((diff > 0).float().mean())
+    assert frac <= 1e-2, (what, "fraction of differing elements", frac)

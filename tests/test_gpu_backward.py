@@ -5,7 +5,7 @@ import torch
 
 import oracle
 from paper_2603_17484_b200 import l2a, synth
-from tests.gpu_util import Case, check_close, check_backward_full, run_backward, to_f64
+from tests.gpu_util import Case, check_close, check_backward_full, check_same_or_rounding, run_backward, to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -53,7 +53,9 @@ def test_backward_identities_at_length():
     assert to_f64(c.buf.dK).__abs__().max() <= 2e-2
 
 
-def test_backward_run_twice_is_bit_identical():
+def test_backward_run_twice():
+    """dK and dV are summed on chip in a fixed order: bit-identical from run to run.  dQ is summed over the key blocks with
+    atomic fp32 additions in no fixed order: equal up to the rounding of sums that differ in their last bits."""
     B, L, Hq, Hkv, D, W = 1, 777, 2, 1, 128, 100
     d = synth.mask_bernoulli(B, L, 0.3, seed=2)
     c = Case(B, L, Hq, Hkv, D, W, d, seed=3, backward=True)
@@ -61,5 +63,6 @@ def test_backward_run_twice_is_bit_identical():
     run_backward(c)
     first = [t.clone() for t in (c.buf.dQ, c.buf.dK, c.buf.dV)]
     run_backward(c)
-    for x, y in zip(first, (c.buf.dQ, c.buf.dK, c.buf.dV)):
+    check_same_or_rounding(first[0], c.buf.dQ, "dQ")
+    for x, y in zip(first[1:], (c.buf.dK, c.buf.dV)):
         assert torch.equal(x.view(torch.int16), y.view(torch.int16))

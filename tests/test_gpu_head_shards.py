@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from paper_2603_17484_b200 import l2a, synth
-from tests.gpu_util import Case, run_backward
+from tests.gpu_util import check_same_or_rounding, Case, run_backward
 
 pytestmark = pytest.mark.gpu
 
@@ -46,5 +46,8 @@ def test_two_head_shards_equal_the_whole_layer(extra):
         assert l2a.l2a_workspace_status(fwd_ws) == 0 and l2a.l2a_workspace_status(bwd_ws) == 0
         dgate += part      # the gate gradient sums over heads: the one value ranks would have to add up
     for k in out:
-        assert torch.equal(out[k].view(torch.int16), whole[k].view(torch.int16)), k
+        if k == "dQ":      # summed over the key blocks with fp32 atomics: order not fixed
+            check_same_or_rounding(out[k], whole[k], k)
+        else:
+            assert torch.equal(out[k].view(torch.int16), whole[k].view(torch.int16)), k
     assert torch.allclose(dgate, whole["dgate"], rtol=1e-5, atol=1e-4)

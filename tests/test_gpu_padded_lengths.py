@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from paper_2603_17484_b200 import l2a, synth
-from tests.gpu_util import Case, run_backward
+from tests.gpu_util import check_same_or_rounding, Case, run_backward
 
 pytestmark = pytest.mark.gpu
 
@@ -39,6 +39,9 @@ def test_right_padded_batch_matches_single_sequences():
             # bit-identical: same tiles and order of operations per row; a key block may see more query tiles than in
             # the single call, but those are masked or carry dO = 0 and add exact zeros
             got, want = getattr(batch.buf, name)[i, :n], getattr(c.buf, name)[0]
-            assert torch.equal(got.contiguous().view(torch.int16), want.view(torch.int16)), (name, i)
+            if name == "dQ":   # summed over the key blocks with fp32 atomics: order not fixed
+                check_same_or_rounding(got.contiguous(), want, name)
+            else:
+                assert torch.equal(got.contiguous().view(torch.int16), want.view(torch.int16)), (name, i)
         assert torch.all(batch.buf.dQ[i, n:] == 0) and torch.all(batch.buf.dK[i, n:] == 0)
         assert torch.all(batch.buf.dV[i, n:] == 0)

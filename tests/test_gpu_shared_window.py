@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from paper_2603_17484_b200 import l2a, synth
-from tests.gpu_util import Case, check_backward_full, check_close, run_backward, to_f64
+from tests.gpu_util import check_same_or_rounding, Case, check_backward_full, check_close, run_backward, to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -100,7 +100,10 @@ def test_shared_window_step_host_and_routed_forward(backward):
         getattr(c.buf, k).zero_()
     l2a.l2a_step_host(c.p, host, c.buf, l2a.ROUTER_MASK_U8, 0.0)
     for k, w in want.items():
-        assert torch.equal(host[k].view(torch.int16), w.cpu().view(torch.int16)), k
+        if k == "dQ":      # summed over the key blocks with fp32 atomics: order not fixed
+            check_same_or_rounding(host[k], w.cpu(), k)
+        else:
+            assert torch.equal(host[k].view(torch.int16), w.cpu().view(torch.int16)), k
 
 
 def test_shared_window_split_backward_falls_back():
@@ -121,4 +124,7 @@ def test_shared_window_split_backward_falls_back():
                            b.lse_loc, b.lse_glb, b.dQ, b.dK, b.dV, None, b.bwd_ws)
     torch.cuda.synchronize()
     for k, w in want.items():
-        assert torch.equal(getattr(b, k).view(torch.int16), w.view(torch.int16)), k
+        if k == "dQ":
+            check_same_or_rounding(getattr(b, k), w, k)
+        else:
+            assert torch.equal(getattr(b, k).view(torch.int16), w.view(torch.int16)), k

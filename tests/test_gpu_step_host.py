@@ -4,7 +4,7 @@ import pytest
 import torch
 
 from paper_2603_17484_b200 import l2a, synth
-from tests.gpu_util import Case, run_backward
+from tests.gpu_util import check_same_or_rounding, Case, run_backward
 
 pytestmark = pytest.mark.gpu
 
@@ -33,4 +33,7 @@ def test_step_host_matches_device_calls(backward, B, L, Lk):
             host[k].fill_(float("nan"))
         l2a.l2a_step_host(c.p, host, c.buf, l2a.ROUTER_MASK_U8, 0.0)
         for k, w in want.items():
-            assert torch.equal(host[k].view(torch.int16), w.cpu().view(torch.int16)), (k, rep)
+            if k == "dQ":      # summed over the key blocks with fp32 atomics: order not fixed
+                check_same_or_rounding(host[k], w.cpu(), k)
+            else:
+                assert torch.equal(host[k].view(torch.int16), w.cpu().view(torch.int16)), (k, rep)

@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from paper_2603_17484_b200 import l2a, synth
-from tests.gpu_util import Case, run_backward
+from tests.gpu_util import check_same_or_rounding, Case, run_backward
 
 pytestmark = pytest.mark.gpu
 
@@ -54,7 +54,7 @@ def test_strided_tensors_match_dense(B, L, Hq, Hkv, D, W, extra):
     assert torch.equal(_bits(Obuf[:, :, :wq]), _bits(dense["O"].view(B, L, wq)))
     assert torch.equal(_bits(b.S_save), _bits(dense["S_save"]))
     assert torch.equal(b.lse_loc, dense["lse_loc"])
-    assert torch.equal(_bits(dQ[:, :L]), _bits(dense["dQ"].view(B, L, wq)))
+    check_same_or_rounding(dQ[:, :L], dense["dQ"].view(B, L, wq), "dQ")   # fp32 atomic sums: order not fixed
     assert torch.equal(_bits(dK[:, :L]), _bits(dense["dK"].view(B, L, wk)))
     assert torch.equal(_bits(dV[:, :L, :wk]), _bits(dense["dV"].view(B, L, wk)))
     assert torch.equal(b.dgate, dense["dgate"])

@@ -31,7 +31,9 @@ def test_two_phase_layer_matches_single_call():
     z_ref = oracle.router_logits(S_bits, w.cpu().numpy(), -0.3)
     z = logits.cpu().numpy()
     assert np.abs(z - z_ref).max() <= 1e-3 * (1 + np.abs(z_ref).max())
-    check_close(sum_sq.cpu().numpy().astype(np.float64), oracle.gate_regulariser_sum(z_ref), "sum sigmoid^2", 1e-2 * L, 1e-2 * L)
+    # the regulariser's sum (Eq. 6) of the kernel's own fp32 logits: fp32 sigmoid and an atomic fp32 sum
+    want_sq = oracle.gate_regulariser_sum(z.astype(np.float64))
+    assert np.abs(sum_sq.cpu().numpy().astype(np.float64) - want_sq).max() <= 1e-4 * want_sq.max()
     # the decision is taken on the kernel's own fp32 logits: integer results are then exact
     d = oracle.route(z, 0.0)
     assert 0.02 < d.mean() < 0.9

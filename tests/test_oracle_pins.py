@@ -273,6 +273,16 @@ def test_router_logits_closed_forms():
     np.testing.assert_allclose(oracle.gate_regulariser_sum(z0), np.full(B, L * 0.25), atol=1e-15)   # sigmoid(0)^2 = 1/4
 
 
+def test_gate_regulariser_closed_forms():
+    # Eq. 6 without its lambda / (n L) factor: sum over tokens of sigmoid(z_t)^2.  sigmoid(ln 3) = 3/4 and
+    # sigmoid(-ln 3) = 1/4, so the squares are 9/16 and 1/16: a sign slip in the exponent, a missing square or a sum over the
+    # wrong axis fails.
+    ln3 = np.log(3.0)
+    z = np.array([[ln3, ln3, -ln3], [-ln3, -ln3, -ln3]])
+    np.testing.assert_allclose(oracle.gate_regulariser_sum(z), [2 * 0.5625 + 0.0625, 3 * 0.0625], rtol=1e-14)
+    np.testing.assert_allclose(oracle.gate_regulariser_sum(np.array([[40.0, -40.0]])), [1.0], rtol=1e-14)
+
+
 def test_router_backward_is_the_gradient_of_the_relaxed_loss():
     # Under the straight-through estimator the loss seen by the router is, with a_t and dL/do_t held fixed,
     #   F(W, bias, s) = sum_t g_t * sigmoid(z_t) + c * sum_t sigmoid(z_t)^2,   z_t = W s_t + bias,  g_t = dL/do_t . a_t
