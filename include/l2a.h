@@ -44,7 +44,9 @@ typedef enum {
   L2A_ERR_UNSUPPORTED = -2,    /* valid request this build does not implement               */
   L2A_ERR_WORKSPACE = -3,      /* workspace pointer NULL / misaligned / too small           */
   L2A_ERR_CUDA = -4,           /* a CUDA runtime or driver call failed (launch, encode)     */
-  L2A_ERR_DEVICE_TIMEOUT = -5  /* a bounded device-side wait ran out (l2a_workspace_status) */
+  L2A_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait ran out (l2a_workspace_status) */
+  L2A_ERR_DEVICE_BOUNDS = -6   /* debug build only (-DL2A_DEBUG): an index derived from q_idx / prefix / tile      */
+                               /* metadata fell outside its tensor; the store was skipped (l2a_workspace_status)   */
 } l2a_status;
 
 /* l2a_params.flags */
@@ -140,7 +142,8 @@ l2a_status l2a_selftest_wait_timeout(void* ws, unsigned limit_us, void* stream);
 /*
  * Reads the status word the kernels of earlier calls left in workspace `ws` (any of the three).
  * Synchronises `stream`.  Returns L2A_OK, or L2A_ERR_DEVICE_TIMEOUT if a bounded device-side wait
- * ran out in some kernel that used this workspace since it was last used by a successful call.
+ * ran out in some kernel that used this workspace since it was last used by a successful call, or
+ * (debug build) L2A_ERR_DEVICE_BOUNDS if an index check failed.
  */
 l2a_status l2a_workspace_status(const void* ws, void* stream);
 
@@ -243,6 +246,28 @@ l2a_status l2a_backward(const l2a_params* p, const void* Q, const void* K, const
                         const int32_t* prefix, const void* dO, const void* S_save, const void* A_c,
                         const float* lse_loc, const float* lse_glb, void* dQ, void* dK, void* dV,
                         float* dgate, void* bwd_ws, size_t bwd_ws_bytes, void* stream);
+
+/*
+ * Forward and backward of a layer whose Global Attention module has its OWN Q/K/V (Section 3.1: both modules are
+ * initialised from the base model's attention and have their own projections; Global Attention projects the local
+ * output s_t).  (Q, K, V) feed Local Attention, (Qg, Kg, Vg) -- same shapes and strides -- feed Global Attention
+ * of the routed rows; o_t = s_t + d_t a_t as before.  All three of Qg, Kg, Vg NULL: one set feeds both modules and the
+ * calls are l2a_forward / l2a_backward.  Otherwise they are the two-phase sequences described above in one call,
+ * bit for bit (dQ up to the order of its fp32 sums): forward = local phase, then global phase added into O;
+ * backward = the local module's gradients into dQ, dK, dV and the global module's into dQg, dKg, dVg (dQg is zero
+ * outside the routed rows); dgate as in l2a_backward.  L2A_FLAG_SHARED_WINDOW does not apply to two sets and is
+ * ignored; the SKIP / PHASE flags (and, in the backward, FORCE_ALL_GLOBAL) are L2A_ERR_INVALID_ARG.
+ */
+l2a_status l2a_forward_sets(const l2a_params* p, const void* Q, const void* K, const void* V, const void* Qg,
+                            const void* Kg, const void* Vg, const uint8_t* d_mask, const int32_t* q_idx,
+                            const int32_t* n_routed, const int32_t* prefix, void* O, void* S_save, void* A_c,
+                            float* lse_loc, float* lse_glb, void* fwd_ws, size_t fwd_ws_bytes, void* stream);
+l2a_status l2a_backward_sets(const l2a_params* p, const void* Q, const void* K, const void* V, const void* Qg,
+                             const void* Kg, const void* Vg, const uint8_t* d_mask, const int32_t* q_idx,
+                             const int32_t* n_routed, const int32_t* prefix, const void* dO, const void* S_save,
+                             const void* A_c, const float* lse_loc, const float* lse_glb, void* dQ, void* dK, void* dV,
+                             void* dQg, void* dKg, void* dVg, float* dgate, void* bwd_ws, size_t bwd_ws_bytes,
+                             void* stream);
 
 /*
  * l2a_backward with a separate gradient for the local output.  o_t = s_t + d_t a_t, but s_t also feeds the

@@ -1,6 +1,6 @@
 """Builds libl2a.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
 
-Usage: python -m paper_2603_17484_b200.build [--force] [--verbose]
+Usage: python -m paper_2603_17484_b200.build [--force] [--verbose] [--debug]
 """
 from __future__ import annotations
 
@@ -12,6 +12,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libl2a.so")
+LIB_DEBUG = os.path.join(HERE, "libl2a_debug.so")   # same sources with -DL2A_DEBUG (index checks; used by one GPU test)
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 
 NVCC_FLAGS = [
@@ -24,23 +25,26 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def stale() -> bool:
-    if not os.path.exists(LIB):
+def stale(lib=LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(INCLUDE, "*.h"))
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_lib(force: bool = False, verbose: bool = False) -> str:
-    if not force and not stale():
-        return LIB
+def build_lib(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    lib = LIB_DEBUG if debug else LIB
+    if not force and not stale(lib):
+        return lib
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")]
     if verbose:
         flags += ["-Xptxas", "-v"]
+    if debug:
+        flags += ["-DL2A_DEBUG"]
     objs = []
-    objdir = os.path.join(HERE, "build")
+    objdir = os.path.join(HERE, "build_debug" if debug else "build")
     os.makedirs(objdir, exist_ok=True)
     procs = []
     for src in sources():
@@ -56,12 +60,12 @@ def build_lib(force: bool = False, verbose: bool = False) -> str:
         failed |= pr.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    tmp = LIB + f".{os.getpid()}.tmp"
+    tmp = lib + f".{os.getpid()}.tmp"
     subprocess.check_call([nvcc, "-shared", "-cudart", "shared", "-o", tmp, *objs,
                            "-Xlinker", "-rpath=/usr/local/cuda/lib64"])
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build_lib(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build_lib(force="--force" in sys.argv, verbose="--verbose" in sys.argv, debug="--debug" in sys.argv))

@@ -536,6 +536,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
       tc_fence_before();
       mbar_arrive(&bar->u_free);       // the values are in registers: dP^T(i+1) may overwrite the columns
       float* dst = acc_prev + warp * (8 * D) + lane * 4;
+      if (acc_prev == nullptr) return true;     // (debug build: the item's indices were out of range and are reported)
 #pragma unroll
       for (int c = 0; c < D / 16; ++c) {
         const int k = sub + 4 * c;
@@ -559,7 +560,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
       }
       const bool masked = st_flags[q] != 0;
       const int item_glb = st_flags[4], item_row0 = st_flags[5], item_h = st_flags[6];
-      float* acc_cur = (item_glb ? a.dq_acc_glb : a.dq_acc_loc) +
+      const bool item_ok = dbg_in_range(item_row0 >= 0 && (item_row0 >> 7) < n_tiles && item_h >= 0 && item_h < a.Hq &&
+                                        (item_glb ? a.dq_acc_glb : a.dq_acc_loc) != nullptr, a.status);
+      float* acc_cur = !item_ok ? nullptr : (item_glb ? a.dq_acc_glb : a.dq_acc_loc) +
                        (((int64_t)b * a.Hq + item_h) * n_tiles + (item_row0 >> 7)) * (int64_t)(kTileM * D);
       // the previous item's dQ leaves TMEM while this item's scores are still being computed
       if (i > 0 && !drain(i - 1)) { ok = false; break; }
@@ -705,7 +708,7 @@ __global__ void __launch_bounds__(256) dq_merge_kernel(const float* __restrict__
                                                        const uint8_t* __restrict__ d_mask,
                                                        const int32_t* __restrict__ prefix, bf16* __restrict__ dQ, int B,
                                                        int L, int Hq, float scale, int64_t bs, int64_t ts,
-                                                       int tile_begin, int tile_count) {
+                                                       int tile_begin, int tile_count, int* status) {
   constexpr int kChunks = D / 8;             // 16-byte chunks per bf16 row
   constexpr int kRowBytes = D * 2 + 16;      // padded: conflict-free 16-byte accesses down a column
   __shared__ __align__(16) uint8_t tile_s[kTileM * kRowBytes];
@@ -727,6 +730,7 @@ __global__ void __launch_bounds__(256) dq_merge_kernel(const float* __restrict__
     }
     if (acc_glb && d_mask[(int64_t)b * L + t]) {
       const int cr = prefix[(int64_t)b * (L + 1) + t];
+      if (!dbg_in_range(cr >= 0 && cr < n_tiles * kTileM, status)) continue;
       const float4* p = reinterpret_cast<const float4*>(
           acc_glb + (((int64_t)b * Hq + h) * n_tiles + (cr >> 7)) * tile_floats + (q * 4 + ((cr & 127) >> 5)) * (8 * D) +
           c * 128 + (cr & 31) * 4);
@@ -806,7 +810,7 @@ cudaError_t launch_bwd(const BwdArgs& base, const CUtensorMap& mapQ, const CUten
     if (t1 > t0)
       dq_merge_kernel<D><<<(unsigned)((t1 - t0) * base.B * base.Hq), 256, 0, s>>>(
           base.dq_acc_loc, base.dq_acc_glb, d_mask, base.prefix, base.dQ, base.B, base.Lq, base.Hq, base.scale,
-          base.dq_st.b, base.dq_st.t, t0, t1 - t0);
+          base.dq_st.b, base.dq_st.t, t0, t1 - t0, base.status);
     phase_events().mark(s);
   }
   return cudaGetLastError();
@@ -831,12 +835,53 @@ extern "C" l2a_status l2a_backward(const l2a_params* p, const void* Q, const voi
                             dV, dgate, bwd_ws, bwd_ws_bytes, stream);
 }
 
+static l2a_status backward_impl(const l2a_params* p, const void* Q, const void* K, const void* V,
+                                const uint8_t* d_mask, const int32_t* q_idx, const int32_t* n_routed,
+                                const int32_t* prefix, const void* dO, const void* dS_loc, const void* S_save,
+                                const void* A_c, const float* lse_loc, const float* lse_glb, void* dQ, void* dK,
+                                void* dV, float* dgate, void* bwd_ws, size_t bwd_ws_bytes, void* stream,
+                                bool clear_status);
+
 extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, const void* K, const void* V,
                                          const uint8_t* d_mask, const int32_t* q_idx, const int32_t* n_routed,
                                          const int32_t* prefix, const void* dO, const void* dS_loc,
                                          const void* S_save, const void* A_c, const float* lse_loc,
                                          const float* lse_glb, void* dQ, void* dK, void* dV, float* dgate,
                                          void* bwd_ws, size_t bwd_ws_bytes, void* stream) {
+  return backward_impl(p, Q, K, V, d_mask, q_idx, n_routed, prefix, dO, dS_loc, S_save, A_c, lse_loc, lse_glb, dQ, dK,
+                       dV, dgate, bwd_ws, bwd_ws_bytes, stream, true);
+}
+
+// Section 3.1: in the paper's layer Global Attention has its own projections of the local output, i.e. its own
+// Q/K/V.  One call for both modules: the local module's backward on (Q, K, V), the global module's on (Qg, Kg, Vg).
+extern "C" l2a_status l2a_backward_sets(const l2a_params* p, const void* Q, const void* K, const void* V, const void* Qg,
+                                        const void* Kg, const void* Vg, const uint8_t* d_mask, const int32_t* q_idx,
+                                        const int32_t* n_routed, const int32_t* prefix, const void* dO,
+                                        const void* S_save, const void* A_c, const float* lse_loc, const float* lse_glb,
+                                        void* dQ, void* dK, void* dV, void* dQg, void* dKg, void* dVg, float* dgate,
+                                        void* bwd_ws, size_t bwd_ws_bytes, void* stream) {
+  if (!p) return L2A_ERR_INVALID_ARG;
+  if (!Qg && !Kg && !Vg)     // one set feeds both modules
+    return l2a_backward(p, Q, K, V, d_mask, q_idx, n_routed, prefix, dO, S_save, A_c, lse_loc, lse_glb, dQ, dK, dV, dgate,
+                        bwd_ws, bwd_ws_bytes, stream);
+  if (!Qg || !Kg || !Vg || !dQg || !dKg || !dVg) return L2A_ERR_INVALID_ARG;
+  if (p->flags & (L2A_FLAG_SKIP_LOCAL | L2A_FLAG_SKIP_GLOBAL | L2A_FLAG_FORCE_ALL_GLOBAL)) return L2A_ERR_INVALID_ARG;
+  l2a_params q = *p;
+  q.flags = (p->flags & ~L2A_FLAG_SHARED_WINDOW) | L2A_FLAG_SKIP_GLOBAL;
+  l2a_status st = backward_impl(&q, Q, K, V, nullptr, nullptr, nullptr, nullptr, dO, dO, S_save, nullptr, lse_loc, nullptr,
+                                dQ, dK, dV, nullptr, bwd_ws, bwd_ws_bytes, stream, true);
+  if (st != L2A_OK) return st;
+  q.flags = (p->flags & ~L2A_FLAG_SHARED_WINDOW) | L2A_FLAG_SKIP_LOCAL;
+  return backward_impl(&q, Qg, Kg, Vg, d_mask, q_idx, n_routed, prefix, dO, dO, nullptr, A_c, nullptr, lse_glb, dQg, dKg,
+                       dVg, dgate, bwd_ws, bwd_ws_bytes, stream, false);
+}
+
+static l2a_status backward_impl(const l2a_params* p, const void* Q, const void* K, const void* V,
+                                const uint8_t* d_mask, const int32_t* q_idx, const int32_t* n_routed,
+                                const int32_t* prefix, const void* dO, const void* dS_loc, const void* S_save,
+                                const void* A_c, const float* lse_loc, const float* lse_glb, void* dQ, void* dK,
+                                void* dV, float* dgate, void* bwd_ws, size_t bwd_ws_bytes, void* stream,
+                                bool clear_status) {
   if (!p) return L2A_ERR_INVALID_ARG;
   if (!dS_loc || !aligned16(dS_loc)) return L2A_ERR_INVALID_ARG;
   size_t need = 0;
@@ -855,7 +900,7 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   if (!bwd_ws || (reinterpret_cast<uintptr_t>(bwd_ws) % 256) != 0 || bwd_ws_bytes < need) return L2A_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   uint8_t* ws = static_cast<uint8_t*>(bwd_ws);
-  if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, s) != cudaSuccess) return L2A_ERR_CUDA;
+  if (clear_status && cudaMemsetAsync(ws, 0, kWsHeaderBytes, s) != cudaSuccess) return L2A_ERR_CUDA;
   bf16* Qc = reinterpret_cast<bf16*>(ws + kWsHeaderBytes);
   bf16* dOc = reinterpret_cast<bf16*>(ws + kWsHeaderBytes + rows_bytes(p));
   float* delta_loc = reinterpret_cast<float*>(ws + kWsHeaderBytes + 2 * rows_bytes(p));
@@ -886,10 +931,10 @@ extern "C" l2a_status l2a_backward_split(const l2a_params* p, const void* Q, con
   pe.mark(s);
   if (!skip_global) {
     if (launch_gather_rows(static_cast<const bf16*>(Q), Qc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s, nullptr, 0,
-                           0, qs) != cudaSuccess)
+                           0, qs, reinterpret_cast<int*>(ws)) != cudaSuccess)
       return L2A_ERR_CUDA;
     if (launch_gather_rows(static_cast<const bf16*>(dO), dOc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s, nullptr,
-                           0, 0, os) != cudaSuccess)
+                           0, 0, os, reinterpret_cast<int*>(ws)) != cudaSuccess)
       return L2A_ERR_CUDA;
   }
   pe.mark(s);

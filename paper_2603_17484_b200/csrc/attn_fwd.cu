@@ -439,7 +439,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
           }
           bf16* dst1 = nullptr;   // row-indexed destination (s rows, or compact a rows)
           bf16* dst2 = nullptr;   // position-indexed destination
-          if (valid) {
+          if (valid && dbg_in_range(row >= 0 && row < a.Lq && seq_row >= 0 && seq_row < a.Lq, a.status)) {
             if (a.out) dst1 = a.out + b * a.out_st.b + row * a.out_st.t + (int64_t)h * D + hf * (D / 2);
             if (a.out2 && (a.combine_mask == nullptr || a.combine_mask[(int64_t)b * a.Lq + seq_row]))
               dst2 = a.out2 + b * a.out2_st.b + seq_row * a.out2_st.t + (int64_t)h * D + hf * (D / 2);

@@ -103,7 +103,11 @@ using namespace l2a;
 
 extern "C" {
 
-const char* l2a_version(void) { return "l2a-b200 0.1 (sm_100a; tcgen05/TMEM/TMA)"; }
+#ifdef L2A_DEBUG
+const char* l2a_version(void) { return "l2a-b200 0.2 (sm_100a; tcgen05/TMEM/TMA; debug build: index checks on)"; }
+#else
+const char* l2a_version(void) { return "l2a-b200 0.2 (sm_100a; tcgen05/TMEM/TMA)"; }
+#endif
 
 const char* l2a_status_string(l2a_status s) {
   switch (s) {
@@ -113,6 +117,7 @@ const char* l2a_status_string(l2a_status s) {
     case L2A_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case L2A_ERR_CUDA: return "CUDA call failed";
     case L2A_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    case L2A_ERR_DEVICE_BOUNDS: return "an index derived from the routing arrays was out of range (debug build)";
   }
   return "unknown status";
 }
@@ -168,7 +173,7 @@ l2a_status l2a_workspace_status(const void* ws, void* stream) {
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (cudaMemcpyAsync(&word, ws, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return L2A_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return L2A_ERR_CUDA;
-  return word == 0 ? L2A_OK : L2A_ERR_DEVICE_TIMEOUT;
+  return word == 0 ? L2A_OK : word == 4 ? L2A_ERR_DEVICE_BOUNDS : L2A_ERR_DEVICE_TIMEOUT;
 }
 
 l2a_status l2a_route_compact(const l2a_params* p, const void* router, int router_kind, float logit_threshold,
@@ -217,6 +222,28 @@ l2a_status l2a_forward(const l2a_params* p, const void* Q, const void* K, const 
                        void* A_c, float* lse_loc, float* lse_glb, void* fwd_ws, size_t fwd_ws_bytes, void* stream) {
   return forward_range(p, Q, K, V, d_mask, q_idx, n_routed, prefix, O, S_save, A_c, lse_loc, lse_glb, fwd_ws,
                        fwd_ws_bytes, stream, 0, -1, true);
+}
+
+// Section 3.1: Global Attention with its own Q/K/V (its own projections of the local output).  Local phase on
+// (Q, K, V), then the global phase of the routed rows on (Qg, Kg, Vg), added into O.
+l2a_status l2a_forward_sets(const l2a_params* p, const void* Q, const void* K, const void* V, const void* Qg,
+                            const void* Kg, const void* Vg, const uint8_t* d_mask, const int32_t* q_idx,
+                            const int32_t* n_routed, const int32_t* prefix, void* O, void* S_save, void* A_c,
+                            float* lse_loc, float* lse_glb, void* fwd_ws, size_t fwd_ws_bytes, void* stream) {
+  if (!p) return L2A_ERR_INVALID_ARG;
+  if (!Qg && !Kg && !Vg)
+    return l2a_forward(p, Q, K, V, d_mask, q_idx, n_routed, prefix, O, S_save, A_c, lse_loc, lse_glb, fwd_ws, fwd_ws_bytes,
+                       stream);
+  if (!Qg || !Kg || !Vg) return L2A_ERR_INVALID_ARG;
+  if (p->flags & (L2A_FLAG_SKIP_LOCAL | L2A_FLAG_SKIP_GLOBAL | L2A_FLAG_GLOBAL_PHASE)) return L2A_ERR_INVALID_ARG;
+  l2a_params q = *p;
+  q.flags = (p->flags & ~(L2A_FLAG_SHARED_WINDOW | L2A_FLAG_FORCE_ALL_GLOBAL)) | L2A_FLAG_SKIP_GLOBAL;
+  l2a_status st = forward_range(&q, Q, K, V, d_mask, q_idx, n_routed, prefix, O, S_save, A_c, lse_loc, lse_glb, fwd_ws,
+                                fwd_ws_bytes, stream, 0, -1, true);
+  if (st != L2A_OK) return st;
+  q.flags = (p->flags & ~L2A_FLAG_SHARED_WINDOW) | L2A_FLAG_GLOBAL_PHASE;
+  return forward_range(&q, Qg, Kg, Vg, d_mask, q_idx, n_routed, prefix, O, S_save, A_c, lse_loc, lse_glb, fwd_ws,
+                       fwd_ws_bytes, stream, 0, -1, false);
 }
 
 static l2a_status forward_range(const l2a_params* p, const void* Q, const void* K, const void* V,
@@ -294,7 +321,7 @@ static l2a_status forward_range(const l2a_params* p, const void* Q, const void* 
   if (!skip_global && !force_all) {
     // consolidate routed query rows (Algorithm 1, step 1); independent of the local pass
     if (launch_gather_rows(static_cast<const bf16*>(Q), Qc, q_idx, n_routed, p->B, p->Lq, p->Hq * p->D, s,
-                           row_range ? prefix : nullptr, row_begin, row_end, qs) != cudaSuccess)
+                           row_range ? prefix : nullptr, row_begin, row_end, qs, status) != cudaSuccess)
       return L2A_ERR_CUDA;
   }
   pe.mark(s);

@@ -18,6 +18,18 @@ constexpr int kTileN = 128;         // keys per KV block
 constexpr int kRowsPerCta = 256;    // two query tiles per CTA in the forward / dQ kernels
 constexpr size_t kWsHeaderBytes = 256;  // every workspace starts with a header; word 0 = status
 
+// Debug build (-DL2A_DEBUG): every index derived from q_idx / prefix / tile metadata is checked against the tensor
+// extent before it is used for a store; a violation sets the workspace status word to 4 (l2a_workspace_status then
+// returns L2A_ERR_DEVICE_BOUNDS) and the store is skipped -- nothing traps.  In the normal build the check folds away.
+#ifdef L2A_DEBUG
+__device__ __forceinline__ bool dbg_in_range(bool ok, int* status) {
+  if (!ok && status != nullptr) atomicExch(status, 4);
+  return ok;
+}
+#else
+__device__ __forceinline__ bool dbg_in_range(bool, int*) { return true; }
+#endif
+
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -68,7 +80,8 @@ cudaError_t launch_route_compact(const RouteArgs& a, cudaStream_t stream);
 // routed rows t in [row_begin, row_end) are gathered (the padding with the range that ends at L).
 cudaError_t launch_gather_rows(const bf16* src, bf16* dst, const int32_t* q_idx, const int32_t* n_routed,
                                int B, int L, int row_elems, cudaStream_t stream, const int32_t* prefix = nullptr,
-                               int row_begin = 0, int row_end = 0, RowStrides src_strides = RowStrides{0, 0});
+                               int row_begin = 0, int row_end = 0, RowStrides src_strides = RowStrides{0, 0},
+                               int* status = nullptr);   // status: workspace status word (debug-build index checks)
 
 // z[b,t] = w . S[b,t,:] + bias (fp32 accumulation); optional sum over t of sigmoid(z)^2 per batch entry
 cudaError_t launch_router_logits(const bf16* S, const float* w, float bias, float* logits, float* sum_sq, int B,

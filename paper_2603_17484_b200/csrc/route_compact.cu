@@ -125,7 +125,7 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const bf16* __restrict
                                                           int row_chunks /* 16-byte chunks per row */,
                                                           const int32_t* __restrict__ prefix, int row_begin,
                                                           int row_end, int64_t src_batch_chunks,
-                                                          int64_t src_row_chunks) {
+                                                          int64_t src_row_chunks, int* status) {
   const int b = blockIdx.y;
   const int n_c = n_routed[b];
   int n_pad = (n_c + kRowsPerCta - 1) / kRowsPerCta * kRowsPerCta;
@@ -142,6 +142,7 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const bf16* __restrict
   for (int c = c_begin + blockIdx.x; c < n_pad; c += gridDim.x) {
     if (c < n_c) {
       const int t = q_idx[(int64_t)b * L + c];
+      if (!dbg_in_range(t >= 0 && t < L, status)) continue;
       for (int i = threadIdx.x; i < row_chunks; i += blockDim.x)
         d[(int64_t)c * row_chunks + i] = __ldg(&s[t * src_row_chunks + i]);
     } else {
@@ -244,14 +245,14 @@ cudaError_t launch_route_compact(const RouteArgs& a, cudaStream_t stream) {
 
 cudaError_t launch_gather_rows(const bf16* src, bf16* dst, const int32_t* q_idx, const int32_t* n_routed, int B,
                                int L, int row_elems, cudaStream_t stream, const int32_t* prefix, int row_begin,
-                               int row_end, RowStrides src_strides) {
+                               int row_end, RowStrides src_strides, int* status) {
   const int row_chunks = row_elems * 2 / 16;
   const int64_t ts = src_strides.t > 0 ? src_strides.t : row_elems;
   const int64_t bs = src_strides.b > 0 ? src_strides.b : (int64_t)L * ts;
   int gx = L < 148 * 16 ? L : 148 * 16;
   dim3 grid(gx, B);
   gather_rows_kernel<<<grid, 256, 0, stream>>>(src, dst, q_idx, n_routed, L, row_chunks, prefix, row_begin, row_end,
-                                               bs / 8, ts / 8);
+                                               bs / 8, ts / 8, status);
   return cudaGetLastError();
 }
 

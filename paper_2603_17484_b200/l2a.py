@@ -31,6 +31,7 @@ EXPORTS = (
     "l2a_route_compact", "l2a_forward", "l2a_backward", "l2a_step_host", "l2a_profile_next_call",
     "l2a_route_compact_static", "l2a_router_logits", "l2a_decode_workspace_bytes", "l2a_decode",
     "l2a_backward_split", "l2a_router_backward", "l2a_forward_routed", "l2a_selftest_wait_timeout",
+    "l2a_forward_sets", "l2a_backward_sets",
 )
 
 
@@ -198,6 +199,33 @@ def l2a_backward(p, Q, K, V, d_mask, q_idx, n_routed, prefix, dO, S_save, A_c, l
     return code
 
 
+def _nbytes(t):
+    return ctypes.c_size_t(t.numel() * t.element_size() if t is not None else 0)
+
+
+def l2a_forward_sets(p, Q, K, V, Qg, Kg, Vg, d_mask, q_idx, n_routed, prefix, O, S_save, A_c, lse_loc, lse_glb, fwd_ws,
+                     stream=None, check=True) -> int:
+    """l2a_forward with a second Q/K/V set for the Global Attention module (None, None, None = one set)."""
+    code = lib().l2a_forward_sets(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(Qg), _ptr(Kg), _ptr(Vg), _ptr(d_mask),
+                                  _ptr(q_idx), _ptr(n_routed), _ptr(prefix), _ptr(O), _ptr(S_save), _ptr(A_c),
+                                  _ptr(lse_loc), _ptr(lse_glb), _ptr(fwd_ws), _nbytes(fwd_ws), _stream(stream))
+    if check:
+        _check(code, "l2a_forward_sets")
+    return code
+
+
+def l2a_backward_sets(p, Q, K, V, Qg, Kg, Vg, d_mask, q_idx, n_routed, prefix, dO, S_save, A_c, lse_loc, lse_glb, dQ, dK,
+                      dV, dQg, dKg, dVg, dgate, bwd_ws, stream=None, check=True) -> int:
+    """l2a_backward with a second Q/K/V set: gradients of the local module's set and of the global module's set."""
+    code = lib().l2a_backward_sets(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(Qg), _ptr(Kg), _ptr(Vg),
+                                   _ptr(d_mask), _ptr(q_idx), _ptr(n_routed), _ptr(prefix), _ptr(dO), _ptr(S_save),
+                                   _ptr(A_c), _ptr(lse_loc), _ptr(lse_glb), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dQg),
+                                   _ptr(dKg), _ptr(dVg), _ptr(dgate), _ptr(bwd_ws), _nbytes(bwd_ws), _stream(stream))
+    if check:
+        _check(code, "l2a_backward_sets")
+    return code
+
+
 def l2a_backward_split(p, Q, K, V, d_mask, q_idx, n_routed, prefix, dO, dS_loc, S_save, A_c, lse_loc, lse_glb, dQ,
                        dK, dV, dgate, bwd_ws, stream=None, check=True) -> int:
     """l2a_backward with a separate gradient dS_loc for the local output (dO + the router path)."""
@@ -304,35 +332,64 @@ class Buffers:
     fwd_ws: torch.Tensor = None
     bwd_ws: torch.Tensor = None
 
+    GUARD_BYTES = 4096
+    GUARD_BYTE = 0xA5
+
     @staticmethod
-    def allocate(p: L2AParams, backward: bool = False, device="cuda", router_dtype=torch.uint8) -> "Buffers":
+    def allocate(p: L2AParams, backward: bool = False, device="cuda", router_dtype=torch.uint8,
+                 guard: bool = False) -> "Buffers":
+        """guard: every tensor sits between two 4 KB regions filled with a byte pattern; check_guards() tells whether a
+        kernel wrote outside a buffer (the stand-in for a memory checker in the GPU tests)."""
         B, Lq, Lk, Hq, Hkv, D = p.B, p.Lq, p.Lk, p.Hq, p.Hkv, p.D
         bf, dev = torch.bfloat16, device
         r, f, w = l2a_workspace_bytes(p)
         b = Buffers(p)
-        b.Q = torch.empty((B, Lq, Hq, D), dtype=bf, device=dev)
-        b.K = torch.empty((B, Lk, Hkv, D), dtype=bf, device=dev)
-        b.V = torch.empty((B, Lk, Hkv, D), dtype=bf, device=dev)
-        b.router = torch.empty((B, Lq), dtype=router_dtype, device=dev)
-        b.d_mask = torch.empty((B, Lq), dtype=torch.uint8, device=dev)
-        b.q_idx = torch.empty((B, Lq), dtype=torch.int32, device=dev)
-        b.n_routed = torch.empty((B,), dtype=torch.int32, device=dev)
-        b.prefix = torch.empty((B, Lq + 1), dtype=torch.int32, device=dev)
-        b.O = torch.empty((B, Lq, Hq, D), dtype=bf, device=dev)
-        b.route_ws = torch.empty((r,), dtype=torch.uint8, device=dev)
-        b.fwd_ws = torch.empty((f,), dtype=torch.uint8, device=dev)
+        b._raw = []
+        G = Buffers.GUARD_BYTES
+
+        def new(shape, dtype):
+            if not guard:
+                return torch.empty(shape, dtype=dtype, device=dev)
+            n = 1
+            for x in shape:
+                n *= x
+            nbytes = n * torch.empty((), dtype=dtype).element_size()
+            pad = (-nbytes) % 256                                  # the back guard starts right after the last byte
+            raw = torch.full((G + nbytes + pad + G,), Buffers.GUARD_BYTE, dtype=torch.uint8, device=dev)
+            b._raw.append((raw, nbytes))
+            return raw[G:G + nbytes].view(dtype).view(shape)
+
+        b.Q = new((B, Lq, Hq, D), bf)
+        b.K = new((B, Lk, Hkv, D), bf)
+        b.V = new((B, Lk, Hkv, D), bf)
+        b.router = new((B, Lq), router_dtype)
+        b.d_mask = new((B, Lq), torch.uint8)
+        b.q_idx = new((B, Lq), torch.int32)
+        b.n_routed = new((B,), torch.int32)
+        b.prefix = new((B, Lq + 1), torch.int32)
+        b.O = new((B, Lq, Hq, D), bf)
+        b.route_ws = new((r,), torch.uint8)
+        b.fwd_ws = new((f,), torch.uint8)
         if backward:
-            b.S_save = torch.empty((B, Lq, Hq, D), dtype=bf, device=dev)
-            b.A_c = torch.empty((B, Lq, Hq, D), dtype=bf, device=dev)
-            b.lse_loc = torch.empty((B, Hq, Lq), dtype=torch.float32, device=dev)
-            b.lse_glb = torch.empty((B, Hq, Lq), dtype=torch.float32, device=dev)
-            b.dO = torch.empty((B, Lq, Hq, D), dtype=bf, device=dev)
-            b.dQ = torch.empty((B, Lq, Hq, D), dtype=bf, device=dev)
-            b.dK = torch.empty((B, Lk, Hkv, D), dtype=bf, device=dev)
-            b.dV = torch.empty((B, Lk, Hkv, D), dtype=bf, device=dev)
-            b.dgate = torch.empty((B, Lq), dtype=torch.float32, device=dev)
-            b.bwd_ws = torch.empty((w,), dtype=torch.uint8, device=dev)
+            b.S_save = new((B, Lq, Hq, D), bf)
+            b.A_c = new((B, Lq, Hq, D), bf)
+            b.lse_loc = new((B, Hq, Lq), torch.float32)
+            b.lse_glb = new((B, Hq, Lq), torch.float32)
+            b.dO = new((B, Lq, Hq, D), bf)
+            b.dQ = new((B, Lq, Hq, D), bf)
+            b.dK = new((B, Lk, Hkv, D), bf)
+            b.dV = new((B, Lk, Hkv, D), bf)
+            b.dgate = new((B, Lq), torch.float32)
+            b.bwd_ws = new((w,), torch.uint8)
         return b
+
+    def check_guards(self) -> bool:
+        """True if no guard byte around any buffer changed (always True without guard=True)."""
+        G = Buffers.GUARD_BYTES
+        for raw, nbytes in getattr(self, "_raw", []):
+            if not bool((raw[:G] == Buffers.GUARD_BYTE).all()) or not bool((raw[G + nbytes:] == Buffers.GUARD_BYTE).all()):
+                return False
+        return True
 
     def route(self, router_kind=ROUTER_MASK_U8, threshold=0.0, stream=None):
         return l2a_route_compact(self.p, self.router, router_kind, threshold, self.d_mask, self.q_idx,

@@ -72,7 +72,8 @@ class Case:
         self.d = np.ascontiguousarray(d, dtype=np.uint8)
         fl = flags | (l2a.FLAG_SAVE_FOR_BWD if backward else 0)
         self.p = l2a.params(B, Lq, Lk, Hq, Hkv, D, W, softmax_scale=scale, flags=fl)
-        self.buf = l2a.Buffers.allocate(self.p, backward=backward,
+        # every buffer between pattern-filled guards: a write outside a tensor or workspace fails the test
+        self.buf = l2a.Buffers.allocate(self.p, backward=backward, guard=True,
                                         router_dtype=torch.float32 if logits is not None else torch.uint8)
         self.buf.Q.copy_(t["Q"]); self.buf.K.copy_(t["K"]); self.buf.V.copy_(t["V"])
         if backward:
@@ -96,6 +97,7 @@ class Case:
         b.forward()
         torch.cuda.synchronize()
         assert l2a.l2a_workspace_status(b.fwd_ws) == 0, "device-side wait timed out in the forward"
+        assert b.check_guards(), "the forward wrote outside a buffer"
         return b
 
     def check_routing(self):
@@ -133,6 +135,7 @@ def run_backward(case: "Case", with_dgate=True):
     b.backward(with_dgate=with_dgate)
     torch.cuda.synchronize()
     assert l2a.l2a_workspace_status(b.bwd_ws) == 0, "device-side wait timed out in the backward"
+    assert b.check_guards(), "the backward wrote outside a buffer"
     return b
 
 

@@ -6,7 +6,7 @@ import torch
 
 import oracle
 from paper_2603_17484_b200 import l2a, synth
-from tests.gpu_util import Case, check_close, to_f64
+from tests.gpu_util import Case, check_close, check_same_or_rounding, to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -63,3 +63,30 @@ def test_separate_qkv_for_the_global_module():
     # dgate_t = dO_t . a_t with a_t from the global set (Eq. 7)
     want_gate = (to_f64(b.dO) * ref_glb["a"]).sum(axis=(2, 3)) * d
     check_close(b.dgate.cpu().numpy().astype(np.float64), want_gate, "dgate", 2e-2 * np.sqrt(Hq * D), 2e-3 * np.sqrt(Hq * D))
+
+
+    # the same layer through the one-call forms: equal to the sequences above (dQ of either set up to the order of its
+    # fp32 sums), and with no second set they are l2a_forward / l2a_backward
+    two = {k: v.clone() for k, v in dict(O=b.O, S=b.S_save, A=b.A_c, dQ=dQ, dK=dK, dV=dV, dQg=dQg, dKg=dKg, dVg=dVg).items()}
+    p = l2a.params(B, L, L, Hq, Hkv, D, W, flags=flags)
+    for t in (b.O, dQ, dK, dV, dQg, dKg, dVg):
+        t.fill_(float("nan"))
+    l2a.l2a_forward_sets(p, b.Q, b.K, b.V, Qg, Kg, Vg, b.d_mask, b.q_idx, b.n_routed, b.prefix, b.O, b.S_save, b.A_c,
+                         b.lse_loc, b.lse_glb, b.fwd_ws)
+    l2a.l2a_backward_sets(p, b.Q, b.K, b.V, Qg, Kg, Vg, b.d_mask, b.q_idx, b.n_routed, b.prefix, b.dO, b.S_save, b.A_c,
+                          b.lse_loc, b.lse_glb, dQ, dK, dV, dQg, dKg, dVg, b.dgate, b.bwd_ws)
+    torch.cuda.synchronize()
+    assert l2a.l2a_workspace_status(b.fwd_ws) == 0 and l2a.l2a_workspace_status(b.bwd_ws) == 0
+    n = b.n_routed.cpu().numpy()
+    for k, got in dict(O=b.O, S=b.S_save, dK=dK, dV=dV, dKg=dKg, dVg=dVg).items():
+        assert torch.equal(got.view(torch.int16), two[k].view(torch.int16)), k
+    for bi in range(B):
+        assert torch.equal(b.A_c[bi, :n[bi]].view(torch.int16), two["A"][bi, :n[bi]].view(torch.int16))
+    check_same_or_rounding(dQ, two["dQ"], "dQ (local set)")
+    check_same_or_rounding(dQg, two["dQg"], "dQ (global set)")
+    c.run_forward()
+    want_o = b.O.clone()
+    l2a.l2a_forward_sets(c.p, b.Q, b.K, b.V, None, None, None, b.d_mask, b.q_idx, b.n_routed, b.prefix, b.O, b.S_save,
+                         b.A_c, b.lse_loc, b.lse_glb, b.fwd_ws)
+    torch.cuda.synchronize()
+    assert torch.equal(b.O.view(torch.int16), want_o.view(torch.int16))
