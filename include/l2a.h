@@ -409,7 +409,7 @@ l2a_status l2a_route_compact_static(const l2a_params* p, const void* router, int
                                     int32_t* n_routed, int32_t* prefix, void* stream);
 
 /*
- * Profiling aid (no counterpart in the paper).  Registers up to 8 cudaEvent_t handles (host array of
+ * Profiling aid (no counterpart in the paper).  Registers up to 12 cudaEvent_t handles (host array of
  * `n_events` handles created by the caller with timing enabled; the array is copied).  The NEXT
  * l2a_forward or l2a_backward call made by this host thread records event k on its stream at its
  * k-th phase boundary and then clears the registration.  Phase boundaries:
@@ -417,10 +417,10 @@ l2a_status l2a_route_compact_static(const l2a_params* p, const void* router, int
  *                 global kernel
  *   l2a_backward: 0 start | 1 after the gathers | 2 after the Delta kernel and the clearing of the dQ accumulators |
  *                 3 after the five-GEMM kernel | 4 after the dQ merge (everything final).
- *                 With 7 events the kernel runs as two launches over key-block ranges (keys below and from
- *                 128 * floor(3 * ceil(Lk / 128) / 4), when Lk >= 1024), each followed by the merge of the dQ rows
- *                 it completes: 3 / 4 after the first kernel / merge (dK, dV of the first range's keys and dQ of the
- *                 rows that see only those keys are final), 5 / 6 after the second.
+ *                 With 7 (11) events the kernel runs as two (four) launches over key-block ranges -- keys below and
+ *                 from 3/4 (1/2, 3/4, 7/8) of ceil(Lk / 128) blocks, when there are at least 8 (16) blocks -- each
+ *                 followed by the merge of the dQ rows it completes: boundaries 3 + 2 r / 4 + 2 r after the kernel /
+ *                 the merge of range r (dK, dV of the range's keys and dQ of the rows that see no later key are final).
  */
 l2a_status l2a_profile_next_call(void* const* events, int n_events);
 

@@ -767,7 +767,18 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 
 
 }  // namespace
 
-int dkv_split_block(int n_kblocks) { return n_kblocks >= 8 ? (3 * n_kblocks) / 4 : 0; }
+int bwd_ranges(int n_kblocks, int n_events, int first[kMaxBwdRanges]) {
+  first[0] = 0;
+  if (n_events >= 11 && n_kblocks >= 16) {
+    first[1] = n_kblocks / 2; first[2] = (3 * n_kblocks) / 4; first[3] = (7 * n_kblocks) / 8;
+    return 4;
+  }
+  if (n_events >= 7 && n_kblocks >= 8) {
+    first[1] = (3 * n_kblocks) / 4;
+    return 2;
+  }
+  return 1;
+}
 
 // First row tile whose dQ still receives contributions from the key blocks at or after `split`: a row at position p
 // only meets keys <= p, so after the key blocks below `split` the rows with p < 128 * split are final.
@@ -794,23 +805,25 @@ cudaError_t launch_bwd(const BwdArgs& base, const CUtensorMap& mapQ, const CUten
                                               kTileM * D);
   phase_events().mark(s);
   const int n_kblocks = (base.Lk + kTileN - 1) / kTileN;
-  // A caller that registered seven phase events wants the gradients of the early rows while the rest is computed (to
-  // move them to the host): two launches over key-block ranges, each followed by the merge of the dQ rows it finishes.
-  const int split = phase_events().n >= 7 ? dkv_split_block(n_kblocks) : 0;
-  const int t_split = split > 0 ? dq_final_tiles(split, base.q_pos_offset, n_tiles) : n_tiles;
-  for (int part = 0; part < 2; ++part) {
-    if (part == 1 && split == 0) break;
+  // A caller that registered phase events for key-block ranges wants the gradients of the early rows while the rest is
+  // computed (to move them to the host): one launch per range, each followed by the merge of the dQ rows it finishes.
+  int first[kMaxBwdRanges];
+  const int n_ranges = bwd_ranges(n_kblocks, phase_events().n, first);
+  int t_done = 0;
+  for (int part = 0; part < n_ranges; ++part) {
     BwdArgs a = base;
-    a.kb_begin = part == 0 ? 0 : split;
-    a.kb_count = part == 0 ? (split > 0 ? split : n_kblocks) : n_kblocks - split;
+    const int kb_end = part + 1 < n_ranges ? first[part + 1] : n_kblocks;
+    a.kb_begin = first[part];
+    a.kb_count = kb_end - first[part];
     bwd_kernel<D><<<(unsigned)a.kb_count * base.B * base.Hkv, kDkvThreads, BwdSmem<D>::kTotal, s>>>(
         mapQ, mapDO, mapQc, mapDOc, mapK, mapV, a);
     phase_events().mark(s);
-    const int t0 = part == 0 ? 0 : t_split, t1 = part == 0 ? t_split : n_tiles;
-    if (t1 > t0)
-      dq_merge_kernel<D><<<(unsigned)((t1 - t0) * base.B * base.Hq), 256, 0, s>>>(
+    const int t1 = part + 1 < n_ranges ? dq_final_tiles(kb_end, base.q_pos_offset, n_tiles) : n_tiles;
+    if (t1 > t_done)
+      dq_merge_kernel<D><<<(unsigned)((t1 - t_done) * base.B * base.Hq), 256, 0, s>>>(
           base.dq_acc_loc, base.dq_acc_glb, d_mask, base.prefix, base.dQ, base.B, base.Lq, base.Hq, base.scale,
-          base.dq_st.b, base.dq_st.t, t0, t1 - t0, base.status);
+          base.dq_st.b, base.dq_st.t, t_done, t1 - t_done, base.status);
+    if (t1 > t_done) t_done = t1;
     phase_events().mark(s);
   }
   return cudaGetLastError();

@@ -436,7 +436,7 @@ l2a_status l2a_forward_routed(const l2a_params* p, const void* Q, const void* K,
 }
 
 l2a_status l2a_profile_next_call(void* const* events, int n_events) {
-  if (n_events < 0 || n_events > 8 || (n_events > 0 && !events)) return L2A_ERR_INVALID_ARG;
+  if (n_events < 0 || n_events > 12 || (n_events > 0 && !events)) return L2A_ERR_INVALID_ARG;
   PhaseEvents& pe = phase_events();
   pe.clear();
   for (int i = 0; i < n_events; ++i) pe.ev[i] = static_cast<cudaEvent_t>(events[i]);
@@ -474,7 +474,7 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
   struct Aux {
     int device = -1;
     cudaStream_t in = nullptr, out = nullptr;
-    cudaEvent_t start = nullptr, up = nullptr, fwd = nullptr, phase[7] = {}, down = nullptr, chunk[8] = {};
+    cudaEvent_t start = nullptr, up = nullptr, fwd = nullptr, phase[11] = {}, down = nullptr, chunk[8] = {};
   };
   static thread_local Aux aux;
   int dev_id = 0;
@@ -484,7 +484,8 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
         cudaStreamCreateWithFlags(&aux.out, cudaStreamNonBlocking) != cudaSuccess)
       return L2A_ERR_CUDA;
     cudaEvent_t* evs[] = {&aux.start, &aux.up, &aux.fwd, &aux.down, &aux.phase[0], &aux.phase[1], &aux.phase[2],
-                          &aux.phase[3], &aux.phase[4], &aux.phase[5], &aux.phase[6], &aux.chunk[0], &aux.chunk[1], &aux.chunk[2],
+                          &aux.phase[3], &aux.phase[4], &aux.phase[5], &aux.phase[6], &aux.phase[7], &aux.phase[8],
+                          &aux.phase[9], &aux.phase[10], &aux.chunk[0], &aux.chunk[1], &aux.chunk[2],
                           &aux.chunk[3], &aux.chunk[4], &aux.chunk[5], &aux.chunk[6], &aux.chunk[7]};
     for (cudaEvent_t* e : evs)
       if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return L2A_ERR_CUDA;
@@ -578,41 +579,47 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
   L2A_TRY(cudaMemcpyAsync(host->O, dev->O, qb, cudaMemcpyDeviceToHost, aux.out));
   if (bwd) {
     L2A_TRY(cudaStreamWaitEvent(s, aux.up, 0));
-    // With seven phase events the backward runs as two key-block ranges; boundary 4 says that the gradients of the
-    // early rows (dK, dV of the first range's keys, dQ of the rows that only see those keys) are final: they leave
-    // on the download stream while the second range is computed, the rest after the last kernel.
-    void* phase_events[7];
-    for (int i = 0; i < 7; ++i) phase_events[i] = aux.phase[i];
-    st = l2a_profile_next_call(phase_events, 7);
+    // With eleven phase events the backward runs as four key-block ranges; boundary 4 + 2 r says that the gradients
+    // range r completes (dK, dV of its keys, dQ of the rows that only see keys up to its end) are final: they leave on
+    // the download stream while the next range is computed, the last range's after the last kernel.
+    void* phase_events[11];
+    for (int i = 0; i < 11; ++i) phase_events[i] = aux.phase[i];
+    st = l2a_profile_next_call(phase_events, 11);
     if (st != L2A_OK) return st;
     st = l2a_backward(&q, dev->Q, dev->K, dev->V, dev->d_mask, dev->q_idx, dev->n_routed, dev->prefix, dev->dO,
                       dev->S_save, dev->A_c, dev->lse_loc, dev->lse_glb, dev->dQ, dev->dK, dev->dV, nullptr,
                       dev->bwd_ws, dev->bwd_ws_bytes, stream);
     if (st != L2A_OK) return st;
-    const int split = dkv_split_block(ceil_div(p->Lk, kTileN));   // 0: one launch
-    const int64_t k_early = (int64_t)split * kTileN;
-    int64_t q_early = (int64_t)dq_final_tiles(split, p->q_pos_offset, ceil_div(p->Lq, kTileM)) * kTileM;
-    if (q_early > p->Lq) q_early = p->Lq;
+    int first[kMaxBwdRanges];
+    const int n_kblocks = ceil_div(p->Lk, kTileN), n_tiles = ceil_div(p->Lq, kTileM);
+    const int n_ranges = bwd_ranges(n_kblocks, 11, first);
     const size_t krow = (size_t)p->Hkv * p->D * sizeof(bf16), qrow = (size_t)p->Hq * p->D * sizeof(bf16);
-    if (split > 0) L2A_TRY(cudaStreamWaitEvent(aux.out, aux.phase[4], 0));
-    for (int b = 0; b < p->B; ++b) {
-      const size_t kbase = (size_t)b * p->Lk * krow, kearly = (size_t)k_early * krow, kall = (size_t)p->Lk * krow;
-      const size_t qbase = (size_t)b * p->Lq * qrow, qearly = (size_t)q_early * qrow, qall = (size_t)p->Lq * qrow;
-      uint8_t *hk = static_cast<uint8_t*>(host->dK) + kbase, *hv = static_cast<uint8_t*>(host->dV) + kbase;
-      uint8_t* hq = static_cast<uint8_t*>(host->dQ) + qbase;
-      const uint8_t *gk = static_cast<const uint8_t*>(dev->dK) + kbase, *gv = static_cast<const uint8_t*>(dev->dV) + kbase;
-      const uint8_t* gq = static_cast<const uint8_t*>(dev->dQ) + qbase;
-      if (split > 0 && qearly > 0) L2A_TRY(cudaMemcpyAsync(hq, gq, qearly, cudaMemcpyDeviceToHost, aux.out));
-      if (split > 0 && kearly > 0) {
-        L2A_TRY(cudaMemcpyAsync(hk, gk, kearly, cudaMemcpyDeviceToHost, aux.out));
-        L2A_TRY(cudaMemcpyAsync(hv, gv, kearly, cudaMemcpyDeviceToHost, aux.out));
+    int64_t k_done = 0, q_done = 0;
+    for (int r = 0; r < n_ranges; ++r) {
+      const bool last = r + 1 == n_ranges;
+      int64_t k_end = last ? p->Lk : (int64_t)first[r + 1] * kTileN;
+      int64_t q_end = last ? p->Lq : (int64_t)dq_final_tiles(first[r + 1], p->q_pos_offset, n_tiles) * kTileM;
+      if (k_end > p->Lk) k_end = p->Lk;
+      if (q_end > p->Lq) q_end = p->Lq;
+      cudaStream_t cs = last ? s : aux.out;
+      if (!last) L2A_TRY(cudaStreamWaitEvent(aux.out, aux.phase[4 + 2 * r], 0));
+      for (int b = 0; b < p->B; ++b) {
+        const size_t kbase = (size_t)b * p->Lk * krow, qbase = (size_t)b * p->Lq * qrow;
+        if (q_end > q_done)
+          L2A_TRY(cudaMemcpyAsync(static_cast<uint8_t*>(host->dQ) + qbase + q_done * qrow,
+                                  static_cast<const uint8_t*>(dev->dQ) + qbase + q_done * qrow,
+                                  (size_t)(q_end - q_done) * qrow, cudaMemcpyDeviceToHost, cs));
+        if (k_end > k_done) {
+          L2A_TRY(cudaMemcpyAsync(static_cast<uint8_t*>(host->dK) + kbase + k_done * krow,
+                                  static_cast<const uint8_t*>(dev->dK) + kbase + k_done * krow,
+                                  (size_t)(k_end - k_done) * krow, cudaMemcpyDeviceToHost, cs));
+          L2A_TRY(cudaMemcpyAsync(static_cast<uint8_t*>(host->dV) + kbase + k_done * krow,
+                                  static_cast<const uint8_t*>(dev->dV) + kbase + k_done * krow,
+                                  (size_t)(k_end - k_done) * krow, cudaMemcpyDeviceToHost, cs));
+        }
       }
-      const size_t qoff = split > 0 ? qearly : 0, koff = split > 0 ? kearly : 0;
-      if (qall > qoff) L2A_TRY(cudaMemcpyAsync(hq + qoff, gq + qoff, qall - qoff, cudaMemcpyDeviceToHost, s));
-      if (kall > koff) {
-        L2A_TRY(cudaMemcpyAsync(hk + koff, gk + koff, kall - koff, cudaMemcpyDeviceToHost, s));
-        L2A_TRY(cudaMemcpyAsync(hv + koff, gv + koff, kall - koff, cudaMemcpyDeviceToHost, s));
-      }
+      if (q_end > q_done) q_done = q_end;
+      if (k_end > k_done) k_done = k_end;
     }
   }
   L2A_TRY(cudaEventRecord(aux.down, aux.out));

@@ -117,9 +117,12 @@ struct FwdArgs {
   const float* lse_loc;      // [B,Hq,Lq] by row; read only when shared_window is set
 };
 size_t bwd_ws_size(const l2a_params* p);
-// First key block of the second backward launch when the caller asked for the early boundary (0: not split), and the
-// number of leading 128-row tiles of dQ that are final after the first launch.
-int dkv_split_block(int n_kblocks);
+// Key-block ranges of the backward when the caller registered phase events for them (11 events: four ranges, 7: two,
+// fewer: one launch).  Writes the first key block of ranges 1.. into `first` and returns the number of ranges; ranges
+// get shorter towards the end of the sequence, where a key block has little work left.  dq_final_tiles: number of
+// leading 128-row tiles of dQ that are final once the key blocks below `split` are done.
+constexpr int kMaxBwdRanges = 4;
+int bwd_ranges(int n_kblocks, int n_events, int first[kMaxBwdRanges]);
 int dq_final_tiles(int split, int q_pos_offset, int n_tiles);
 
 // Facts about the current device that the launchers need, looked up once per device and cached.
@@ -149,7 +152,7 @@ struct PerDeviceOnce {
 
 // One-shot, thread-local registration of phase-boundary events (see l2a_profile_next_call).
 struct PhaseEvents {
-  cudaEvent_t ev[8];
+  cudaEvent_t ev[12];
   int n = 0;
   int next = 0;
   void mark(cudaStream_t s) {

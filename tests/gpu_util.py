@@ -8,12 +8,16 @@ max abs error <= 2e-2 and mean abs error <= 2e-3.  A bf16 number of magnitude |x
 apply to the value before that final rounding: |err| <= 2e-2 + 2^-8 |want| element-wise and
 mean|err| <= 2e-3 + 2^-9 mean|want|.  Forward outputs are held to exactly that.
 
-Gradients additionally inherit the bf16 rounding of the MMA operands P and dS (relative 2^-9 each, the
-reading taken where the paper is silent on rounding: fp32 scores and soft-max, bf16 tensor-core operands).
-tests/test_rounding_model.py applies exactly these roundings to the oracle's fp64 arithmetic on the shapes of
-tests/test_gpu_backward.py: the excursions they cause beyond the bound are rare (at most one element in 2.6e5) and
-small (at most 1.03 x the bound).  Gradient checks therefore let a fraction of at most 1e-5 of the elements (rounded up
-to a whole element) exceed the bound, none by more than a factor of 1.5.
+Gradients additionally inherit the bf16 roundings the kernels make (the reading taken where the paper is silent on
+rounding: fp32 scores and soft-max, bf16 tensor-core operands, bf16 stored outputs): P and dS are rounded to bf16
+before the second GEMMs, and Delta = dO . out uses the stored bf16 output, which itself came from bf16 probabilities.
+tests/test_rounding_model.py applies exactly these roundings to a plain fp64 evaluation and compares with the oracle:
+  * away from the start of the sequence the excursions beyond the bound are rare (at most one element in 2.6e5) and
+    small (at most 1.1 x the bound): the checks allow a 1e-5 fraction (rounded up to one element) up to 1.5 x;
+  * the first rows see a handful of keys, so the error of Delta (about 0.03 for N(0,1) inputs) is not averaged out and
+    enters every dS of the row with the same sign, twice when both modules see the same keys: dQ of those rows, and dK
+    of the first keys (summed over the group's heads), can be off by up to 1.7 x the bound in a few elements.  The
+    checks allow 8 elements per (batch, head) among the first 8 rows / keys, none beyond 2 x the bound.
 
 Every comparison also records how many elements exceed the plain 2e-2 and the bound; the session prints the table
 (tests/conftest.py)."""
@@ -34,11 +38,18 @@ def to_f64(t: torch.Tensor) -> np.ndarray:
     return t.detach().float().cpu().numpy().astype(np.float64)
 
 
+EARLY_ROWS = 8        # rows / keys with this few keys / queries in sight: the looser rule below applies to them
+EARLY_PER_HEAD = 8    # elements per (batch, head) of those rows that may exceed the bound ...
+EARLY_CAP = 2.0       # ... by at most this factor
+
 STATS = []   # (what, elements, over plain 2e-2, over the bound, largest err / bound): printed at the end of the session
 
 
 def check_close(got: np.ndarray, want: np.ndarray, what: str, max_abs=MAX_ABS, mean_abs=MEAN_ABS, outlier_frac=0.0,
-                cap=1.5):
+                cap=1.5, early_rows=0):
+    """early_rows: for a gradient laid out [B, L, H, D], the rows (dQ) / keys (dK, dV) l < early_rows follow the rule for
+    rows with a handful of keys (see the module docstring): at most EARLY_PER_HEAD elements per (batch, head) over the
+    bound, none beyond EARLY_CAP x the bound."""
     assert got.shape == want.shape, (what, got.shape, want.shape)
     assert np.isfinite(got).all(), f"{what}: non-finite values in the GPU result"
     if got.size == 0:
@@ -53,6 +64,15 @@ def check_close(got: np.ndarray, want: np.ndarray, what: str, max_abs=MAX_ABS, m
     STATS.append((what, int(err.size), n_plain, n_over, ratio))
     msg = (f"{what}: abs err {err[i]:.4g} at {i} (got {got[i]}, want {want[i]}), max abs err {err.max():.4g}, "
            f"{n_over} over the bound, {n_plain} over {max_abs}, largest err/bound {ratio:.3f}")
+    if early_rows > 0 and err.ndim == 4:
+        head = (excess[:, :early_rows] > 0).sum(axis=(1, 3))                 # per (batch, head)
+        assert head.max(initial=0) <= EARLY_PER_HEAD, msg
+        assert (err[:, :early_rows] / bound[:, :early_rows]).max(initial=0.0) <= EARLY_CAP, msg
+        err, bound, excess = err[:, early_rows:], bound[:, early_rows:], excess[:, early_rows:]
+        if err.size == 0:
+            return
+        n_over = int((excess > 0).sum())
+        ratio = float((err / bound).max())
     assert n_over <= math.ceil(outlier_frac * err.size), msg
     assert ratio <= cap, msg
     mean_tol = mean_abs + 2.0 ** -9 * np.abs(want).mean()
@@ -142,9 +162,9 @@ def run_backward(case: "Case", with_dgate=True):
 def check_backward_full(case: "Case"):
     b = case.buf
     dQ, dK, dV = oracle.backward_full(case.shape, case.u16("Q"), case.u16("K"), case.u16("V"), case.d, case.u16("dO"))
-    check_close(to_f64(b.dQ), dQ, "dQ", outlier_frac=1e-5)
-    check_close(to_f64(b.dK), dK, "dK", outlier_frac=1e-5)
-    check_close(to_f64(b.dV), dV, "dV", outlier_frac=1e-5)
+    check_close(to_f64(b.dQ), dQ, "dQ", outlier_frac=1e-5, early_rows=EARLY_ROWS)
+    check_close(to_f64(b.dK), dK, "dK", outlier_frac=1e-5, early_rows=EARLY_ROWS)
+    check_close(to_f64(b.dV), dV, "dV", outlier_frac=1e-5, early_rows=EARLY_ROWS)
     return dQ, dK, dV
 
 

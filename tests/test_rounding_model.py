@@ -9,8 +9,11 @@ the CUDA path or the C oracle) on shapes of tests/test_gpu_backward.py and compa
   * without the roundings the evaluation equals the oracle to 1e-12 (so the model is the same function);
   * with them, some elements leave the plain bound 2e-2 (large dK / dV entries cannot even be stored that accurately),
     which is why the bound carries the 2^-8 |want| term;
-  * against 2e-2 + 2^-8 |want| the excursions are rare and small: at most one element per array here, never beyond
-    1.1 x the bound.  tests/gpu_util.py allows a 1e-5 fraction (at least one element) up to 1.5 x the bound.
+  * against 2e-2 + 2^-8 |want|, rows and keys beyond the first eight have rare, small excursions (at most one element per
+    array, never beyond 1.1 x the bound; tests/gpu_util.py allows a 1e-5 fraction up to 1.5 x);
+  * the first eight rows / keys, which see a handful of keys / are seen through rows with a handful of keys, can exceed
+    the bound in a few elements per head (the error of Delta is not averaged out there), by at most 1.7 x here;
+    tests/gpu_util.py allows 8 elements per (batch, head) up to 2 x.
 """
 import math
 
@@ -58,7 +61,9 @@ def backward_model(B, Lq, Lk, Hq, Hkv, D, W, d, t, rounded):
                 l = e.sum(axis=1, keepdims=True)
                 l[l == 0] = 1.0
                 p = e / l
-                delta = (do * rnd(p @ v)).sum(axis=1, keepdims=True)     # Delta from the stored (bf16) output
+                # the forward's output: probabilities rounded to bf16 before P V, normalised by the fp32 row sum,
+                # stored as bf16; Delta is formed from that stored output
+                delta = (do * rnd((rnd(e) @ v) / l)).sum(axis=1, keepdims=True)
                 pb = rnd(p)
                 ds = rnd(pb * (do @ v.T - delta)) * rows
                 dV[b, :, g] += pb.T @ (do * rows)
@@ -66,6 +71,8 @@ def backward_model(B, Lq, Lk, Hq, Hkv, D, W, d, t, rounded):
                 dQ[b, :, h] += scale * (ds @ k)
     return rnd(dQ), rnd(dK), rnd(dV)
 
+
+EARLY = 8     # the first rows / keys, treated separately (tests/gpu_util.EARLY_ROWS)
 
 CASES = [
     (1, 1024, 1024, 1, 1, 64, 128, 0.2),
@@ -90,10 +97,37 @@ def test_operand_roundings_explain_the_gradient_tolerance(B, Lq, Lk, Hq, Hkv, D,
         err = np.abs(g - w)
         bound = 2e-2 + 2.0 ** -8 * np.abs(w)
         over_plain += int((err > 2e-2).sum())
-        n_over = int((err > bound).sum())
-        assert n_over <= 1, (name, n_over)                              # the GPU tests allow ceil(1e-5 * size) >= 1
-        assert (err / bound).max() <= 1.1, (name, (err / bound).max())  # the GPU tests allow 1.5
+        late, late_b = err[:, EARLY:], bound[:, EARLY:]
+        if late.size:
+            assert int((late > late_b).sum()) <= 1, name                  # the GPU tests allow ceil(1e-5 * size) >= 1
+            assert (late / late_b).max() <= 1.1, (name, (late / late_b).max())  # the GPU tests allow 1.5
+        early = (err[:, :EARLY] > bound[:, :EARLY]).sum(axis=(1, 3))
+        assert early.max() <= 6, (name, early)                            # the GPU tests allow 8 per (batch, head)
+        assert (err[:, :EARLY] / bound[:, :EARLY]).max() <= 1.7, name     # the GPU tests allow 2
         assert err.mean() <= 0.5 * (2e-3 + 2.0 ** -9 * np.abs(w).mean()), (name, err.mean())
     if (B, Lq) == (2, 513):
         # large dK / dV entries of early keys (sums over ~2000 rows) cannot be stored in bf16 to within 2e-2
         assert over_plain > 0
+
+
+def test_first_rows_exceed_the_bound_only_slightly():
+    """All tokens routed, four query heads per KV head: the configuration in which the error of Delta adds up most (both
+    modules see the same few keys; dK sums the heads).  Over 40 seeds the excursions stay within the first rows / keys,
+    at most five elements per head, at most 1.7 x the bound -- and they do occur, so the looser rule is needed."""
+    B, Lq, Lk, Hq, Hkv, D, W = 1, 64, 64, 4, 1, 128, 16
+    seen = 0
+    for sd in range(40):
+        d = np.ones((B, Lq), np.uint8)
+        t = synth.qkv(B, Lq, Hq, Hkv, D, 5000 + sd, with_dO=True, Lk=Lk)
+        sh = oracle.Shape(B, Lq, Lk, Hq, Hkv, D, W)
+        want = oracle.backward_full(sh, *(synth.as_u16(t[k]) for k in ("Q", "K", "V")), d, synth.as_u16(t["dO"]))
+        got = backward_model(B, Lq, Lk, Hq, Hkv, D, W, d, t, rounded=True)
+        for g, w in zip(got, want):
+            err = np.abs(g - w)
+            bound = 2e-2 + 2.0 ** -8 * np.abs(w)
+            over = err > bound
+            seen += int(over.sum())
+            assert not over[:, EARLY:].any()
+            assert over[:, :EARLY].sum(axis=(1, 3)).max() <= 6
+            assert (err / bound).max() <= 1.7
+    assert seen > 0
