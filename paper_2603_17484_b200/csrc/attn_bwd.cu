@@ -180,9 +180,17 @@ struct BwdArgs {
 //   warps 0-15 : compute.  Warp w owns TMEM lanes 32*(w%4)..+31 (its thread's key, or query row of dQ) and the
 //                32 score columns of quarter w/4, so that 16 warps hide each other's TMEM and MUFU latency.
 //   warp 16    : TMA producer          warp 17 : tcgen05 MMA issuer, TMEM owner
-//   warp 18    : stages the row statistics of each query tile
+//   warp 18    : stages the row statistics of each query tile          warp 19 : idle
+//   warps 20-27: read every dQ(i) tile out of TMEM (one lane group and one half of the columns each) and add it into the
+//                fp32 accumulators: the reductions leave an SM at about 32 bytes per clock, and a warp that issues them
+//                stalls that long, so they are kept off the warps whose progress the tensor pipe waits for
+// Registers: 896 threads start with 72 each (64512 in all, which is also all that setmaxnreg can redistribute: an
+// increase is served from what the CTA's own warps released); the service warpgroup goes down to 40, the read-out
+// warpgroups to 56, the compute warpgroups up to 88.
 constexpr int kComputeWarps = 16;
-constexpr int kDkvThreads = (kComputeWarps + 3) * 32;   // 608
+constexpr int kDkvThreads = 28 * 32;   // 896
+template <int N> __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
 __device__ __forceinline__ float bf16lo_to_f32(uint32_t packed) { return __uint_as_float(packed << 16); }
 __device__ __forceinline__ float bf16hi_to_f32(uint32_t packed) { return __uint_as_float(packed & 0xffff0000u); }
@@ -241,9 +249,9 @@ struct ItemCursor {
 //         then dQ(i).
 //   Shared memory: K, V resident; Q and dO in two-stage rings; dS(i) (bf16, [key][query], swizzled like a TMA
 //   tile) -- the A operand of both dK += dS^T Q (read K-major) and dQ = dS K (read MN-major).
-//   MMA order per item i:  dK(i-1) | dV(i) | dQ(i) | S^T(i+1) | dP^T(i+1).  Two loops run through the order with
-//   slack: T: S^T -> P -> dV -> S^T and U: dP^T -> dS -> dQ -> read-out -> dP^T; dK(i-1) fills the pipe while the
-//   exponentials of item i run.
+//   MMA order per item i:  dV(i) | dQ(i) | S^T(i+1) | dK(i) | dP^T(i+1).  Two loops run through the order with
+//   slack: T: S^T -> P -> dV -> S^T and U: dP^T -> dS -> dQ -> read-out -> dP^T; dK(i) keeps the pipe busy while the
+//   read-out warps take dQ(i) out of TMEM and the compute warps start on item i+1.
 template <int D>
 struct BwdSmem {
   static constexpr int kTileBytes = 128 * D * 2;
@@ -326,7 +334,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
     mbar_init(&bar->ds_full, kComputeWarps * 32);    // dS(i) is in shared memory and dP^T(i) has been read
     mbar_init(&bar->ds_free, 1);                     // dQ(i) and dK(i) have consumed dS(i)
     mbar_init(&bar->dq_full, 1);                     // dQ(i) is in TMEM
-    mbar_init(&bar->u_free, kComputeWarps * 32);     // dQ(i) has been read out: the columns may take dP^T(i+1)
+    mbar_init(&bar->u_free, 8 * 32);     // dQ(i) has been read out: the columns may take dP^T(i+1)
     mbar_init(&bar->final_bar, 1);
     bar->abort_flag = 0;
     fence_mbar_init();
@@ -345,8 +353,55 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
     return;
   }
 
-  if (warp == 16) {
+  // register shares by warpgroup: every warp of a warpgroup executes the same setmaxnreg at the top of its role
+  if (warp >= 20) {
+    // ------------------------------------------------------------------ dQ read-out: TMEM -> fp32 accumulators
+    setmaxnreg_dec<56>();
+    // lane == query row of the item's tile; this warp owns the 32 rows of its lane group and one half of the D columns,
+    // taken 32 at a time: each 32 x 4 piece is one 512-byte reduction (accumulator layout: see above)
+    const int grp = warp & 3, half = (warp - 20) >> 2;
+    const uint32_t lane_base = static_cast<uint32_t>(grp * 32) << 16;
+    const int n_tiles = (a.Lq + kTileM - 1) / kTileM;
+    constexpr int kChunks = D / 32;     // read out 32 columns at a time: one TMEM load, eight reductions
+    constexpr int kCols = D / 4;        // columns per quarter in the accumulator layout
+    ItemCursor cur(plan, g * G);
+    for (int i = 0; i < plan.total; ++i) {
+      const int h = cur.h, glb = cur.glb(), tile = cur.tile();
+      cur.next();
+      float* acc = glb ? a.dq_acc_glb : a.dq_acc_loc;
+      const bool item_ok = dbg_in_range(tile >= 0 && tile < n_tiles && h >= 0 && h < a.Hq && acc != nullptr, a.status);
+      acc += (((int64_t)b * a.Hq + h) * n_tiles + tile) * (int64_t)(kTileM * D) + lane * 4;
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->dq_full, i & 1, abort_flag))) break;
+      tc_fence_after();
+#pragma unroll
+      for (int cc = 0; cc < kChunks / 2; ++cc) {
+        const int ch = half * (kChunks / 2) + cc;
+        uint32_t v[32];
+        tmem_ld32(tmem + lane_base + 384 + ch * 32, v);
+        tmem_ld_wait();
+        if (cc == kChunks / 2 - 1) {
+          tc_fence_before();
+          mbar_arrive(&bar->u_free);       // everything is in registers: dP^T(i+1) may overwrite the columns
+        }
+        if (item_ok) {
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            // columns 32 ch + 4 c .. + 3: quarter (32 ch + 4 c) / kCols, piece ((32 ch + 4 c) % kCols) / 4
+            const int col = 32 * ch + 4 * c;
+            float* dst = acc + ((col / kCols) * 4 + grp) * (8 * D) + ((col % kCols) / 4) * 128;
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(__uint_as_float(v[4 * c])),
+                         "f"(__uint_as_float(v[4 * c + 1])), "f"(__uint_as_float(v[4 * c + 2])),
+                         "f"(__uint_as_float(v[4 * c + 3]))
+                         : "memory");
+          }
+        }
+      }
+    }
+  } else if (warp == 19) {
+    setmaxnreg_dec<40>();     // idle
+  } else if (warp == 16) {
     // ------------------------------------------------------------------ TMA producer
+    setmaxnreg_dec<40>();
     if (lane == 0) {
       tma_prefetch_desc(&mapQ); tma_prefetch_desc(&mapDO); tma_prefetch_desc(&mapQc); tma_prefetch_desc(&mapDOc);
       mbar_expect_tx(&bar->kv_full, 2 * SM::kTileBytes);
@@ -369,6 +424,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
     __syncwarp();
   } else if (warp == 18) {
     // ------------------------------------------------------------------ row statistics of each item
+    setmaxnreg_dec<40>();
     // lse * log2(e) and Delta of the item's 128 query rows, plus per-quarter mask flags, go to shared memory.
     // The global loads of item i+1 are issued before waiting for its slot, so their latency is hidden.
     float r_lse[4], r_delta[4];
@@ -419,6 +475,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
   } else if (warp == 17) {
     // ------------------------------------------------------------------ MMA issuer
     // (whole warp runs the loop; only the tcgen05 instructions are predicated on lane 0)
+    setmaxnreg_dec<40>();
     {
       const uint32_t leader = (lane == 0);
       constexpr uint32_t tmem = 0;   // checked above: TMEM operand addresses are immediates in this loop
@@ -485,7 +542,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
       }
       for (int i = 0; ok && i < plan.total; ++i) {
         const bool more = i + 1 < plan.total;
-        if (i > 0) issue_dK((i - 1) & 1, i == 1);     // its dS was waited for before dQ(i-1)
         if (!mbar_spin_warp(&bar->p_full, i & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         issue_dV(i & 1, i == 0);
@@ -493,12 +549,15 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
         tc_fence_after();
         issue_dQ();
         if (more) {
+          // S^T(i+1) overwrites P^T(i): dV(i) precedes it in issue order
+          if (!mbar_spin_warp(&bar->q_full[(i + 1) & 1], ((i + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          issue_S((i + 1) & 1);
+        }
+        issue_dK(i & 1, i == 0);       // keeps the pipe busy while dQ(i) is read out
+        if (more) {
           const int sn = (i + 1) & 1;
           const uint32_t phn = ((i + 1) >> 1) & 1;
-          // S^T(i+1) overwrites P^T(i): dV(i) precedes it in issue order
-          if (!mbar_spin_warp(&bar->q_full[sn], phn, abort_flag)) { ok = false; break; }
-          tc_fence_after();
-          issue_S(sn);
           // dP^T(i+1) overwrites dQ(i): wait for its read-out
           if (!mbar_spin_warp(&bar->u_free, i & 1, abort_flag) ||
               !mbar_spin_warp(&bar->do_full[sn], phn, abort_flag)) { ok = false; break; }
@@ -506,46 +565,19 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
           issue_dP(sn);
         }
       }
-      if (ok) {
-        issue_dK((plan.total - 1) & 1, plan.total == 1);
-        tc_commit(&bar->final_bar, leader);
-      }
+      if (ok) tc_commit(&bar->final_bar, leader);
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------------ P^T, dS, dQ read-out and epilogue
+    // ------------------------------------------------------------------ P^T, dS and epilogue
+    setmaxnreg_inc<88>();
     const int q = warp >> 2;                           // query-column quarter of this warp
     const int kr = (warp & 3) * 32 + lane;             // key inside the block == TMEM lane
     const int kp = k0 + kr;
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const uint32_t s_addr = tmem + lane_base + 256 + q * 32;
     const uint32_t dp_addr = tmem + lane_base + 384 + q * 32;
-    constexpr int kCols = D / 4;                       // dQ columns per quarter: 32 (D = 128) or 16 (D = 64)
-    const uint32_t dq_addr = tmem + lane_base + 384 + ((q * kCols) & ~31);
-    const int sub = (D == 64) ? (q & 1) * 16 : 0;
-    const int n_tiles = (a.Lq + kTileM - 1) / kTileM;
-    float* acc_prev = nullptr;                         // accumulator block of the previous item's query tile
     bool ok = true;
-    // dQ(i) read-out: lane == query row; each warp adds its 32 rows x D/4 columns as D/16 pieces of 512 bytes
-    auto drain = [&](int i_prev) -> bool {
-      if (!__all_sync(0xffffffffu, mbar_wait(&bar->dq_full, i_prev & 1, abort_flag))) return false;
-      tc_fence_after();
-      uint32_t v[32];
-      tmem_ld32(dq_addr, v);
-      tmem_ld_wait();
-      tc_fence_before();
-      mbar_arrive(&bar->u_free);       // the values are in registers: dP^T(i+1) may overwrite the columns
-      float* dst = acc_prev + warp * (8 * D) + lane * 4;
-      if (acc_prev == nullptr) return true;     // (debug build: the item's indices were out of range and are reported)
-#pragma unroll
-      for (int c = 0; c < D / 16; ++c) {
-        const int k = sub + 4 * c;
-        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + c * 128), "f"(__uint_as_float(v[k])),
-                     "f"(__uint_as_float(v[k + 1])), "f"(__uint_as_float(v[k + 2])), "f"(__uint_as_float(v[k + 3]))
-                     : "memory");
-      }
-      return true;
-    };
     for (int i = 0; i < plan.total; ++i) {
       const int s = i & 1;
       // this item's row statistics go to registers before the scores are waited for
@@ -559,14 +591,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
         st[4 * c] = v.x; st[4 * c + 1] = v.y; st[4 * c + 2] = v.z; st[4 * c + 3] = v.w;
       }
       const bool masked = st_flags[q] != 0;
-      const int item_glb = st_flags[4], item_row0 = st_flags[5], item_h = st_flags[6];
-      const bool item_ok = dbg_in_range(item_row0 >= 0 && (item_row0 >> 7) < n_tiles && item_h >= 0 && item_h < a.Hq &&
-                                        (item_glb ? a.dq_acc_glb : a.dq_acc_loc) != nullptr, a.status);
-      float* acc_cur = !item_ok ? nullptr : (item_glb ? a.dq_acc_glb : a.dq_acc_loc) +
-                       (((int64_t)b * a.Hq + item_h) * n_tiles + (item_row0 >> 7)) * (int64_t)(kTileM * D);
-      // the previous item's dQ leaves TMEM while this item's scores are still being computed
-      if (i > 0 && !drain(i - 1)) { ok = false; break; }
-      acc_prev = acc_cur;
+      const int item_glb = st_flags[4], item_row0 = st_flags[5];
       if (!__all_sync(0xffffffffu, mbar_wait(&bar->s_full, i & 1, abort_flag))) { ok = false; break; }
       tc_fence_after();
       uint32_t pp[16];
@@ -645,7 +670,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
       tc_fence_before();         // orders the dP^T read above before the dQ MMA that overwrites those columns
       mbar_arrive(&bar->ds_full);
     }
-    if (ok && plan.total > 0 && !drain(plan.total - 1)) ok = false;
     // epilogue: quarters 0,1 store the two column halves of dV, quarters 2,3 those of dK
     if (ok && __all_sync(0xffffffffu, mbar_wait(&bar->final_bar, 0, abort_flag))) {
       tc_fence_after();
