@@ -385,6 +385,22 @@ def main():
         pw = int(sum((np.minimum(x, cfg.W) + 1).sum() for x in t))
         return pl, pg, pw
 
+    def issued_pairs(mask, shared):
+        """Score elements the tensor cores really compute: every (128-row tile, 128-key block) pair a launch issues
+        MMAs for counts whole (edge blocks are masked after the product, ragged tiles are padded with zero rows)."""
+        T = 128
+        loc = glb = 0
+        for b in range(cfg.B):
+            r0 = np.arange(0, cfg.L, T, dtype=np.int64)
+            r1 = np.minimum(r0 + T, cfg.L) - 1
+            loc += int((r1 // T - np.maximum(r0 - cfg.W, 0) // T + 1).sum())
+            t = np.nonzero(mask[b])[0].astype(np.int64)
+            if len(t):
+                last = t[np.minimum(np.arange(T - 1, len(t) + T - 1, T), len(t) - 1)]      # last row of each compact tile
+                bound = last - (cfg.W + 1 if shared else 0)
+                glb += int((bound[bound >= 0] // T + 1).sum())
+        return loc * T * T, glb * T * T
+
     def step(profile=None):
         buf.route(kind, 0.0)
         if profile is not None:
@@ -508,6 +524,8 @@ def main():
     tensor_phases = {k: v for k, v in phase_ms.items() if k in kernel_pairs}
     dom = max(tensor_phases, key=tensor_phases.get)
     per, credited, visited = kernel_pairs[dom]
+    il, ig = issued_pairs(d, shared_now)
+    issued = {"attn_fwd_local": il, "attn_fwd_global": ig, "bwd": il + ig}[dom]
     achieved = per * HD * credited / phase_ms[dom] / 1e9
     achieved_visited = per * HD * visited / phase_ms[dom] / 1e9
     # DRAM traffic of the dominant kernel: not captured on this workload (a counter capture of a 12 GB, 100 ms launch is
@@ -528,7 +546,9 @@ def main():
                 "peak_kind": f"sustained bf16 GEMM, {peaks['source']}", "launch_ms": phase_ms[dom],
                 "algorithmic_flops_per_launch": per * HD * credited, "pairs_credited": int(credited),
                 "pairs_visited": int(visited), "achieved_visited": achieved_visited,
-                "frac_visited": achieved_visited / peaks["sustained"]}
+                "frac_visited": achieved_visited / peaks["sustained"],
+                # executed MMA work, tile-granular (masked elements of edge blocks and padding rows included)
+                "pairs_issued": int(issued), "executed_tflops": per * HD * issued / phase_ms[dom] / 1e9}
 
     cpu = None
     if args.cpu_rows > 0 and world == 1:
