@@ -108,6 +108,8 @@ def make_workload(args, seed_offset=0):
     seed = synth.seed_for(idx, int(round(rho * 10))) + replicas.rank_seed_offset(seed_offset)
     if args.routing:
         cfg = synth.Config(**{**cfg.__dict__, "routing": args.routing})
+    if getattr(args, "kv_heads", None):       # a slice of the workload: the first KV heads and their query heads
+        cfg = synth.Config(**{**cfg.__dict__, "Hkv": args.kv_heads, "Hq": args.kv_heads * (cfg.Hq // cfg.Hkv)})
     d, logits = synth.routing(cfg, seed, density=rho)
     return cfg, rho, seed, d, logits
 
@@ -314,6 +316,9 @@ def main():
     ap.add_argument("--density", type=float, default=None)
     ap.add_argument("--routing", default=None, choices=[None, "bernoulli", "clustered", "all", "none"])
     ap.add_argument("--forward-only", action="store_true")
+    ap.add_argument("--kv-heads", type=int, default=None,
+                    help="run a slice of the workload with this many KV heads (and their query heads): small enough "
+                         "for counter captures at the full sequence length")
     ap.add_argument("--shared-window", action=argparse.BooleanOptionalAction, default=False,
                     help="L2A_FLAG_SHARED_WINDOW for the headline run (default off: in the paper's layer the two modules "
                          "have their own Q/K/V; the fusion is only valid when one set feeds both, and is reported as a "

@@ -4,8 +4,8 @@ Only the tests, the smoke check and the benchmark's CPU-baseline leg may import 
 It shares no code with the CUDA library and never imports it.
 
 ``l2a_oracle.c`` holds the plain definition (Eq. 2-5, masks of Section 2, textbook VJP);
-``alg1.py`` holds an independent transcription of Algorithm 1 (tiled, online softmax) that the
-tests require to equal the plain definition.
+``chunked.py`` evaluates the same attention as a running soft-max over arbitrary key chunks (the evaluation order of
+Algorithm 1); the tests require it to equal the plain definition for any chunking.
 """
 from .binding import (  # noqa: F401
     Shape,

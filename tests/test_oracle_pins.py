@@ -7,7 +7,7 @@ import numpy as np
 import pytest
 
 import oracle
-from oracle.alg1 import l2a_alg1_forward
+from oracle.chunked import attend_chunked
 from tests.brute import bf16_bits_to_f64, f64_to_bf16_bits, layer_brute
 
 RNG = np.random.default_rng(1234)
@@ -81,20 +81,35 @@ def test_custom_scale_and_offset():
     np.testing.assert_allclose(got["o"], ref["o"], rtol=0, atol=1e-12)
 
 
-def test_algorithm1_equals_definition():
-    # independent tiled / online-softmax transcription, ragged tiles on both axes
+def test_running_softmax_over_any_chunking_equals_definition():
+    # Algorithm 1's evaluation order (key chunks, carried maximum / sum / values, early stop at the chunk of the
+    # group's last position) for uniform, ragged and random chunkings and row groupings, against the two-pass oracle
     rng = np.random.default_rng(5)
-    for n, D, Bq, Bk, rho in [(37, 8, 4, 4, 0.5), (64, 4, 4, 8, 0.2), (50, 8, 7, 5, 1.0), (30, 8, 4, 4, 0.05)]:
+    for n, D, rows_per_group, chunking, rho in [(37, 8, 4, 4, 0.5), (64, 4, 4, 8, 0.2), (50, 8, 7, 5, 1.0),
+                                                (30, 8, 4, 4, 0.05), (61, 8, 5, "random", 0.4), (48, 4, 48, 1, 0.3)]:
         Q, K, V, d = make(1, n, 1, 1, D, rng=rng, density=rho)
         d[0, 3] = 1
-        sh = oracle.Shape(1, n, n, 1, 1, D, 4)
-        got = oracle.forward_full(sh, Q, K, V, d)
+        W = 4
+        got = oracle.forward_full(oracle.Shape(1, n, n, 1, 1, D, W), Q, K, V, d)
         q_idx, n_c, _ = oracle.compact(d)
-        O, O_c, L_c = l2a_alg1_forward(bf16_bits_to_f64(Q)[0, :, 0], bf16_bits_to_f64(K)[0, :, 0],
-                                       bf16_bits_to_f64(V)[0, :, 0], q_idx[0, :n_c[0]], Bq, Bk)
-        np.testing.assert_allclose(O, got["a"][0, :, 0], rtol=0, atol=1e-12)
-        np.testing.assert_allclose(L_c, got["lse_glb"][0, 0, q_idx[0, :n_c[0]]], rtol=0, atol=1e-12)
-        assert (O[~d[0].astype(bool)] == 0).all()
+        idx = q_idx[0, :n_c[0]]
+        q, k, v = (bf16_bits_to_f64(x)[0, :, 0] for x in (Q, K, V))
+        if chunking == "random":
+            cuts = np.sort(rng.choice(np.arange(1, n), size=9, replace=False))
+            bounds = [0, *cuts.tolist(), n]
+        else:
+            bounds = list(range(0, n, chunking)) + [n]
+        for g0 in range(0, len(idx), rows_per_group):       # routed rows, grouped as a compact tile would be
+            rows = idx[g0:g0 + rows_per_group]
+            out, lse, visited = attend_chunked(q[rows], k, v, rows, bounds)
+            np.testing.assert_allclose(out, got["a"][0, rows, 0], rtol=0, atol=1e-12)
+            np.testing.assert_allclose(lse, got["lse_glb"][0, 0, rows], rtol=0, atol=1e-12)
+            assert visited == np.searchsorted(bounds, rows.max(), side="right")    # no chunk after the last position
+        for g0 in range(0, n, rows_per_group):              # all rows with the window bound: the local module
+            rows = np.arange(g0, min(g0 + rows_per_group, n))
+            out, lse, _ = attend_chunked(q[rows], k, v, rows, bounds, lowest=rows - W)
+            np.testing.assert_allclose(out, got["s"][0, rows, 0], rtol=0, atol=1e-12)
+            np.testing.assert_allclose(lse, got["lse_loc"][0, 0, rows], rtol=0, atol=1e-12)
 
 
 # ---------------------------------------------------------------- closed forms
