@@ -9,12 +9,11 @@
 //          the compact output O_c and log-sum-exp L_c.
 //
 // Structure (per CTA: two 128-row query tiles of one head, sharing the K/V stream):
-//   warps 0-15      : soft-max + correction + epilogue.  Warpgroup 2t+hf (4 warps) owns the 64 score columns of
-//                     half hf of tile t; the two threads that share a query row exchange their row maxima (and,
-//                     at the end, their row sums) through shared memory.  Sixteen warps hide each other's TMEM
-//                     and special-function latency.
-//   warp 16         : TMA producer (Q once; K and V blocks through 2-stage rings)
-//   warp 17         : tcgen05 MMA issuer and TMEM owner
+//   warps 0-7       : soft-max + correction + epilogue.  Warpgroup t (4 warps) owns tile t; one thread per query
+//                     row (= TMEM lane) holds the row's 128 scores of a key block in registers, so the row maximum
+//                     and the row sum need no exchange between threads.
+//   warp 8          : TMA producer (Q once; K and V blocks through 2-stage rings)
+//   warp 9          : tcgen05 MMA issuer and TMEM owner
 //   TMEM (512 cols) : S0 | S1 | O0 | O1 (fp32); the bf16 probabilities P overwrite the first half
 //                     of their own S columns and are consumed from TMEM as the A operand of P*V.
 // While one tile's soft-max runs on the CUDA cores, the tensor core works on the other tile.
@@ -29,8 +28,13 @@ namespace {
 
 constexpr int kNumTiles = 2;
 constexpr int kStages = 2;
-constexpr int kSoftmaxWarps = 16;
-constexpr int kFwdThreads = (kSoftmaxWarps + 2) * 32;   // 576
+constexpr int kSoftmaxWarps = 8;
+constexpr int kTmaWarp = kSoftmaxWarps, kMmaWarp = kSoftmaxWarps + 1;
+// Twelve warps start with 168 registers each (warps are allocated four at a time, so ten would cost the same); the
+// warpgroup of the TMA, MMA and two idle warps hands most of its share to the soft-max warps.
+constexpr int kFwdThreads = (kSoftmaxWarps + 4) * 32;   // 384
+constexpr int kSoftmaxRegs = 216, kOtherRegs = 72;
+static_assert(kSoftmaxWarps * kSoftmaxRegs + 4 * kOtherRegs <= (kSoftmaxWarps + 4) * 168, "register shares exceed the launch allocation");
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
 template <int D>
@@ -42,8 +46,7 @@ struct FwdSmem {
   static constexpr int kKOff = kQOff + kNumTiles * kQTileBytes;
   static constexpr int kVOff = kKOff + kStages * kKVTileBytes;
   static constexpr int kBarOff = kVOff + kStages * kKVTileBytes;
-  static constexpr int kXchOff = kBarOff + 256;                 // row-statistics exchange: [2][tile][half][128] fp32
-  static constexpr int kTotal = kXchOff + 2 * kNumTiles * 2 * kTileM * 4 + 1024 /* alignment slack */;
+  static constexpr int kTotal = kBarOff + 256 + 1024 /* alignment slack */;
 };
 
 struct Barriers {
@@ -52,7 +55,6 @@ struct Barriers {
   uint64_t v_full[kStages], v_empty[kStages];
   uint64_t s_full[kNumTiles];
   uint64_t p_full[kNumTiles];
-  uint64_t xch[kNumTiles];     // the two halves of a tile meet here after publishing their row maxima
   uint64_t o_final;
   uint32_t tmem_base;
   int abort_flag;
@@ -137,8 +139,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     for (int t = 0; t < kNumTiles; ++t) {
       mbar_init(&bar->q_full[t], 1);
       mbar_init(&bar->s_full[t], 1);
-      mbar_init(&bar->p_full[t], 2 * kTileM);
-      mbar_init(&bar->xch[t], 2 * kTileM);
+      mbar_init(&bar->p_full[t], kTileM);
     }
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&bar->k_full[s], 1);
@@ -150,7 +151,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     bar->abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 17) {
+  if (warp == kMmaWarp) {
     tmem_alloc(&bar->tmem_base, 512);
     tmem_relinquish();
   }
@@ -162,13 +163,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     // all 512 columns were requested, so the allocation must start at column 0; the MMA warp relies on it to
     // keep its TMEM operand addresses compile-time constants
     __syncthreads();
-    if (warp == 17) tmem_dealloc(tmem, 512);
+    if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
     if (tid == 0) atomicExch(a.status, 3);
     return;
   }
 
-  if (warp == 16) {
+  if (warp == kTmaWarp) {
     // =========================================================================== TMA producer
+    setmaxnreg_dec<kOtherRegs>();
     if (lane == 0) {
       tma_prefetch_desc(&mapQ);
       tma_prefetch_desc(&mapK);
@@ -190,8 +192,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       }
     }
     __syncwarp();
-  } else if (warp == 17) {
+  } else if (warp == kMmaWarp) {
     // =========================================================================== MMA issuer
+    setmaxnreg_dec<kOtherRegs>();
     // The whole warp runs this loop (uniform control flow keeps the descriptor arithmetic in uniform registers);
     // only the tcgen05 instructions themselves are predicated on lane 0.  Operand descriptors are built once per
     // tile / stage and advanced by compile-time constants, so that issuing stays well under the 64 clocks one
@@ -289,15 +292,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       if (ok) tc_commit(&bar->o_final, leader);
     }
     __syncwarp();
+  } else if (warp > kMmaWarp) {
+    setmaxnreg_dec<kOtherRegs>();     // idle warps of the fourth warpgroup
   } else {
     // =========================================================================== soft-max warpgroups
-    const int t = warp >> 3;                 // tile of this warpgroup
-    const int hf = (warp >> 2) & 1;          // which 64 score columns (and which half of the output columns)
+    setmaxnreg_inc<kSoftmaxRegs>();
+    const int t = warp >> 2;                 // tile of this warpgroup
     const int r = (warp & 3) * 32 + lane;    // row inside the tile == TMEM lane
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    const uint32_t s_addr = tmem + lane_base + t * kTileN + hf * 64;        // this thread's 64 score columns
-    const uint32_t o_addr = tmem + lane_base + kOCol0 + t * D + hf * (D / 2);  // its D/2 accumulator columns
-    float* xch = reinterpret_cast<float*>(smem + SM::kXchOff);
+    const uint32_t s_addr = tmem + lane_base + t * kTileN;        // this row's 128 score columns
+    const uint32_t o_addr = tmem + lane_base + kOCol0 + t * D;    // its D accumulator columns
     const TileRange my = t ? tr[1] : tr[0];
     if (my.active) {
       const int row = row0 + t * kTileM + r;           // sequence row (local) or compact row (global)
@@ -305,8 +309,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       const int seq_row = valid ? (compact ? q_idx_b[row] : row) : -1;
       const int pos = valid ? seq_row + a.q_pos_offset - vis_shift : -1;   // largest visible key position
       const int pos_lo = valid ? (pos - w_eff) : 0x7fffffff;               // smallest visible key position
-      float m_use = -INFINITY;   // reference maximum, exp2 domain (identical in both threads of a row)
-      float l = 0.f;             // this thread's part of the row sum
+      float m_use = -INFINITY;   // reference maximum, exp2 domain
+      float l = 0.f;             // row sum
       bool ok = true;
       const int n_my = my.hi - my.lo + 1;
 
@@ -315,40 +319,33 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         // warp-uniform outcome: the TMEM loads/stores below are warp-collective
         if (!__all_sync(0xffffffffu, mbar_wait(&bar->s_full[t], i & 1, abort_flag))) { ok = false; break; }
         tc_fence_after();
-        const int k0 = j * kTileN + hf * 64;
-        const bool partial = (k0 + 63 > my.min_pos - vis_shift) || (k0 < my.max_pos - w_eff);
-        // pass 1: row maximum of this half (32 columns at a time: the scores are re-read from TMEM in pass 2
-        // rather than kept in 64 registers)
-        float mx = -INFINITY;
-        {
-          // both loads in flight before the one wait (nothing else is live in this pass)
-          uint32_t v0[32], v1[32];
-          tmem_ld32(s_addr, v0);
-          tmem_ld32(s_addr + 32, v1);
-          tmem_ld_wait();
-          if (partial) {
+        const int k0 = j * kTileN;
+        const bool partial = (k0 + kTileN - 1 > my.min_pos - vis_shift) || (k0 < my.max_pos - w_eff);
+        uint32_t v[4][32];       // the row's scores of this key block
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, v[c]);
+        tmem_ld_wait();
+        if (partial) {
+          // edge block (causal diagonal, left window edge, ragged rows): masked scores become -inf, whose
+          // exponential is an exact zero below
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
 #pragma unroll
             for (int e = 0; e < 32; ++e) {
-              const int kp = k0 + e;
-              if (kp <= pos && kp >= pos_lo) mx = fmaxf(mx, __uint_as_float(v0[e]));
-              if (kp + 32 <= pos && kp + 32 >= pos_lo) mx = fmaxf(mx, __uint_as_float(v1[e]));
+              const int kp = k0 + c * 32 + e;
+              v[c][e] = (kp <= pos && kp >= pos_lo) ? v[c][e] : 0xff800000u;
             }
-          } else {
-            float mx1 = -INFINITY;
-#pragma unroll
-            for (int e = 0; e < 32; e += 2) {
-              mx = fmax3(mx, __uint_as_float(v0[e]), __uint_as_float(v0[e + 1]));
-              mx1 = fmax3(mx1, __uint_as_float(v1[e]), __uint_as_float(v1[e + 1]));
-            }
-            mx = fmaxf(mx, mx1);
           }
         }
-        // row maximum over both halves: publish mine, meet the other half, read theirs
-        float* slot = xch + (((i & 1) * kNumTiles + t) * 2) * kTileM;
-        slot[hf * kTileM + r] = mx;
-        mbar_arrive(&bar->xch[t]);
-        if (!__all_sync(0xffffffffu, mbar_wait(&bar->xch[t], i & 1, abort_flag))) { ok = false; break; }
-        mx = fmaxf(mx, slot[(hf ^ 1) * kTileM + r]);
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+          mx0 = fmax3(mx0, __uint_as_float(v[0][e]), __uint_as_float(v[0][e + 1]));
+          mx1 = fmax3(mx1, __uint_as_float(v[1][e]), __uint_as_float(v[1][e + 1]));
+          mx2 = fmax3(mx2, __uint_as_float(v[2][e]), __uint_as_float(v[2][e + 1]));
+          mx3 = fmax3(mx3, __uint_as_float(v[3][e]), __uint_as_float(v[3][e + 1]));
+        }
+        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
         const float m_new = fmaxf(m_use, mx * a.scale_log2);
 
         // correction: rescale the running sum and the TMEM accumulator only when the maximum moved a lot
@@ -357,53 +354,35 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         if (__any_sync(0xffffffffu, need)) {
           const float alpha = need ? fast_exp2(m_use - m_new) : 1.0f;
           l *= alpha;
-#pragma unroll
-          for (int c = 0; c < D / 64; ++c) {
-            uint32_t v[32];
-            tmem_ld32(o_addr + c * 32, v);
+#pragma unroll 1
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(o_addr + c * 32, o);
             tmem_ld_wait();
 #pragma unroll
-            for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
-            tmem_st32(o_addr + c * 32, v);
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st32(o_addr + c * 32, o);
           }
           if (need) m_use = m_new;
         }
         const float m_eff = (m_use == -INFINITY) ? 0.f : m_use;
         const float neg_m = -m_eff;
-        // pass 2: probabilities, 32 columns at a time; P overwrites the first 32 of this half's 64 columns
-        float sum = 0.f;
+        // probabilities; the bf16 P of keys 64h .. 64h+63 overwrites score columns 64h .. 64h+31
+        float2 sum2 = make_float2(0.f, 0.f);
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t v[32];
-          tmem_ld32(s_addr + c * 32, v);
-          tmem_ld_wait();
+        for (int c = 0; c < 4; ++c) {
           uint32_t pk[16];
-          if (partial) {
 #pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              const int kp = k0 + c * 32 + 2 * e;
-              float p0 = fast_exp2(fmaf(__uint_as_float(v[2 * e]), a.scale_log2, neg_m));
-              float p1 = fast_exp2(fmaf(__uint_as_float(v[2 * e + 1]), a.scale_log2, neg_m));
-              p0 = (kp <= pos && kp >= pos_lo) ? p0 : 0.f;
-              p1 = (kp + 1 <= pos && kp + 1 >= pos_lo) ? p1 : 0.f;
-              sum += p0 + p1;
-              pk[e] = pack_bf16(p0, p1);
-            }
-          } else {
-            float2 sum2 = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[2 * e]), __uint_as_float(v[2 * e + 1])),
-                                          make_float2(a.scale_log2, a.scale_log2), make_float2(neg_m, neg_m));
-              const float2 p = make_float2(fast_exp2(x.x), fast_exp2(x.y));
-              sum2 = __fadd2_rn(sum2, p);
-              pk[e] = pack_bf16(p.x, p.y);
-            }
-            sum += sum2.x + sum2.y;
+          for (int e = 0; e < 16; ++e) {
+            const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[c][2 * e]), __uint_as_float(v[c][2 * e + 1])),
+                                        make_float2(a.scale_log2, a.scale_log2), make_float2(neg_m, neg_m));
+            const float2 p = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+            sum2 = __fadd2_rn(sum2, p);
+            pk[e] = pack_bf16(p.x, p.y);
           }
-          tmem_st16(s_addr + c * 16, pk);
+          tmem_st16(s_addr + (c >> 1) * 64 + (c & 1) * 16, pk);
         }
-        l += sum;
+        l += sum2.x + sum2.y;
         tmem_st_wait();
         tc_fence_before();
         mbar_arrive(&bar->p_full[t]);
@@ -412,88 +391,81 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       // ---- epilogue: O / l, log-sum-exp, store (local) or scatter + combine (global)
       if (ok && (n_my == 0 || __all_sync(0xffffffffu, mbar_wait(&bar->o_final, 0, abort_flag)))) {
         tc_fence_after();
-        // total row sum: exchange the two partial sums (the slot of parity n_my & 1 is free by now)
-        float* slot = xch + (((n_my & 1) * kNumTiles + t) * 2) * kTileM;
-        slot[hf * kTileM + r] = l;
-        mbar_arrive(&bar->xch[t]);
-        if (__all_sync(0xffffffffu, mbar_wait(&bar->xch[t], n_my & 1, abort_flag))) {
-          l += slot[(hf ^ 1) * kTileM + r];
-          float inv_l = (l > 0.f) ? 1.0f / l : 0.f;
-          float lse2 = m_use + log2f(l);   // log-sum-exp in the exp2 domain
-          float c_loc = 0.f;               // shared-window mode: weight of the local result s_t in a_t
-          if (shared && valid) {
-            // a_t = (e^{lse_out} o_out + e^{lse_loc} s_t) / (e^{lse_out} + e^{lse_loc}): the softmax over the whole
-            // prefix, split into the keys before the window (this kernel) and the window (the local pass)
-            const float lse_out2 = (l > 0.f) ? lse2 : -INFINITY;
-            const float lse_loc2 = a.lse_loc[((int64_t)b * a.Hq + h) * a.Lq + seq_row] * 1.4426950408889634f;
-            const float mm = fmaxf(lse_out2, lse_loc2);
-            const float w_out = fast_exp2(lse_out2 - mm), w_loc = fast_exp2(lse_loc2 - mm);
-            const float inv = 1.0f / (w_out + w_loc);
-            inv_l *= w_out * inv;
-            c_loc = w_loc * inv;
-            lse2 = mm + log2f(w_out + w_loc);
-          }
-          if (valid && hf == 0 && a.lse != nullptr) {
-            const float lse = lse2 * 0.6931471805599453f;
-            a.lse[((int64_t)b * a.Hq + h) * a.Lq + row] = lse;
-          }
-          bf16* dst1 = nullptr;   // row-indexed destination (s rows, or compact a rows)
-          bf16* dst2 = nullptr;   // position-indexed destination
-          if (valid && dbg_in_range(row >= 0 && row < a.Lq && seq_row >= 0 && seq_row < a.Lq, a.status)) {
-            if (a.out) dst1 = a.out + b * a.out_st.b + row * a.out_st.t + (int64_t)h * D + hf * (D / 2);
-            if (a.out2 && (a.combine_mask == nullptr || a.combine_mask[(int64_t)b * a.Lq + seq_row]))
-              dst2 = a.out2 + b * a.out2_st.b + seq_row * a.out2_st.t + (int64_t)h * D + hf * (D / 2);
-          }
-          const bool accumulate = a.global_mode && a.accumulate_into_out2;
+        float inv_l = (l > 0.f) ? 1.0f / l : 0.f;
+        float lse2 = m_use + log2f(l);   // log-sum-exp in the exp2 domain
+        float c_loc = 0.f;               // shared-window mode: weight of the local result s_t in a_t
+        if (shared && valid) {
+          // a_t = (e^{lse_out} o_out + e^{lse_loc} s_t) / (e^{lse_out} + e^{lse_loc}): the softmax over the whole
+          // prefix, split into the keys before the window (this kernel) and the window (the local pass)
+          const float lse_out2 = (l > 0.f) ? lse2 : -INFINITY;
+          const float lse_loc2 = a.lse_loc[((int64_t)b * a.Hq + h) * a.Lq + seq_row] * 1.4426950408889634f;
+          const float mm = fmaxf(lse_out2, lse_loc2);
+          const float w_out = fast_exp2(lse_out2 - mm), w_loc = fast_exp2(lse_loc2 - mm);
+          const float inv = 1.0f / (w_out + w_loc);
+          inv_l *= w_out * inv;
+          c_loc = w_loc * inv;
+          lse2 = mm + log2f(w_out + w_loc);
+        }
+        if (valid && a.lse != nullptr) {
+          const float lse = lse2 * 0.6931471805599453f;
+          a.lse[((int64_t)b * a.Hq + h) * a.Lq + row] = lse;
+        }
+        bf16* dst1 = nullptr;   // row-indexed destination (s rows, or compact a rows)
+        bf16* dst2 = nullptr;   // position-indexed destination
+        if (valid && dbg_in_range(row >= 0 && row < a.Lq && seq_row >= 0 && seq_row < a.Lq, a.status)) {
+          if (a.out) dst1 = a.out + b * a.out_st.b + row * a.out_st.t + (int64_t)h * D;
+          if (a.out2 && (a.combine_mask == nullptr || a.combine_mask[(int64_t)b * a.Lq + seq_row]))
+            dst2 = a.out2 + b * a.out2_st.b + seq_row * a.out2_st.t + (int64_t)h * D;
+        }
+        const bool accumulate = a.global_mode && a.accumulate_into_out2;
+#pragma unroll 1
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t o[32];
+          if (n_my > 0) {
+            tmem_ld32(o_addr + c * 32, o);
+            tmem_ld_wait();
+          } else {
 #pragma unroll
-          for (int c = 0; c < D / 64; ++c) {
-            uint32_t v[32];
-            if (n_my > 0) {
-              tmem_ld32(o_addr + c * 32, v);
-              tmem_ld_wait();
-            } else {
+            for (int e = 0; e < 32; ++e) o[e] = 0u;    // no key before the window: the accumulator was never written
+          }
+          float f[32];
 #pragma unroll
-              for (int e = 0; e < 32; ++e) v[e] = 0u;    // no key before the window: the accumulator was never written
+          for (int e = 0; e < 32; ++e) f[e] = __uint_as_float(o[e]) * inv_l;
+          if (shared && dst2) {
+            const uint4* s4 = reinterpret_cast<const uint4*>(dst2 + c * 32);   // s_t, written by the local pass
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const uint4 old = s4[q];
+              const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                f[8 * q + 2 * k] = fmaf(c_loc, __uint_as_float(ow[k] << 16), f[8 * q + 2 * k]);
+                f[8 * q + 2 * k + 1] = fmaf(c_loc, __uint_as_float(ow[k] & 0xffff0000u), f[8 * q + 2 * k + 1]);
+              }
             }
-            float f[32];
+          }
+          if (dst1) {
+            uint4* d4 = reinterpret_cast<uint4*>(dst1 + c * 32);
 #pragma unroll
-            for (int e = 0; e < 32; ++e) f[e] = __uint_as_float(v[e]) * inv_l;
-            if (shared && dst2) {
-              const uint4* s4 = reinterpret_cast<const uint4*>(dst2 + c * 32);   // s_t, written by the local pass
+            for (int q = 0; q < 4; ++q)
+              d4[q] = make_uint4(pack_bf16(f[8 * q], f[8 * q + 1]), pack_bf16(f[8 * q + 2], f[8 * q + 3]),
+                                 pack_bf16(f[8 * q + 4], f[8 * q + 5]), pack_bf16(f[8 * q + 6], f[8 * q + 7]));
+          }
+          if (dst2) {
+            uint4* d4 = reinterpret_cast<uint4*>(dst2 + c * 32);
 #pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                const uint4 old = s4[q];
+            for (int q = 0; q < 4; ++q) {
+              if (accumulate) {
+                const uint4 old = d4[q];
                 const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                  f[8 * q + 2 * k] = fmaf(c_loc, __uint_as_float(ow[k] << 16), f[8 * q + 2 * k]);
-                  f[8 * q + 2 * k + 1] = fmaf(c_loc, __uint_as_float(ow[k] & 0xffff0000u), f[8 * q + 2 * k + 1]);
+                  f[8 * q + 2 * k] += __uint_as_float(ow[k] << 16);
+                  f[8 * q + 2 * k + 1] += __uint_as_float(ow[k] & 0xffff0000u);
                 }
               }
-            }
-            if (dst1) {
-              uint4* d4 = reinterpret_cast<uint4*>(dst1 + c * 32);
-#pragma unroll
-              for (int q = 0; q < 4; ++q)
-                d4[q] = make_uint4(pack_bf16(f[8 * q], f[8 * q + 1]), pack_bf16(f[8 * q + 2], f[8 * q + 3]),
-                                   pack_bf16(f[8 * q + 4], f[8 * q + 5]), pack_bf16(f[8 * q + 6], f[8 * q + 7]));
-            }
-            if (dst2) {
-              uint4* d4 = reinterpret_cast<uint4*>(dst2 + c * 32);
-#pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                if (accumulate) {
-                  const uint4 old = d4[q];
-                  const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
-#pragma unroll
-                  for (int k = 0; k < 4; ++k) {
-                    f[8 * q + 2 * k] += __uint_as_float(ow[k] << 16);
-                    f[8 * q + 2 * k + 1] += __uint_as_float(ow[k] & 0xffff0000u);
-                  }
-                }
-                d4[q] = make_uint4(pack_bf16(f[8 * q], f[8 * q + 1]), pack_bf16(f[8 * q + 2], f[8 * q + 3]),
-                                   pack_bf16(f[8 * q + 4], f[8 * q + 5]), pack_bf16(f[8 * q + 6], f[8 * q + 7]));
-              }
+              d4[q] = make_uint4(pack_bf16(f[8 * q], f[8 * q + 1]), pack_bf16(f[8 * q + 2], f[8 * q + 3]),
+                                 pack_bf16(f[8 * q + 4], f[8 * q + 5]), pack_bf16(f[8 * q + 6], f[8 * q + 7]));
             }
           }
         }
@@ -511,7 +483,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     if (tid == 0) atomicExch(a.status, 1);
     __syncthreads();
   }
-  if (warp == 17) tmem_dealloc(tmem, 512);
+  if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
 }
 
 }  // namespace
