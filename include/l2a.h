@@ -110,6 +110,17 @@ typedef struct l2a_params {
    * dense.  l2a_step_host, l2a_router_backward and the q / O arguments of l2a_decode take dense tensors only
    * (L2A_ERR_UNSUPPORTED otherwise). */
   int64_t q_stride[2], k_stride[2], v_stride[2], o_stride[2];
+  /* Packed variable-length batch (optional; NULL = every batch entry is one sequence).  Device pointer to the
+   * per-token table written by l2a_pack_sequences: int32 [Lq][2] = {first token of the token's sequence, one past its
+   * last token}.  The token axis then holds several sequences back to back and no query attends across a sequence
+   * boundary: token t sees the keys max(t - W, first) .. t (Local Attention) and first .. t (Global Attention);
+   * key blocks and query tiles that lie wholly in other sequences are not visited.  Needs B == 1, Lq == Lk and
+   * q_pos_offset == 0.  Routing, compaction and every output keep their meaning on the packed token axis, and the
+   * results are, sequence by sequence, those of one call per sequence (equal up to fp32 rounding: the key blocks are
+   * aligned to the packed axis, not to each sequence's start).  The table is read by l2a_forward*, l2a_backward* and
+   * l2a_forward_routed; l2a_step_host and l2a_decode reject it (L2A_ERR_UNSUPPORTED).  The paper evaluates padded
+   * batches only; this layout is the usual one for training on documents of mixed length. */
+  const int32_t* seq_bounds;
 } l2a_params;
 
 /* Version / capability string of the loaded library (host pointer, static storage). */
@@ -146,6 +157,18 @@ l2a_status l2a_selftest_wait_timeout(void* ws, unsigned limit_us, void* stream);
  * (debug build) L2A_ERR_DEVICE_BOUNDS if an index check failed.
  */
 l2a_status l2a_workspace_status(const void* ws, void* stream);
+
+/*
+ * Packed variable-length batches: expands the sequence boundaries into the per-token table that
+ * l2a_params.seq_bounds points to.
+ *   cu_seqlens  device int32 [n_seq + 1], ascending, cu_seqlens[0] = 0: sequence i holds the tokens
+ *               cu_seqlens[i] .. cu_seqlens[i + 1] - 1 of the packed axis
+ *   seq_bounds  device int32 [Lq][2], written: {first token, one past the last token} of each token's sequence.
+ *               Tokens at or after cu_seqlens[n_seq] (padding at the end of the axis) become sequences of their own.
+ * One small kernel on `stream`; no allocation.  Entries of cu_seqlens that are not ascending give masks that
+ * correspond to no batch, but no access outside the tensors.
+ */
+l2a_status l2a_pack_sequences(const int32_t* cu_seqlens, int n_seq, int Lq, int32_t* seq_bounds, void* stream);
 
 /*
  * Routing decision and query compaction (Eq. 3; Section 3.2: the routed queries are gathered into one

@@ -165,6 +165,7 @@ struct BwdArgs {
   const int32_t* q_idx;
   const int32_t* n_routed;
   const int32_t* prefix;
+  const int32_t* seq_bounds;   // packed sequences (B == 1): per token {first token of its sequence, one past the last}
   const float* lse_loc;    // [B,Hq,Lq] by row
   const float* lse_glb;    // [B,Hq,Lq] by compact row
   const float* delta_loc;  // same indexing
@@ -202,10 +203,16 @@ struct ItemPlan {
 
 __device__ __forceinline__ ItemPlan make_plan(const BwdArgs& a, int b, int k0, int span = kTileN) {
   ItemPlan p;
+  // packed sequences: no row at or after the end of the sequence that holds the block's last key sees any of its keys
+  int row_end = a.Lq;
+  if (a.seq_bounds != nullptr) {
+    const int k_last = min(k0 + span, a.Lk) - 1;
+    row_end = max(0, min(a.Lq, a.seq_bounds[2 * k_last + 1]));
+  }
   // local: rows t with position in [k0, k0 + span - 1 + W]
   int tmin = k0 - a.q_pos_offset;
   const long long tmax_ll = (long long)k0 + span - 1 + a.window - a.q_pos_offset;
-  int tmax = tmax_ll > a.Lq - 1 ? a.Lq - 1 : (int)tmax_ll;
+  int tmax = tmax_ll > row_end - 1 ? row_end - 1 : (int)tmax_ll;
   if (tmin < 0) tmin = 0;
   if (tmax < tmin || a.skip_local) { p.loc_t0 = 0; p.loc_nt = 0; }
   else { p.loc_t0 = tmin / kTileM; p.loc_nt = tmax / kTileM - p.loc_t0 + 1; }
@@ -213,11 +220,12 @@ __device__ __forceinline__ ItemPlan make_plan(const BwdArgs& a, int b, int k0, i
   const int n_c = a.skip_global ? 0 : a.n_routed[b];
   long long tmin_g = (long long)k0 - a.q_pos_offset + a.vis_shift;
   if (tmin_g < 0) tmin_g = 0;
-  if (tmin_g > a.Lq - 1 || n_c == 0) { p.glb_t0 = 0; p.glb_nt = 0; }
+  if (tmin_g > row_end - 1 || n_c == 0) { p.glb_t0 = 0; p.glb_nt = 0; }
   else {
     const int c_min = a.prefix[(int64_t)b * (a.Lq + 1) + (int)tmin_g];
-    if (c_min >= n_c) { p.glb_t0 = 0; p.glb_nt = 0; }
-    else { p.glb_t0 = c_min / kTileM; p.glb_nt = (n_c - 1) / kTileM - p.glb_t0 + 1; }
+    const int c_end = row_end < a.Lq ? min(n_c, a.prefix[(int64_t)b * (a.Lq + 1) + row_end]) : n_c;
+    if (c_min >= c_end) { p.glb_t0 = 0; p.glb_nt = 0; }
+    else { p.glb_t0 = c_min / kTileM; p.glb_nt = (c_end - 1) / kTileM - p.glb_t0 + 1; }
   }
   p.per_head = p.loc_nt + p.glb_nt;
   p.total = p.per_head * (a.Hq / a.Hkv);
@@ -426,7 +434,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
     // lse * log2(e) and Delta of the item's 128 query rows, plus per-quarter mask flags, go to shared memory.
     // The global loads of item i+1 are issued before waiting for its slot, so their latency is hidden.
     float r_lse[4], r_delta[4];
-    int r_pos[4], r_glb = 0, r_row0 = 0, r_h = 0;
+    int r_pos[4], r_lo[4], r_glb = 0, r_row0 = 0, r_h = 0;   // r_lo: first token of the row's sequence (packed batches)
     ItemCursor cur(plan, g * G);
     auto load_item = [&]() {
       const int h = cur.h, glb = cur.glb(), row0 = cur.tile() * kTileM;
@@ -444,7 +452,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
         const int64_t si = ((int64_t)b * a.Hq + h) * a.Lq + (valid ? row : 0);
         r_lse[q] = valid ? __ldg(&lse[si]) * kLog2e : 0.f;
         r_delta[q] = valid ? __ldg(&dl[si]) : 0.f;
-        r_pos[q] = valid ? (glb ? __ldg(&a.q_idx[(int64_t)b * a.Lq + row]) - a.vis_shift : row) + a.q_pos_offset : -1;
+        const int token = valid ? (glb ? __ldg(&a.q_idx[(int64_t)b * a.Lq + row]) : row) : 0;
+        r_pos[q] = valid ? token - (glb ? a.vis_shift : 0) + a.q_pos_offset : -1;
+        r_lo[q] = (valid && a.seq_bounds != nullptr) ? __ldg(&a.seq_bounds[2 * token]) : -0x40000000;
       }
     };
     load_item();
@@ -461,7 +471,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
         st_lse[col] = r_lse[q];
         st_delta[col] = -r_delta[q];   // negated: dS = P * (dP + (-Delta)) with packed f32x2 arithmetic
         // quarter q needs the element mask unless every (key, query) pair of it is visible
-        const bool lane_ok = r_pos[q] >= 0 && (k0 + kTileN - 1 <= r_pos[q]) && (k0 >= r_pos[q] - w_eff);
+        const bool lane_ok = r_pos[q] >= 0 && (k0 + kTileN - 1 <= r_pos[q]) && (k0 >= max(r_pos[q] - w_eff, r_lo[q]));
         const bool interior = __all_sync(0xffffffffu, lane_ok);
         if (lane == 0) st_flags[q] = interior ? 0 : 1;
       }
@@ -612,16 +622,20 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
           const int32_t* qi = a.q_idx + (int64_t)b * a.Lq;
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
-            int pos[2];
+            int pos[2], lo[2];
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
               const int row = item_row0 + q * 32 + e + u;
-              pos[u] = row < n_rows ? (item_glb ? __ldg(&qi[row]) - a.vis_shift : row) + a.q_pos_offset : -1;
+              const bool valid = row < n_rows;
+              const int token = valid ? (item_glb ? __ldg(&qi[row]) : row) : 0;
+              pos[u] = valid ? token - (item_glb ? a.vis_shift : 0) + a.q_pos_offset : -1;
+              lo[u] = pos[u] - w_eff;
+              if (valid && a.seq_bounds != nullptr) lo[u] = max(lo[u], __ldg(&a.seq_bounds[2 * token]));
             }
             float p0 = fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, -st[e]));
             float p1 = fast_exp2(fmaf(__uint_as_float(sv[e + 1]), a.scale_log2, -st[e + 1]));
-            p0 = (kp <= pos[0] && kp >= pos[0] - w_eff) ? p0 : 0.f;
-            p1 = (kp <= pos[1] && kp >= pos[1] - w_eff) ? p1 : 0.f;
+            p0 = (kp <= pos[0] && kp >= lo[0]) ? p0 : 0.f;
+            p1 = (kp <= pos[1] && kp >= lo[1]) ? p1 : 0.f;
             pp[e >> 1] = pack_bf16(p0, p1);
           }
         }
@@ -1002,6 +1016,7 @@ static l2a_status backward_impl(const l2a_params* p, const void* Q, const void* 
   a.skip_local = skip_local ? 1 : 0;
   a.skip_global = skip_global ? 1 : 0;
   a.q_idx = q_idx; a.n_routed = n_routed; a.prefix = prefix;
+  a.seq_bounds = p->seq_bounds;
   a.lse_loc = share ? lse_c : lse_loc; a.lse_glb = force_all ? lse_c : lse_glb;
   a.vis_shift = share ? (p->window < (1 << 30) ? p->window : (1 << 30)) + 1 : 0; a.delta_loc = delta_loc; a.delta_glb = delta_glb;
   a.dQ = static_cast<bf16*>(dQ); a.dK = static_cast<bf16*>(dK); a.dV = static_cast<bf16*>(dV);

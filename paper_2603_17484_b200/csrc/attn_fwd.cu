@@ -63,6 +63,7 @@ struct Barriers {
 struct TileRange {
   int active;    // tile has at least one valid row
   int min_pos, max_pos;
+  int max_lo;    // largest "first visible key position" among the rows (the last row's)
   int lo, hi;    // first / last key block
 };
 
@@ -107,11 +108,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
     if (last > n_rows - 1) last = n_rows - 1;
     tr[t].active = first < n_rows;
     if (tr[t].active) {
-      tr[t].min_pos = (compact ? q_idx_b[first] : first) + a.q_pos_offset;
-      tr[t].max_pos = (compact ? q_idx_b[last] : last) + a.q_pos_offset;
-      const int lo_pos = tr[t].min_pos - w_eff;
+      const int first_seq = compact ? q_idx_b[first] : first, last_seq = compact ? q_idx_b[last] : last;
+      tr[t].min_pos = first_seq + a.q_pos_offset;
+      tr[t].max_pos = last_seq + a.q_pos_offset;
+      int lo_pos = tr[t].min_pos - w_eff;
+      tr[t].max_lo = tr[t].max_pos - w_eff;
+      if (a.seq_bounds != nullptr) {
+        // packed sequences: no key before the start of the row's own sequence (starts ascend with the rows)
+        lo_pos = max(lo_pos, a.seq_bounds[2 * first_seq]);
+        tr[t].max_lo = max(tr[t].max_lo, a.seq_bounds[2 * last_seq]);
+      }
       const int hi_pos = tr[t].max_pos - vis_shift;   // last key position any row of the tile attends to
-      if (hi_pos >= 0) {
+      if (hi_pos >= 0 && hi_pos >= lo_pos) {
         tr[t].lo = lo_pos > 0 ? lo_pos / kTileN : 0;
         tr[t].hi = hi_pos / kTileN;
         jlo = min(jlo, tr[t].lo);
@@ -120,7 +128,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         tr[t].lo = 1; tr[t].hi = 0;   // shared-window mode: every key of these rows lies inside the window
       }
     } else {
-      tr[t].min_pos = tr[t].max_pos = 0;
+      tr[t].min_pos = tr[t].max_pos = tr[t].max_lo = 0;
       tr[t].lo = 1; tr[t].hi = 0;
     }
   }
@@ -308,7 +316,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
       const bool valid = row < n_rows;
       const int seq_row = valid ? (compact ? q_idx_b[row] : row) : -1;
       const int pos = valid ? seq_row + a.q_pos_offset - vis_shift : -1;   // largest visible key position
-      const int pos_lo = valid ? (pos - w_eff) : 0x7fffffff;               // smallest visible key position
+      int pos_lo = valid ? (pos - w_eff) : 0x7fffffff;                     // smallest visible key position
+      if (valid && a.seq_bounds != nullptr) pos_lo = max(pos_lo, a.seq_bounds[2 * seq_row]);
       float m_use = -INFINITY;   // reference maximum, exp2 domain
       float l = 0.f;             // row sum
       bool ok = true;
@@ -320,7 +329,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant_
         if (!__all_sync(0xffffffffu, mbar_wait(&bar->s_full[t], i & 1, abort_flag))) { ok = false; break; }
         tc_fence_after();
         const int k0 = j * kTileN;
-        const bool partial = (k0 + kTileN - 1 > my.min_pos - vis_shift) || (k0 < my.max_pos - w_eff);
+        const bool partial = (k0 + kTileN - 1 > my.min_pos - vis_shift) || (k0 < my.max_lo);
         uint32_t v[4][32];       // the row's scores of this key block
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, v[c]);

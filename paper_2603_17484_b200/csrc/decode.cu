@@ -341,6 +341,7 @@ extern "C" l2a_status l2a_decode(const l2a_params* p, const void* q, const void*
        reinterpret_cast<uintptr_t>(O)) & 15)
     return L2A_ERR_INVALID_ARG;
   if (p->Hq / p->Hkv > kMaxGroup) return L2A_ERR_UNSUPPORTED;
+  if (p->seq_bounds) return L2A_ERR_UNSUPPORTED;   // a decode step has one cache per batch entry
   if (p->q_pos_offset >= p->Lk) return L2A_ERR_INVALID_ARG;     // the new token's own key must be in the cache
   if (!ws || (reinterpret_cast<uintptr_t>(ws) % 256) != 0 || ws_bytes < need) return L2A_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -40,6 +40,9 @@ l2a_status check_params(const l2a_params* p) {
   if (!strides_ok(p->q_stride, p->Lq, p->Hq * p->D) || !strides_ok(p->k_stride, p->Lk, p->Hkv * p->D) ||
       !strides_ok(p->v_stride, p->Lk, p->Hkv * p->D) || !strides_ok(p->o_stride, p->Lq, p->Hq * p->D))
     return L2A_ERR_INVALID_ARG;
+  // packed sequences: one token axis, positions are token indices
+  if (p->seq_bounds && (p->B != 1 || p->Lq != p->Lk || p->q_pos_offset != 0 || !aligned(p->seq_bounds, 8)))
+    return L2A_ERR_INVALID_ARG;
   return L2A_OK;
 }
 
@@ -174,6 +177,12 @@ l2a_status l2a_workspace_status(const void* ws, void* stream) {
   if (cudaMemcpyAsync(&word, ws, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return L2A_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return L2A_ERR_CUDA;
   return word == 0 ? L2A_OK : word == 4 ? L2A_ERR_DEVICE_BOUNDS : L2A_ERR_DEVICE_TIMEOUT;
+}
+
+l2a_status l2a_pack_sequences(const int32_t* cu_seqlens, int n_seq, int Lq, int32_t* seq_bounds, void* stream) {
+  if (!cu_seqlens || !seq_bounds || n_seq < 0 || Lq <= 0 || !aligned(seq_bounds, 8)) return L2A_ERR_INVALID_ARG;
+  return launch_pack_sequences(cu_seqlens, n_seq, Lq, seq_bounds, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? L2A_OK : L2A_ERR_CUDA;
 }
 
 l2a_status l2a_route_compact(const l2a_params* p, const void* router, int router_kind, float logit_threshold,
@@ -314,6 +323,7 @@ static l2a_status forward_range(const l2a_params* p, const void* Q, const void* 
   a.row_end = row_range ? row_end : 0x7fffffff;
   a.shared_window = 0;
   a.lse_loc = nullptr;
+  a.seq_bounds = p->seq_bounds;
 
   PhaseEvents& pe = phase_events();
   struct ClearOnExit { PhaseEvents& p; ~ClearOnExit() { p.clear(); } } clear_on_exit{pe};
@@ -449,6 +459,7 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
   l2a_status st = check_params(p);
   if (st != L2A_OK) return st;
   if (!host || !dev) return L2A_ERR_INVALID_ARG;
+  if (p->seq_bounds) return L2A_ERR_UNSUPPORTED;   // the row-range pipeline assumes one sequence per batch entry
   const bool bwd = host->dO != nullptr;
   if (!host->Q || !host->K || !host->V || !host->router || !host->O || !dev->Q || !dev->K || !dev->V ||
       !dev->router || !dev->O)

@@ -74,6 +74,7 @@ struct RouteArgs {
 };
 constexpr int kRouteBlockElems = 4096;  // positions per CTA of the route/compact kernels
 cudaError_t launch_route_compact(const RouteArgs& a, cudaStream_t stream);
+cudaError_t launch_pack_sequences(const int32_t* cu_seqlens, int n_seq, int L, int32_t* seq_bounds, cudaStream_t stream);
 
 // Gathers rows src[b, q_idx[b][c], :] -> dst[b, c, :] for c < n_routed[b], and zero-fills rows up to
 // the next multiple of kRowsPerCta (bounded by L) so that padded MMA tiles read zeros.  With `prefix` given, only the
@@ -115,6 +116,8 @@ struct FwdArgs {
   // local result (s_t read from out2, its log-sum-exp from lse_loc).
   int shared_window;
   const float* lse_loc;      // [B,Hq,Lq] by row; read only when shared_window is set
+  // Packed variable-length batch (B == 1): per token {first token of its sequence, one past the last}; NULL otherwise
+  const int32_t* seq_bounds;
 };
 size_t bwd_ws_size(const l2a_params* p);
 // Key-block ranges of the backward when the caller registered phase events for them (11 events: four ranges, 7: two,

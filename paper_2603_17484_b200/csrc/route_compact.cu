@@ -220,6 +220,28 @@ __global__ void __launch_bounds__(256) router_logits_kernel(const bf16* __restri
   if (sum_sq != nullptr && lane == 0 && t_end > t_begin) atomicAdd(&sum_sq[reg_b], reg_sum);
 }
 
+// Packed variable-length batches: token t belongs to the sequence i with cu[i] <= t < cu[i + 1] (binary search over
+// the n_seq + 1 boundaries); tokens at or after cu[n_seq] are sequences of their own.
+__global__ void __launch_bounds__(256) pack_sequences_kernel(const int32_t* __restrict__ cu, int n_seq, int L,
+                                                             int32_t* __restrict__ seq_bounds) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= L) return;
+  int lo = 0, hi = n_seq;                  // invariant: cu[lo] <= t (cu[0] = 0); answer in [lo, hi)
+  if (n_seq <= 0 || t >= __ldg(&cu[n_seq])) {
+    reinterpret_cast<int2*>(seq_bounds)[t] = make_int2(t, t + 1);
+    return;
+  }
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (__ldg(&cu[mid]) <= t) lo = mid; else hi = mid;
+  }
+  int first = __ldg(&cu[lo]), end = __ldg(&cu[lo + 1]);
+  // boundaries that are not ascending must still give a range that holds t and stays inside the axis
+  first = max(0, min(first, t));
+  end = min(L, max(end, t + 1));
+  reinterpret_cast<int2*>(seq_bounds)[t] = make_int2(first, end);
+}
+
 }  // namespace
 
 cudaError_t launch_router_logits(const bf16* S, const float* w, float bias, float* logits, float* sum_sq, int B, int L,
@@ -233,6 +255,11 @@ cudaError_t launch_router_logits(const bf16* S, const float* w, float bias, floa
   const int64_t max_blocks = ((int64_t)B * L + 8 * kRlTokens - 1) / (8 * kRlTokens);
   if (blocks > max_blocks) blocks = max_blocks;
   router_logits_kernel<<<(unsigned)blocks, 256, 0, stream>>>(S, w, bias, logits, sum_sq, B, L, row_elems);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pack_sequences(const int32_t* cu_seqlens, int n_seq, int L, int32_t* seq_bounds, cudaStream_t stream) {
+  pack_sequences_kernel<<<ceil_div(L, 256), 256, 0, stream>>>(cu_seqlens, n_seq, L, seq_bounds);
   return cudaGetLastError();
 }
 

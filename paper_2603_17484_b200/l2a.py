@@ -31,7 +31,7 @@ EXPORTS = (
     "l2a_route_compact", "l2a_forward", "l2a_backward", "l2a_step_host", "l2a_profile_next_call",
     "l2a_route_compact_static", "l2a_router_logits", "l2a_decode_workspace_bytes", "l2a_decode",
     "l2a_backward_split", "l2a_router_backward", "l2a_forward_routed", "l2a_selftest_wait_timeout",
-    "l2a_forward_sets", "l2a_backward_sets",
+    "l2a_forward_sets", "l2a_backward_sets", "l2a_pack_sequences",
 )
 
 
@@ -43,6 +43,7 @@ class L2AParams(ctypes.Structure):
         ("softmax_scale", ctypes.c_float), ("flags", ctypes.c_uint32),
         ("q_stride", ctypes.c_int64 * 2), ("k_stride", ctypes.c_int64 * 2),
         ("v_stride", ctypes.c_int64 * 2), ("o_stride", ctypes.c_int64 * 2),
+        ("seq_bounds", ctypes.c_void_p),
     ]
 
 
@@ -80,12 +81,14 @@ def status_string(code: int) -> str:
 
 
 def params(B, Lq, Lk, Hq, Hkv, D, window, q_pos_offset=None, softmax_scale=0.0, flags=0, q_stride=None,
-           k_stride=None, v_stride=None, o_stride=None) -> L2AParams:
-    """Strides: optional (batch stride, token stride) in elements; None = dense (see include/l2a.h)."""
+           k_stride=None, v_stride=None, o_stride=None, seq_bounds=None) -> L2AParams:
+    """Strides: optional (batch stride, token stride) in elements; None = dense (see include/l2a.h).
+    seq_bounds: the int32 [Lq, 2] device table of l2a_pack_sequences for a packed variable-length batch (the caller
+    keeps the tensor alive while the parameters are in use)."""
     two = ctypes.c_int64 * 2
     st = [two(*(s if s is not None else (0, 0))) for s in (q_stride, k_stride, v_stride, o_stride)]
     return L2AParams(B, Lq, Lk, Hq, Hkv, D, window, Lk - Lq if q_pos_offset is None else q_pos_offset,
-                     softmax_scale, flags, *st)
+                     softmax_scale, flags, *st, None if seq_bounds is None else seq_bounds.data_ptr())
 
 
 def _ptr(t):
@@ -137,6 +140,15 @@ def l2a_route_compact(p, router, router_kind, logit_threshold, d_mask, q_idx, n_
     if check:
         _check(code, "l2a_route_compact")
     return code
+
+
+def l2a_pack_sequences(cu_seqlens, Lq, seq_bounds=None, stream=None):
+    """cu_seqlens: int32 device tensor [n_seq + 1]; returns the int32 [Lq, 2] table for `params(seq_bounds=...)`."""
+    if seq_bounds is None:
+        seq_bounds = torch.empty((Lq, 2), dtype=torch.int32, device=cu_seqlens.device)
+    _check(lib().l2a_pack_sequences(_ptr(cu_seqlens), ctypes.c_int(cu_seqlens.numel() - 1), ctypes.c_int(Lq),
+                                    _ptr(seq_bounds), _stream(stream)), "l2a_pack_sequences")
+    return seq_bounds
 
 
 def l2a_route_compact_static(p, router, router_kind, logit_threshold, d_mask, q_idx, n_routed, prefix, stream=None,

@@ -57,9 +57,10 @@ def test_workspace_sizes_and_validation(lib):
 
 
 def test_params_struct_layout_matches_header():
-    # ten 32-bit fields, then four {batch, token} stride pairs of 64-bit integers
-    assert ctypes.sizeof(l2a.L2AParams) == 40 + 4 * 2 * 8
+    # ten 32-bit fields, four {batch, token} stride pairs of 64-bit integers, the packed-sequence table pointer
+    assert ctypes.sizeof(l2a.L2AParams) == 40 + 4 * 2 * 8 + 8
     assert l2a.L2AParams.q_stride.offset == 40 and l2a.L2AParams.o_stride.offset == 88
+    assert l2a.L2AParams.seq_bounds.offset == 104
 
 
 def test_stride_arguments_are_validated_on_the_host():
