@@ -316,6 +316,9 @@ def main():
     ap.add_argument("--density", type=float, default=None)
     ap.add_argument("--routing", default=None, choices=[None, "bernoulli", "clustered", "all", "none"])
     ap.add_argument("--forward-only", action="store_true")
+    ap.add_argument("--packed-seqs", type=int, default=0,
+                    help="treat the token axis as this many equal sequences packed back to back (one launch per "
+                         "kernel; no end-to-end, CPU-baseline or extra legs)")
     ap.add_argument("--kv-heads", type=int, default=None,
                     help="run a slice of the workload with this many KV heads (and their query heads): small enough "
                          "for counter captures at the full sequence length")
@@ -357,8 +360,15 @@ def main():
     use_logits = logits is not None
     kind = l2a.ROUTER_LOGITS_F32 if use_logits else l2a.ROUTER_MASK_U8
 
+    seq_table, seq_cu = None, None
+    if args.packed_seqs > 0:
+        assert cfg.B == 1, "--packed-seqs needs a single token axis"
+        seq_cu = np.linspace(0, cfg.L, args.packed_seqs + 1).astype(np.int32)
+        seq_table = l2a.l2a_pack_sequences(torch.from_numpy(seq_cu).cuda(), cfg.L)
+        args.e2e_steps, args.cpu_rows, args.extras = 0, 0, False
+
     def params_for(shared):
-        return l2a.params(cfg.B, cfg.L, cfg.L, cfg.Hq, cfg.Hkv, cfg.D, cfg.W,
+        return l2a.params(cfg.B, cfg.L, cfg.L, cfg.Hq, cfg.Hkv, cfg.D, cfg.W, seq_bounds=seq_table,
                           flags=(l2a.FLAG_SAVE_FOR_BWD if backward else 0) | (l2a.FLAG_SHARED_WINDOW if shared else 0))
 
     p = params_for(args.shared_window)
@@ -383,6 +393,10 @@ def main():
     per_pair = 4.0 + (10.0 if backward else 0.0)
 
     def pair_counts(mask):
+        if seq_cu is not None:       # packed: every sequence by itself
+            pl = sum(synth.pairs_local(int(e - s), cfg.W) for s, e in zip(seq_cu[:-1], seq_cu[1:]))
+            pg = sum(synth.pairs_global(mask[0, s:e]) for s, e in zip(seq_cu[:-1], seq_cu[1:]))
+            return pl, pg, 0
         pl = sum(synth.pairs_local(cfg.L, cfg.W) for _ in range(cfg.B))
         pg = sum(synth.pairs_global(mask[b]) for b in range(cfg.B))
         # pairs the shared-window launches do not visit: the in-window pairs of routed rows are done once, by the local items
@@ -529,8 +543,8 @@ def main():
     tensor_phases = {k: v for k, v in phase_ms.items() if k in kernel_pairs}
     dom = max(tensor_phases, key=tensor_phases.get)
     per, credited, visited = kernel_pairs[dom]
-    il, ig = issued_pairs(d, shared_now)
-    issued = {"attn_fwd_local": il, "attn_fwd_global": ig, "bwd": il + ig}[dom]
+    il, ig = issued_pairs(d, shared_now) if seq_cu is None else (credited, 0)   # (not modelled for packed batches)
+    issued = {"attn_fwd_local": il, "attn_fwd_global": ig, "bwd": il + ig}[dom] if seq_cu is None else credited
     achieved = per * HD * credited / phase_ms[dom] / 1e9
     achieved_visited = per * HD * visited / phase_ms[dom] / 1e9
     # DRAM traffic of the dominant kernel: not captured on this workload (a counter capture of a 12 GB, 100 ms launch is
@@ -574,6 +588,7 @@ def main():
         "config": {"workload": args.workload, "B": cfg.B, "L": cfg.L, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "D": cfg.D,
                    "W": cfg.W, "routing": args.routing or cfg.routing, "density": rho_real,
                    "pass": "fwd+bwd" if backward else "fwd", "shared_window": shared_now,
+                   **({"packed_sequences": args.packed_seqs} if args.packed_seqs else {}),
                    "parallelism": f"replicas x{world}",
                    "l2_policy": "inputs larger than L2 (Q alone is %.2f GB)" % (host["Q"].numel() * 2 / 1e9),
                    "useful_tflop_per_step": step_flops / 1e12, "pairs_per_head": pl + pg,
