@@ -468,7 +468,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const int col = q * 32 + lane;
-        st_lse[col] = r_lse[q];
+        st_lse[col] = -r_lse[q];       // negated, like Delta: P = exp2(scale * s + (-lse)) is one fused multiply-add
         st_delta[col] = -r_delta[q];   // negated: dS = P * (dP + (-Delta)) with packed f32x2 arithmetic
         // quarter q needs the element mask unless every (key, query) pair of it is visible
         const bool lane_ok = r_pos[q] >= 0 && (k0 + kTileN - 1 <= r_pos[q]) && (k0 >= max(r_pos[q] - w_eff, r_lo[q]));
@@ -613,7 +613,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
             const float2 x = __ffma2_rn(make_float2(__uint_as_float(sv[2 * e]), __uint_as_float(sv[2 * e + 1])),
-                                        make_float2(a.scale_log2, a.scale_log2), make_float2(-st[2 * e], -st[2 * e + 1]));
+                                        make_float2(a.scale_log2, a.scale_log2), make_float2(st[2 * e], st[2 * e + 1]));
             pp[e] = pack_bf16(fast_exp2(x.x), fast_exp2(x.y));
           }
         } else {
@@ -632,8 +632,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
               lo[u] = pos[u] - w_eff;
               if (valid && a.seq_bounds != nullptr) lo[u] = max(lo[u], __ldg(&a.seq_bounds[2 * token]));
             }
-            float p0 = fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, -st[e]));
-            float p1 = fast_exp2(fmaf(__uint_as_float(sv[e + 1]), a.scale_log2, -st[e + 1]));
+            float p0 = fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, st[e]));
+            float p1 = fast_exp2(fmaf(__uint_as_float(sv[e + 1]), a.scale_log2, st[e + 1]));
             p0 = (kp <= pos[0] && kp >= lo[0]) ? p0 : 0.f;
             p1 = (kp <= pos[1] && kp >= lo[1]) ? p1 : 0.f;
             pp[e >> 1] = pack_bf16(p0, p1);
