@@ -85,3 +85,19 @@ def test_flag_and_router_constants_match_the_header():
         assert getattr(l2a, name) == value, name
     flags = [v for k, v in defines.items() if k.startswith("FLAG_")]
     assert len(set(flags)) == len(flags) and all(v & (v - 1) == 0 for v in flags)   # distinct single bits
+
+
+def test_packed_sequence_table_is_validated_on_the_host():
+    """l2a_params.seq_bounds needs one token axis (B = 1), Lq = Lk, no position offset and an 8-byte aligned table;
+    the check runs before anything is launched (the pointer is never dereferenced on the host)."""
+    class Fake:                      # stands in for a device tensor: only its address is marshalled
+        def __init__(self, addr): self.addr = addr
+        def data_ptr(self): return self.addr
+    ok = dict(B=1, Lq=512, Lk=512, Hq=4, Hkv=2, D=128, window=16)
+    l2a.l2a_workspace_bytes(l2a.params(**ok, seq_bounds=Fake(0x10000)))
+    for bad in (dict(ok, B=2), dict(ok, Lk=1024), dict(ok, Lk=1024, q_pos_offset=0)):
+        with pytest.raises(l2a.L2AError) as e:
+            l2a.l2a_workspace_bytes(l2a.params(**bad, seq_bounds=Fake(0x10000)))
+        assert e.value.code == -1
+    with pytest.raises(l2a.L2AError):
+        l2a.l2a_workspace_bytes(l2a.params(**ok, seq_bounds=Fake(0x10004)))
