@@ -32,6 +32,11 @@ for (B, Lq, Lk, Hq, Hkv, D, W, rho, flags) in [(1, 700, 700, 2, 1, 128, 200, 0.3
     run_backward(c)
     check_backward_full(c)
 
+# 1b. a packed variable-length batch: the same checks with per-sequence masks, tile ranges and item lists
+from tests.test_gpu_packed import packed_case, check_packed
+c, want = packed_case([300, 1, 129, 450], 4, 2, 128, 100, 0.4, seed=77)
+check_packed(c, want)
+
 # 2. a compact index one past the end: reported, the row is not stored, the guards stay intact
 B, L, Hq, Hkv, D, W = 1, 600, 2, 1, 128, 64
 d = synth.mask_bernoulli(B, L, 0.3, seed=4)
