@@ -108,3 +108,25 @@ def test_packed_rejects_what_it_does_not_cover():
         with pytest.raises(l2a.L2AError) as e:
             l2a.l2a_workspace_bytes(p)
         assert e.value.code == -1
+
+
+def test_packed_batch_with_global_attention_for_every_token():
+    """Forced-global iterations (Section 3.3) on a packed batch: a_t of every token comes from its own sequence."""
+    lengths = [200, 515, 129, 300]
+    c, want = packed_case(lengths, 4, 2, 128, 80, 0.3, seed=751, flags=l2a.FLAG_FORCE_ALL_GLOBAL)
+    b = c.run_forward()
+    run_backward(c)
+    sh = c.shape
+    for s, e, fwd, grads in oracle_by_sequence(c, want, True):
+        n = e - s
+        one = oracle.Shape(1, n, n, sh.Hq, sh.Hkv, sh.D, sh.window)
+        sl = {k: np.ascontiguousarray(c.u16(k)[:, s:e]) for k in ("Q", "K", "V", "dO")}
+        every = oracle.forward_full(one, sl["Q"], sl["K"], sl["V"], np.ones((1, n), np.uint8))
+        check_close(to_f64(b.O[:, s:e]), fwd["o"], "O (packed, forced global)")
+        check_close(to_f64(b.A_c[:, s:e]), every["a"], "A by row (packed)")
+        check_close(to_f64(b.lse_glb[:, :, s:e]), every["lse_glb"], "lse_glb by row", LSE_ABS, LSE_ABS)
+        for got, ref, name in zip((b.dQ, b.dK, b.dV), grads, ("dQ", "dK", "dV")):
+            check_close(to_f64(got[:, s:e]), ref, name + " (packed, forced global)", outlier_frac=1e-5, early_rows=EARLY_ROWS)
+        rt = np.arange(n)
+        gate = oracle.dgate_rows(one, sl["Q"], sl["K"], sl["V"], sl["dO"], np.zeros_like(rt), rt)
+        check_close(to_f64(b.dgate[:, s:e]), gate.reshape(1, n), "dgate (packed, every token)", 5e-2, 5e-3)
