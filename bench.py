@@ -114,6 +114,25 @@ def make_workload(args, seed_offset=0):
     return cfg, rho, seed, d, logits
 
 
+def issued_tile_pairs(mask, L, W, shared=False, tile=128):
+    """Score elements the tensor cores really compute, (local, global): every (128-row tile, 128-key block) pair a launch
+    issues MMAs for counts whole (edge blocks are masked after the product, ragged tiles are padded with zero rows).
+    Local: the blocks between the first row's window start and the last row's diagonal; global: the blocks up to the
+    last row of each compact tile of 128 routed rows (up to its position - W - 1 with the shared-window flag)."""
+    T = tile
+    loc = glb = 0
+    for b in range(mask.shape[0]):
+        r0 = np.arange(0, L, T, dtype=np.int64)
+        r1 = np.minimum(r0 + T, L) - 1
+        loc += int((r1 // T - np.maximum(r0 - W, 0) // T + 1).sum())
+        t = np.nonzero(mask[b])[0].astype(np.int64)
+        if len(t):
+            last = t[np.minimum(np.arange(T - 1, len(t) + T - 1, T), len(t) - 1)]      # last row of each compact tile
+            bound = last - (W + 1 if shared else 0)
+            glb += int((bound[bound >= 0] // T + 1).sum())
+    return loc * T * T, glb * T * T
+
+
 def cpu_oracle_sample(cfg, seed, d, rows_per_head=96, key_span=2500, n_keys=8, backward=True, host=None):
     """The fp64 oracle on a bounded sample of the workload at its FULL length: `rows_per_head` random rows of the second
     half of the sequence (half of them routed when there are enough) in every head -- forward (s, a, o) and dQ -- and
@@ -405,20 +424,7 @@ def main():
         return pl, pg, pw
 
     def issued_pairs(mask, shared):
-        """Score elements the tensor cores really compute: every (128-row tile, 128-key block) pair a launch issues
-        MMAs for counts whole (edge blocks are masked after the product, ragged tiles are padded with zero rows)."""
-        T = 128
-        loc = glb = 0
-        for b in range(cfg.B):
-            r0 = np.arange(0, cfg.L, T, dtype=np.int64)
-            r1 = np.minimum(r0 + T, cfg.L) - 1
-            loc += int((r1 // T - np.maximum(r0 - cfg.W, 0) // T + 1).sum())
-            t = np.nonzero(mask[b])[0].astype(np.int64)
-            if len(t):
-                last = t[np.minimum(np.arange(T - 1, len(t) + T - 1, T), len(t) - 1)]      # last row of each compact tile
-                bound = last - (cfg.W + 1 if shared else 0)
-                glb += int((bound[bound >= 0] // T + 1).sum())
-        return loc * T * T, glb * T * T
+        return issued_tile_pairs(mask, cfg.L, cfg.W, shared)
 
     def step(profile=None):
         buf.route(kind, 0.0)
