@@ -11,10 +11,10 @@
  * Conventions shared by every call
  *   - Every pointer is a DEVICE pointer unless its comment says "host".  The caller owns all
  *     buffers, including the workspaces; the library allocates no device memory and never
- *     synchronises the stream (only l2a_workspace_status and l2a_step_host do).  State kept between
+ *     synchronises the stream (only l2a_workspace_status, l2a_step_host and l2a_step_host_wait do).  State kept between
  *     calls: per-device facts looked up once (SM count, kernel attributes); the fixed device array
  *     and its cached address of l2a_route_compact_static; the per-thread helper streams and events of
- *     l2a_step_host; the one-shot event registration of l2a_profile_next_call.
+ *     l2a_step_host / l2a_step_host_async; the one-shot event registration of l2a_profile_next_call.
  *   - Tensors are contiguous bf16:  Q, O, dO, dQ, S_save, A_c : [B, Lq, Hq, D]
  *                                   K, V, dK, dV              : [B, Lk, Hkv, D]
  *     D contiguous, base pointers 16-byte aligned.  D is 64 or 128.  Hq % Hkv == 0 (GQA: query
@@ -401,6 +401,23 @@ typedef struct l2a_device_io {
 
 l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a_device_io* dev,
                          int router_kind, float logit_threshold, void* stream);
+
+/*
+ * The same step, enqueued only: the call returns when its copies and kernels are queued, and l2a_step_host_wait
+ * blocks until every step enqueued by this host thread has delivered its results.  For a training loop that keeps
+ * two steps in flight on TWO sets of device tensors used alternately (`dev` of step i + 1 differs from that of
+ * step i and equals that of step i - 1): the uploads of step i + 1 then run under the kernels of step i and the
+ * downloads of step i under the kernels of step i + 1, so that in steady state a step costs its kernels only.
+ * Ordering the library provides: the uploads of a step wait for the kernels of the step before the previous one
+ * (the last user of the same device tensors), its kernels for that step's downloads; kernels of successive steps
+ * run in order on `stream`.  What the caller provides: at most two steps in flight between waits, alternating
+ * device sets as above, the same `stream` for every step, and host result buffers of a step that are not read
+ * before l2a_step_host_wait returns (successive steps may share them: they are written in step order).
+ * Results are those of l2a_step_host.
+ */
+l2a_status l2a_step_host_async(const l2a_params* p, const l2a_host_io* host, const l2a_device_io* dev,
+                               int router_kind, float logit_threshold, void* stream);
+l2a_status l2a_step_host_wait(void* stream);
 
 /*
  * l2a_route_compact without any caller-provided scratch (an addition of this library; the paper has

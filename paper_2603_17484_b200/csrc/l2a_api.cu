@@ -454,8 +454,43 @@ l2a_status l2a_profile_next_call(void* const* events, int n_events) {
   return L2A_OK;
 }
 
+// Helper streams and events of the host-buffer step, created once per host thread and device.
+namespace {
+struct StepAux {
+  int device = -1;
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr, up = nullptr, fwd = nullptr, phase[11] = {}, down = nullptr, chunk[8] = {};
+  // pipelined steps: kernels_done[k] / delivered[k] of the last two steps (k = step parity)
+  cudaEvent_t kernels_done[2] = {}, delivered[2] = {};
+  int n_async = 0;          // steps enqueued since the last wait
+};
+thread_local StepAux g_step_aux;
+}  // namespace
+
+static l2a_status step_host_impl(const l2a_params* p, const l2a_host_io* host, const l2a_device_io* dev,
+                                 int router_kind, float logit_threshold, void* stream, bool async);
+
 l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a_device_io* dev, int router_kind,
                          float logit_threshold, void* stream) {
+  return step_host_impl(p, host, dev, router_kind, logit_threshold, stream, false);
+}
+
+l2a_status l2a_step_host_async(const l2a_params* p, const l2a_host_io* host, const l2a_device_io* dev,
+                               int router_kind, float logit_threshold, void* stream) {
+  return step_host_impl(p, host, dev, router_kind, logit_threshold, stream, true);
+}
+
+l2a_status l2a_step_host_wait(void* stream) {
+  StepAux& aux = g_step_aux;
+  aux.n_async = 0;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return L2A_ERR_CUDA;
+  if (aux.device >= 0 && (cudaStreamSynchronize(aux.out) != cudaSuccess || cudaStreamSynchronize(aux.in) != cudaSuccess))
+    return L2A_ERR_CUDA;
+  return L2A_OK;
+}
+
+static l2a_status step_host_impl(const l2a_params* p, const l2a_host_io* host, const l2a_device_io* dev,
+                                 int router_kind, float logit_threshold, void* stream, bool async) {
   l2a_status st = check_params(p);
   if (st != L2A_OK) return st;
   if (!host || !dev) return L2A_ERR_INVALID_ARG;
@@ -482,12 +517,7 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
   // dO is uploaded while the forward runs, O is downloaded while the backward runs, dQ while the dK/dV kernel
   // runs (the backward computes dQ first for this reason); only dK and dV, the small results, leave after the
   // last kernel.  With pageable host memory the copies simply serialise.
-  struct Aux {
-    int device = -1;
-    cudaStream_t in = nullptr, out = nullptr;
-    cudaEvent_t start = nullptr, up = nullptr, fwd = nullptr, phase[11] = {}, down = nullptr, chunk[8] = {};
-  };
-  static thread_local Aux aux;
+  StepAux& aux = g_step_aux;
   int dev_id = 0;
   if (cudaGetDevice(&dev_id) != cudaSuccess) return L2A_ERR_CUDA;
   if (aux.device != dev_id) {
@@ -497,26 +527,47 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
     cudaEvent_t* evs[] = {&aux.start, &aux.up, &aux.fwd, &aux.down, &aux.phase[0], &aux.phase[1], &aux.phase[2],
                           &aux.phase[3], &aux.phase[4], &aux.phase[5], &aux.phase[6], &aux.phase[7], &aux.phase[8],
                           &aux.phase[9], &aux.phase[10], &aux.chunk[0], &aux.chunk[1], &aux.chunk[2],
-                          &aux.chunk[3], &aux.chunk[4], &aux.chunk[5], &aux.chunk[6], &aux.chunk[7]};
+                          &aux.chunk[3], &aux.chunk[4], &aux.chunk[5], &aux.chunk[6], &aux.chunk[7],
+                          &aux.kernels_done[0], &aux.kernels_done[1], &aux.delivered[0], &aux.delivered[1]};
     for (cudaEvent_t* e : evs)
       if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return L2A_ERR_CUDA;
     aux.device = dev_id;
+    aux.n_async = 0;
   }
 #define L2A_TRY(x) do { if ((x) != cudaSuccess) return L2A_ERR_CUDA; } while (0)
-  L2A_TRY(cudaEventRecord(aux.start, s));
-  L2A_TRY(cudaMemcpyAsync(dev->router, host->router, rb, cudaMemcpyHostToDevice, s));
+  // Blocking step: the uploads start behind whatever the caller had queued on `stream` before this call.  Pipelined
+  // step: they start behind the kernels of the step before the previous one (the last user of these device tensors),
+  // and this step's kernels behind that step's downloads; the router input rides the upload stream as well.
+  const int parity = aux.n_async & 1;
+  if (!async && aux.n_async > 0) return L2A_ERR_INVALID_ARG;   // pipelined steps pending: l2a_step_host_wait first
+  if (!async) {
+    L2A_TRY(cudaEventRecord(aux.start, s));
+    L2A_TRY(cudaMemcpyAsync(dev->router, host->router, rb, cudaMemcpyHostToDevice, s));
+  } else {
+    if (aux.n_async >= 2) {
+      L2A_TRY(cudaStreamWaitEvent(aux.in, aux.kernels_done[parity], 0));
+      L2A_TRY(cudaStreamWaitEvent(s, aux.delivered[parity], 0));
+    }
+    L2A_TRY(cudaMemcpyAsync(dev->router, host->router, rb, cudaMemcpyHostToDevice, aux.in));
+    L2A_TRY(cudaEventRecord(aux.start, aux.in));
+    L2A_TRY(cudaStreamWaitEvent(s, aux.start, 0));
+  }
   l2a_params q = *p;
   if (!bwd) q.flags &= ~L2A_FLAG_SAVE_FOR_BWD;
   const bool need_lse_loc = bwd || (q.flags & L2A_FLAG_SHARED_WINDOW);   // the fusion reads it back in the forward
   const int n_pairs = ceil_div(p->Lq, kRowsPerCta);
   constexpr int kChunks = 8;
-  const bool chunked = p->B == 1 && n_pairs >= 2 * kChunks &&
+  // A pipelined step that follows another one has its transfers hidden behind that step's kernels: it uploads whole
+  // tensors and runs one forward and one backward launch sequence instead of the row / key-block ranges, which exist
+  // to start early and to drain early and cost a few percent of kernel time.
+  const bool steady = async && aux.n_async > 0;
+  const bool chunked = !steady && p->B == 1 && n_pairs >= 2 * kChunks &&
                        !(p->flags & (L2A_FLAG_SKIP_LOCAL | L2A_FLAG_SKIP_GLOBAL | L2A_FLAG_GLOBAL_PHASE));
   if (chunked) {
     // One sequence: K, V and Q go up in eight row ranges on the upload stream (attention is causal: the queries of a
     // range need no later keys); Local Attention and then the Global Attention of the routed rows of a range start
     // as soon as it has landed, so only the first range's copy is exposed.  Results equal a single l2a_forward call.
-    L2A_TRY(cudaStreamWaitEvent(aux.in, aux.start, 0));
+    if (!async) L2A_TRY(cudaStreamWaitEvent(aux.in, aux.start, 0));
     const size_t row_bytes = (size_t)p->Hq * p->D * sizeof(bf16), krow_bytes = (size_t)p->Hkv * p->D * sizeof(bf16);
     int pair_edge[kChunks + 1];
     for (int c = 0; c <= kChunks; ++c) pair_edge[c] = (int)((int64_t)n_pairs * c / kChunks);
@@ -569,11 +620,16 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
       if (st != L2A_OK) return st;
     }
   } else {
-    L2A_TRY(cudaMemcpyAsync(dev->Q, host->Q, qb, cudaMemcpyHostToDevice, s));
-    L2A_TRY(cudaMemcpyAsync(dev->K, host->K, kb, cudaMemcpyHostToDevice, s));
-    L2A_TRY(cudaMemcpyAsync(dev->V, host->V, kb, cudaMemcpyHostToDevice, s));
+    cudaStream_t us = async ? aux.in : s;
+    L2A_TRY(cudaMemcpyAsync(dev->Q, host->Q, qb, cudaMemcpyHostToDevice, us));
+    L2A_TRY(cudaMemcpyAsync(dev->K, host->K, kb, cudaMemcpyHostToDevice, us));
+    L2A_TRY(cudaMemcpyAsync(dev->V, host->V, kb, cudaMemcpyHostToDevice, us));
+    if (async) {
+      L2A_TRY(cudaEventRecord(aux.chunk[0], aux.in));
+      L2A_TRY(cudaStreamWaitEvent(s, aux.chunk[0], 0));
+    }
     if (bwd) {   // dO rides the second stream, behind whatever the caller had queued before this call
-      L2A_TRY(cudaStreamWaitEvent(aux.in, aux.start, 0));
+      if (!async) L2A_TRY(cudaStreamWaitEvent(aux.in, aux.start, 0));
       L2A_TRY(cudaMemcpyAsync(dev->dO, host->dO, qb, cudaMemcpyHostToDevice, aux.in));
       L2A_TRY(cudaEventRecord(aux.up, aux.in));
     }
@@ -593,9 +649,10 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
     // With eleven phase events the backward runs as four key-block ranges; boundary 4 + 2 r says that the gradients
     // range r completes (dK, dV of its keys, dQ of the rows that only see keys up to its end) are final: they leave on
     // the download stream while the next range is computed, the last range's after the last kernel.
+    const int n_ev = steady ? 5 : 11;
     void* phase_events[11];
     for (int i = 0; i < 11; ++i) phase_events[i] = aux.phase[i];
-    st = l2a_profile_next_call(phase_events, 11);
+    st = l2a_profile_next_call(phase_events, n_ev);
     if (st != L2A_OK) return st;
     st = l2a_backward(&q, dev->Q, dev->K, dev->V, dev->d_mask, dev->q_idx, dev->n_routed, dev->prefix, dev->dO,
                       dev->S_save, dev->A_c, dev->lse_loc, dev->lse_glb, dev->dQ, dev->dK, dev->dV, nullptr,
@@ -603,7 +660,7 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
     if (st != L2A_OK) return st;
     int first[kMaxBwdRanges];
     const int n_kblocks = ceil_div(p->Lk, kTileN), n_tiles = ceil_div(p->Lq, kTileM);
-    const int n_ranges = bwd_ranges(n_kblocks, 11, first);
+    const int n_ranges = bwd_ranges(n_kblocks, n_ev, first);
     const size_t krow = (size_t)p->Hkv * p->D * sizeof(bf16), qrow = (size_t)p->Hq * p->D * sizeof(bf16);
     int64_t k_done = 0, q_done = 0;
     for (int r = 0; r < n_ranges; ++r) {
@@ -612,8 +669,8 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
       int64_t q_end = last ? p->Lq : (int64_t)dq_final_tiles(first[r + 1], p->q_pos_offset, n_tiles) * kTileM;
       if (k_end > p->Lk) k_end = p->Lk;
       if (q_end > p->Lq) q_end = p->Lq;
-      cudaStream_t cs = last ? s : aux.out;
-      if (!last) L2A_TRY(cudaStreamWaitEvent(aux.out, aux.phase[4 + 2 * r], 0));
+      cudaStream_t cs = (last && !async) ? s : aux.out;
+      if (!last || async) L2A_TRY(cudaStreamWaitEvent(aux.out, aux.phase[4 + 2 * r], 0));
       for (int b = 0; b < p->B; ++b) {
         const size_t kbase = (size_t)b * p->Lk * krow, qbase = (size_t)b * p->Lq * qrow;
         if (q_end > q_done)
@@ -632,6 +689,13 @@ l2a_status l2a_step_host(const l2a_params* p, const l2a_host_io* host, const l2a
       if (q_end > q_done) q_done = q_end;
       if (k_end > k_done) k_done = k_end;
     }
+  }
+  if (async) {
+    // nothing on `stream` waits for the downloads: the next step's kernels follow this step's directly
+    L2A_TRY(cudaEventRecord(aux.kernels_done[parity], s));
+    L2A_TRY(cudaEventRecord(aux.delivered[parity], aux.out));
+    ++aux.n_async;
+    return L2A_OK;
   }
   L2A_TRY(cudaEventRecord(aux.down, aux.out));
   L2A_TRY(cudaStreamWaitEvent(s, aux.down, 0));   // the caller's stream ends the step with every result delivered

@@ -31,7 +31,7 @@ EXPORTS = (
     "l2a_route_compact", "l2a_forward", "l2a_backward", "l2a_step_host", "l2a_profile_next_call",
     "l2a_route_compact_static", "l2a_router_logits", "l2a_decode_workspace_bytes", "l2a_decode",
     "l2a_backward_split", "l2a_router_backward", "l2a_forward_routed", "l2a_selftest_wait_timeout",
-    "l2a_forward_sets", "l2a_backward_sets", "l2a_pack_sequences",
+    "l2a_forward_sets", "l2a_backward_sets", "l2a_pack_sequences", "l2a_step_host_async", "l2a_step_host_wait",
 )
 
 
@@ -294,7 +294,7 @@ def _addr(t):
 
 
 def l2a_step_host(p, host: dict, bufs: "Buffers", router_kind=ROUTER_MASK_U8, logit_threshold=0.0, stream=None,
-                  check=True) -> int:
+                  check=True, pipelined=False) -> int:
     """Whole step from HOST tensors (dict with Q, K, V, router, O and, for a backward, dO, dQ, dK, dV):
     copies in, routes, runs forward (+ backward), copies the results out, synchronises."""
     h = HostIO(*[_addr(host.get(n)) for n in ("Q", "K", "V", "router", "dO", "O", "dQ", "dK", "dV")])
@@ -303,10 +303,23 @@ def l2a_step_host(p, host: dict, bufs: "Buffers", router_kind=ROUTER_MASK_U8, lo
     d = DeviceIO(*[_addr(getattr(bufs, n)) for n in names],
                  _addr(bufs.route_ws), bufs.route_ws.numel(), _addr(bufs.fwd_ws), bufs.fwd_ws.numel(),
                  _addr(bufs.bwd_ws), 0 if bufs.bwd_ws is None else bufs.bwd_ws.numel())
-    code = lib().l2a_step_host(ctypes.byref(p), ctypes.byref(h), ctypes.byref(d), ctypes.c_int(router_kind),
-                               ctypes.c_float(logit_threshold), _stream(stream))
+    fn = lib().l2a_step_host_async if pipelined else lib().l2a_step_host
+    code = fn(ctypes.byref(p), ctypes.byref(h), ctypes.byref(d), ctypes.c_int(router_kind),
+              ctypes.c_float(logit_threshold), _stream(stream))
     if check:
-        _check(code, "l2a_step_host")
+        _check(code, "l2a_step_host_async" if pipelined else "l2a_step_host")
+    return code
+
+
+def l2a_step_host_async(p, host: dict, bufs: "Buffers", router_kind=ROUTER_MASK_U8, logit_threshold=0.0, stream=None,
+                        check=True) -> int:
+    """The same step, enqueued only (two steps in flight on alternating Buffers; see include/l2a.h)."""
+    return l2a_step_host(p, host, bufs, router_kind, logit_threshold, stream, check, pipelined=True)
+
+
+def l2a_step_host_wait(stream=None) -> int:
+    code = lib().l2a_step_host_wait(_stream(stream))
+    _check(code, "l2a_step_host_wait")
     return code
 
 
