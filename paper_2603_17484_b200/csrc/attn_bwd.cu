@@ -184,10 +184,13 @@ struct BwdArgs {
 //   warp 18    : stages the row statistics of each query tile          warp 19 : idle
 //   warps 20-27: read every dQ(i) tile out of TMEM (one lane group and one half of the columns each) and add it into the
 //                fp32 accumulators: the reductions leave an SM at about 32 bytes per clock, and a warp that issues them
-//                stalls that long, so they are kept off the warps whose progress the tensor pipe waits for
+//                stalls that long, so they are kept off the warps whose progress the tensor pipe waits for.  A read-out
+//                warp takes its whole share (64 values per thread) into registers and releases the TMEM columns before
+//                its first reduction.
 // Registers: 896 threads start with 72 each (64512 in all, which is also all that setmaxnreg can redistribute: an
 // increase is served from what the CTA's own warps released); the service warpgroup goes down to 40, the read-out
-// warpgroups to 56, the compute warpgroups up to 88.
+// warpgroups stay at 72, the compute warpgroups go up to 80 -- which they fit because scores and dP^T leave TMEM sixteen
+// columns at a time.
 constexpr int kComputeWarps = 16;
 constexpr int kDkvThreads = 28 * 32;   // 896
 
@@ -255,9 +258,35 @@ struct ItemCursor {
 //         then dQ(i).
 //   Shared memory: K, V resident; Q and dO in two-stage rings; dS(i) (bf16, [key][query], swizzled like a TMA
 //   tile) -- the A operand of both dK += dS^T Q (read K-major) and dQ = dS K (read MN-major).
-//   MMA order per item i:  dV(i) | dQ(i) | S^T(i+1) | dK(i) | dP^T(i+1).  Two loops run through the order with
-//   slack: T: S^T -> P -> dV -> S^T and U: dP^T -> dS -> dQ -> read-out -> dP^T; dK(i) keeps the pipe busy while the
-//   read-out warps take dQ(i) out of TMEM and the compute warps start on item i+1.
+//   MMA order per item i:  dV(i) | S^T(i+1) | dQ(i) | dK(i) | dP^T(i+1).  S^T(i+1) does not depend on dS(i), so it is
+//   issued ahead of the wait for it: the compute warps find the next scores ready when they are done with dS(i).
+//   Two loops run through the order: T: S^T -> P -> dV -> S^T and U: dP^T -> dS -> dQ -> read-out -> dP^T; dK(i) keeps the
+//   pipe busy while the read-out warps take dQ(i) out of TMEM, which frees U well before their reductions are issued.
+
+// The reductions of one read-out warp: piece I of its 32 x D/2 share (4 columns each) goes to a byte offset from the
+// warp's base address that is a compile-time constant, so that all of them share one address register pair.
+template <int kBytes>
+__device__ __forceinline__ void red_add_v4(float* base, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("red.global.add.v4.f32 [%0+%5], {%1, %2, %3, %4};" ::"l"(base), "f"(__uint_as_float(a)),
+               "f"(__uint_as_float(b)), "f"(__uint_as_float(c)), "f"(__uint_as_float(d)), "n"(kBytes)
+               : "memory");
+}
+template <int D, int I>
+struct ReadOutReds {
+  static constexpr int kCols = D / 4;                 // columns per quarter of the accumulator layout
+  static constexpr int kCol = 4 * I;                  // relative to the warp's first column
+  static constexpr int kOff = ((kCol / kCols) * 4 * (8 * D) + ((kCol % kCols) / 4) * 128) * 4;
+  __device__ __forceinline__ static void run(float* base, const uint32_t (&v)[D / 64][32]) {
+    red_add_v4<kOff>(base, v[I / 8][4 * (I % 8)], v[I / 8][4 * (I % 8) + 1], v[I / 8][4 * (I % 8) + 2],
+                     v[I / 8][4 * (I % 8) + 3]);
+    ReadOutReds<D, I + 1>::run(base, v);
+  }
+};
+template <int D>
+struct ReadOutReds<D, D / 8> {
+  __device__ __forceinline__ static void run(float*, const uint32_t (&)[D / 64][32]) {}
+};
+
 template <int D>
 struct BwdSmem {
   static constexpr int kTileBytes = 128 * D * 2;
@@ -362,14 +391,13 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
   // register shares by warpgroup: every warp of a warpgroup executes the same setmaxnreg at the top of its role
   if (warp >= 20) {
     // ------------------------------------------------------------------ dQ read-out: TMEM -> fp32 accumulators
-    setmaxnreg_dec<56>();
+    setmaxnreg_dec<72>();
     // lane == query row of the item's tile; this warp owns the 32 rows of its lane group and one half of the D columns,
-    // taken 32 at a time: each 32 x 4 piece is one 512-byte reduction (accumulator layout: see above)
+    // read in one go: each 32 x 4 piece is then one 512-byte reduction (accumulator layout: see above)
     const int grp = warp & 3, half = (warp - 20) >> 2;
     const uint32_t lane_base = static_cast<uint32_t>(grp * 32) << 16;
     const int n_tiles = (a.Lq + kTileM - 1) / kTileM;
-    constexpr int kChunks = D / 32;     // read out 32 columns at a time: one TMEM load, eight reductions
-    constexpr int kCols = D / 4;        // columns per quarter in the accumulator layout
+    constexpr int kChunks = D / 32;     // 32-column TMEM loads of the whole tile; this warp takes half of them
     ItemCursor cur(plan, g * G);
     for (int i = 0; i < plan.total; ++i) {
       const int h = cur.h, glb = cur.glb(), tile = cur.tile();
@@ -379,28 +407,20 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
       acc += (((int64_t)b * a.Hq + h) * n_tiles + tile) * (int64_t)(kTileM * D) + lane * 4;
       if (!__all_sync(0xffffffffu, mbar_wait(&bar->dq_full, i & 1, abort_flag))) break;
       tc_fence_after();
+      // the warp's whole share (32 rows x D/2 columns) goes to registers first, so that the region is released before
+      // the first reduction is issued: the reductions leave the SM at about 32 bytes per clock and must not hold up
+      // dP^T(i+1)
+      uint32_t v[kChunks / 2][32];
 #pragma unroll
-      for (int cc = 0; cc < kChunks / 2; ++cc) {
-        const int ch = half * (kChunks / 2) + cc;
-        uint32_t v[32];
-        tmem_ld32(tmem + lane_base + 384 + ch * 32, v);
-        tmem_ld_wait();
-        if (cc == kChunks / 2 - 1) {
-          tc_fence_before();
-          mbar_arrive(&bar->u_free);       // everything is in registers: dP^T(i+1) may overwrite the columns
-        }
-        if (item_ok) {
-#pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            // columns 32 ch + 4 c .. + 3: quarter (32 ch + 4 c) / kCols, piece ((32 ch + 4 c) % kCols) / 4
-            const int col = 32 * ch + 4 * c;
-            float* dst = acc + ((col / kCols) * 4 + grp) * (8 * D) + ((col % kCols) / 4) * 128;
-            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(__uint_as_float(v[4 * c])),
-                         "f"(__uint_as_float(v[4 * c + 1])), "f"(__uint_as_float(v[4 * c + 2])),
-                         "f"(__uint_as_float(v[4 * c + 3]))
-                         : "memory");
-          }
-        }
+      for (int cc = 0; cc < kChunks / 2; ++cc) tmem_ld32(tmem + lane_base + 384 + (half * (kChunks / 2) + cc) * 32, v[cc]);
+      tmem_ld_wait();
+      tc_fence_before();
+      mbar_arrive(&bar->u_free);           // everything is in registers: dP^T(i+1) may overwrite the columns
+      if (item_ok) {
+        // this warp's columns start at (D / 2) * half, i.e. at quarter 2 * half of the accumulator layout; every further
+        // offset is a compile-time constant, so that the sixteen reductions share one address register pair
+        float* base = acc + ((2 * half) * 4 + grp) * (8 * D);
+        ReadOutReds<D, 0>::run(base, v);
       }
     }
   } else if (warp == 19) {
@@ -553,15 +573,16 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
         if (!mbar_spin_warp(&bar->p_full, i & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         issue_dV(i & 1, i == 0);
-        if (!mbar_spin_warp(&bar->ds_full, i & 1, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        issue_dQ();
         if (more) {
-          // S^T(i+1) overwrites P^T(i): dV(i) precedes it in issue order
+          // S^T(i+1) overwrites P^T(i): dV(i) precedes it in issue order.  It does not depend on dS(i), so it goes
+          // ahead of that wait: the compute warps find the next scores ready when they are done with dS(i)
           if (!mbar_spin_warp(&bar->q_full[(i + 1) & 1], ((i + 1) >> 1) & 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
           issue_S((i + 1) & 1);
         }
+        if (!mbar_spin_warp(&bar->ds_full, i & 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        issue_dQ();
         issue_dK(i & 1, i == 0);       // keeps the pipe busy while dQ(i) is read out
         if (more) {
           const int sn = (i + 1) & 1;
@@ -578,7 +599,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
     __syncwarp();
   } else {
     // ------------------------------------------------------------------ P^T, dS and epilogue
-    setmaxnreg_inc<88>();
+    setmaxnreg_inc<80>();
     const int q = warp >> 2;                           // query-column quarter of this warp
     const int kr = (warp & 3) * 32 + lane;             // key inside the block == TMEM lane
     const int kp = k0 + kr;
@@ -604,39 +625,45 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
       tc_fence_after();
       uint32_t pp[16];
       {
-        uint32_t sv[32];
-        tmem_ld32(s_addr, sv);
-        tmem_ld_wait();
-        // the element mask is needed only for the few tiles that straddle the causal diagonal or a window edge:
-        // two loop versions, so that the common one has no branches
-        if (!masked) {
+        const int w_eff = item_glb ? 0x3fffffff : a.window;
+        const int n_rows = item_glb ? n_c : a.Lq;
+        const int32_t* qi = a.q_idx + (int64_t)b * a.Lq;
+        // the scores come out of TMEM sixteen columns at a time (register budget of the compute warps)
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const float2 x = __ffma2_rn(make_float2(__uint_as_float(sv[2 * e]), __uint_as_float(sv[2 * e + 1])),
-                                        make_float2(a.scale_log2, a.scale_log2), make_float2(st[2 * e], st[2 * e + 1]));
-            pp[e] = pack_bf16(fast_exp2(x.x), fast_exp2(x.y));
-          }
-        } else {
-          const int w_eff = item_glb ? 0x3fffffff : a.window;
-          const int n_rows = item_glb ? n_c : a.Lq;
-          const int32_t* qi = a.q_idx + (int64_t)b * a.Lq;
+        for (int hh = 0; hh < 2; ++hh) {
+          uint32_t sv[16];
+          tmem_ld16(s_addr + hh * 16, sv);
+          tmem_ld_wait();
+          // the element mask is needed only for the few tiles that straddle the causal diagonal or a window edge:
+          // two loop versions, so that the common one has no branches
+          if (!masked) {
 #pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            int pos[2], lo[2];
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-              const int row = item_row0 + q * 32 + e + u;
-              const bool valid = row < n_rows;
-              const int token = valid ? (item_glb ? __ldg(&qi[row]) : row) : 0;
-              pos[u] = valid ? token - (item_glb ? a.vis_shift : 0) + a.q_pos_offset : -1;
-              lo[u] = pos[u] - w_eff;
-              if (valid && a.seq_bounds != nullptr) lo[u] = max(lo[u], __ldg(&a.seq_bounds[2 * token]));
+            for (int e8 = 0; e8 < 8; ++e8) {
+              const int e = hh * 8 + e8;
+              const float2 x = __ffma2_rn(make_float2(__uint_as_float(sv[2 * e8]), __uint_as_float(sv[2 * e8 + 1])),
+                                          make_float2(a.scale_log2, a.scale_log2), make_float2(st[2 * e], st[2 * e + 1]));
+              pp[e] = pack_bf16(fast_exp2(x.x), fast_exp2(x.y));
             }
-            float p0 = fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, st[e]));
-            float p1 = fast_exp2(fmaf(__uint_as_float(sv[e + 1]), a.scale_log2, st[e + 1]));
-            p0 = (kp <= pos[0] && kp >= lo[0]) ? p0 : 0.f;
-            p1 = (kp <= pos[1] && kp >= lo[1]) ? p1 : 0.f;
-            pp[e >> 1] = pack_bf16(p0, p1);
+          } else {
+#pragma unroll
+            for (int e16 = 0; e16 < 16; e16 += 2) {
+              const int e = hh * 16 + e16;
+              int pos[2], lo[2];
+#pragma unroll
+              for (int u = 0; u < 2; ++u) {
+                const int row = item_row0 + q * 32 + e + u;
+                const bool valid = row < n_rows;
+                const int token = valid ? (item_glb ? __ldg(&qi[row]) : row) : 0;
+                pos[u] = valid ? token - (item_glb ? a.vis_shift : 0) + a.q_pos_offset : -1;
+                lo[u] = pos[u] - w_eff;
+                if (valid && a.seq_bounds != nullptr) lo[u] = max(lo[u], __ldg(&a.seq_bounds[2 * token]));
+              }
+              float p0 = fast_exp2(fmaf(__uint_as_float(sv[e16]), a.scale_log2, st[e]));
+              float p1 = fast_exp2(fmaf(__uint_as_float(sv[e16 + 1]), a.scale_log2, st[e + 1]));
+              p0 = (kp <= pos[0] && kp >= lo[0]) ? p0 : 0.f;
+              p1 = (kp <= pos[1] && kp >= lo[1]) ? p1 : 0.f;
+              pp[e >> 1] = pack_bf16(p0, p1);
+            }
           }
         }
       }
@@ -644,7 +671,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
       tmem_st_wait();
       tc_fence_before();
       mbar_arrive(&bar->p_full);
-      // Delta of the same rows, again ahead of the wait; after this the statistics slot may be refilled
+      // -Delta of the same rows, again ahead of the wait; after this the statistics slot may be refilled
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         const float4 v = lds128(st_base + (128 + q * 32 + c * 4) * 4);
@@ -654,14 +681,18 @@ bwd_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUt
       if (!__all_sync(0xffffffffu, mbar_wait(&bar->dp_full, i & 1, abort_flag))) { ok = false; break; }
       tc_fence_after();
       uint32_t pd[16];
-      {
-        uint32_t dv[32];
-        tmem_ld32(dp_addr, dv);
+      // dP^T comes out of TMEM sixteen columns at a time: with the 32 statistics and the 16 packed probabilities live,
+      // a 32-column load would not fit the compute warps' 80 registers
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        uint32_t dv[16];
+        tmem_ld16(dp_addr + hh * 16, dv);
         tmem_ld_wait();
 #pragma unroll
-        for (int e = 0; e < 16; ++e) {
+        for (int e8 = 0; e8 < 8; ++e8) {
+          const int e = hh * 8 + e8;
           // dS uses the bf16-rounded P, the same value the dV product sees; st[] holds -Delta
-          const float2 t = __fadd2_rn(make_float2(__uint_as_float(dv[2 * e]), __uint_as_float(dv[2 * e + 1])),
+          const float2 t = __fadd2_rn(make_float2(__uint_as_float(dv[2 * e8]), __uint_as_float(dv[2 * e8 + 1])),
                                       make_float2(st[2 * e], st[2 * e + 1]));
           const float2 ds = __fmul2_rn(make_float2(bf16lo_to_f32(pp[e]), bf16hi_to_f32(pp[e])), t);
           pd[e] = pack_bf16(ds.x, ds.y);
