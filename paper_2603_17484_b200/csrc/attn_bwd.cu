@@ -271,12 +271,16 @@ __device__ __forceinline__ void red_add_v4(float* base, uint32_t a, uint32_t b, 
                "f"(__uint_as_float(b)), "f"(__uint_as_float(c)), "f"(__uint_as_float(d)), "n"(kBytes)
                : "memory");
 }
+constexpr int kRedSpacingClk = 32;      // least distance between two reductions of a read-out warp
 template <int D, int I>
 struct ReadOutReds {
   static constexpr int kCols = D / 4;                 // columns per quarter of the accumulator layout
   static constexpr int kCol = 4 * I;                  // relative to the warp's first column
   static constexpr int kOff = ((kCol / kCols) * 4 * (8 * D) + ((kCol % kCols) / 4) * 128) * 4;
   __device__ __forceinline__ static void run(float* base, const uint32_t (&v)[D / 64][32]) {
+    // spaced out: reductions issued back to back fill the queue of the memory pipe, and the compute warps' shared-memory
+    // loads and stores (row statistics, dS) wait behind them; the read-out warps have most of an item's time to spare
+    { const long long t0 = clock64(); while (clock64() - t0 < kRedSpacingClk) __nanosleep(16); }
     red_add_v4<kOff>(base, v[I / 8][4 * (I % 8)], v[I / 8][4 * (I % 8) + 1], v[I / 8][4 * (I % 8) + 2],
                      v[I / 8][4 * (I % 8) + 3]);
     ReadOutReds<D, I + 1>::run(base, v);
