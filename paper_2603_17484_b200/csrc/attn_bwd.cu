@@ -271,7 +271,9 @@ __device__ __forceinline__ void red_add_v4(float* base, uint32_t a, uint32_t b, 
                "f"(__uint_as_float(b)), "f"(__uint_as_float(c)), "f"(__uint_as_float(d)), "n"(kBytes)
                : "memory");
 }
-constexpr int kRedSpacingClk = 32;      // least distance between two reductions of a read-out warp
+// Least distance between two reductions of a read-out warp, in SM clocks (polled: a sleep is too coarse).  Sixteen
+// reductions then take about 1800 clocks of an item's 4000 or more; 96 to 128 measure the same, 64 and 160 are slower.
+constexpr int kRedSpacingClk = 112;
 template <int D, int I>
 struct ReadOutReds {
   static constexpr int kCols = D / 4;                 // columns per quarter of the accumulator layout
@@ -280,7 +282,7 @@ struct ReadOutReds {
   __device__ __forceinline__ static void run(float* base, const uint32_t (&v)[D / 64][32]) {
     // spaced out: reductions issued back to back fill the queue of the memory pipe, and the compute warps' shared-memory
     // loads and stores (row statistics, dS) wait behind them; the read-out warps have most of an item's time to spare
-    { const long long t0 = clock64(); while (clock64() - t0 < kRedSpacingClk) __nanosleep(16); }
+    { const long long t0 = clock64(); while (clock64() - t0 < kRedSpacingClk) { } }
     red_add_v4<kOff>(base, v[I / 8][4 * (I % 8)], v[I / 8][4 * (I % 8) + 1], v[I / 8][4 * (I % 8) + 2],
                      v[I / 8][4 * (I % 8) + 3]);
     ReadOutReds<D, I + 1>::run(base, v);
