@@ -38,7 +38,7 @@ KERNELS_PER_STEP = 11  # route: count, scan | fwd: gather, local, global | bwd: 
 FWD_PHASES = ("gather_q", "attn_fwd_local", "attn_fwd_global")
 BWD_PHASES = ("gather_q_dO", "bwd_delta_zero", "bwd", "bwd_dq_merge")
 # DRAM read + write over algorithmic bytes of a launch, from the ncu captures of the 32K case (profiles/)
-TRAFFIC_RATIO = {"bwd": 1.17, "attn_fwd_local": 0.94, "attn_fwd_global": 1.17}
+TRAFFIC_RATIO = {"bwd": 1.15, "attn_fwd_local": 0.94, "attn_fwd_global": 1.17}
 
 
 def measured_peaks():
