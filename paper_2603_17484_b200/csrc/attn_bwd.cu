@@ -15,7 +15,7 @@
 //                      the G query heads, then the compact routed tiles from the first one at or after the block.
 //                      dK, dV accumulate in TMEM (no atomics, one bf16 store); the scores are built transposed (keys
 //                      on TMEM lanes) so that P^T feeds dV straight from TMEM; dQ(i) = dS(i) K is a fresh tile per
-//                      item that the compute warps add into fp32 accumulators in global memory.
+//                      item that dedicated read-out warps add into fp32 accumulators in global memory.
 //   dq_merge_kernel  : dQ = scale * (local accumulator + routed rows' global accumulator), rounded to bf16 once.
 #include "l2a_common.cuh"
 #include "sm100_prims.cuh"
@@ -247,7 +247,7 @@ struct ItemCursor {
 
 // ================================================================================================
 // Five-GEMM backward kernel: the key/value-stationary kernel above plus the fifth GEMM, dQ(i) = dS(i) K, so that
-// S and dP are computed once per tile pair.  dQ(i) is a fresh 128 x D accumulator per item; the compute warps read
+// S and dP are computed once per tile pair.  dQ(i) is a fresh 128 x D accumulator per item; the read-out warps take
 // it out (lane = query row) and add it into an fp32 accumulator in global memory whose layout is private to this
 // file: per (batch, head, 128-row tile) one block of 128 x D floats ordered [warp 16][piece D/16][lane 32][4], so
 // that every red.global.add.v4.f32 of a warp covers 512 contiguous bytes.  Local items add into the accumulator
